@@ -1,0 +1,212 @@
+/*
+ * rfast.h -- C ABI of the R-FAST activation engine (one CUDA device, sm_100a).
+ *
+ * The engine simulates n workers running R-FAST (Robust Fully-Asynchronous Stochastic
+ * Gradient Tracking) on one GPU.  The problem is the paper's eq. (1): min_x sum_i f_i(x)
+ * over n workers that exchange packets over two graphs, G_R = G(W) with W row-stochastic
+ * (consensus, "pull") and G_C = G(A) with A column-stochastic (tracking, "push"), sharing a
+ * root (Assumptions 1-2).  Asynchrony is data: a schedule says which nodes are active in
+ * each round and, for every packet, whether it is lost or how late it becomes usable
+ * (Algorithm 2, step S.0; Assumption 3).
+ *
+ * Conventions
+ *   - Every call returns an int status: RFAST_OK or a negative RFAST_E* code.  Nothing
+ *     throws, aborts or prints.  rfast_last_error() returns a text for the last failure.
+ *   - All pointers in rfast_problem / rfast_schedule are HOST pointers owned by the caller;
+ *     the library copies what it needs before the call returns.  Output buffers of
+ *     rfast_read_state are HOST pointers owned by the caller.
+ *   - The handle owns all device memory; rfast_destroy frees it.
+ *   - All device work is enqueued on the CUDA stream given at create time (a cudaStream_t
+ *     passed as void*; NULL = the legacy default stream).  One handle is not thread-safe.
+ *   - Node ids are 0-based.  Edge (j, i) of G(M) exists iff M_ij > 0; then j sends to i
+ *     (Section III-A).  Graphs are given by receiver (CSR over receivers).
+ *   - There is no CPU fallback: without a CUDA device rfast_create fails with RFAST_ECUDA.
+ */
+#ifndef RFAST_H
+#define RFAST_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RFAST_OK         0
+#define RFAST_EINVAL   (-1)  /* bad argument / size mismatch */
+#define RFAST_EGRAPH   (-2)  /* Assumption 1 or 2 violated */
+#define RFAST_ESCHED   (-3)  /* inconsistent schedule arrays */
+#define RFAST_ENOMEM   (-4)  /* host or device allocation failed */
+#define RFAST_ECUDA    (-5)  /* CUDA runtime error (text in rfast_last_error) */
+#define RFAST_ETIMEOUT (-6)  /* a bounded device-side wait ran out */
+#define RFAST_ESTATE   (-7)  /* call not valid in this state (e.g. run past the schedule) */
+
+typedef struct rfast_ctx rfast_ctx;
+
+/* Weight matrix M (W or A) by receiver.  Row i lists the in-neighbours of i:
+ * col[rowptr[i] .. rowptr[i+1]) are sender ids j in strictly ascending order, j != i, and
+ * w[e] = M[i][col[e]] > 0.  diag[i] = M[i][i] > 0 (Assumption 1 i). */
+typedef struct rfast_graph {
+    int32_t        n_edges;
+    const int32_t* rowptr;   /* [n+1] */
+    const int32_t* col;      /* [n_edges] */
+    const float*   w;        /* [n_edges] */
+    const float*   diag;     /* [n] */
+} rfast_graph;
+
+/* Local objectives f_i.  A minibatch gradient is the mean over the B sampled rows of node i's
+ * shard; each f_i carries its own (l2/2)||x||^2.  Parameter layouts (x is one flat vector):
+ *   QUAD_DIAG        f_i(x) = 0.5 || d_i .* (x - b_i) ||^2, deterministic, element-wise
+ *   LEAST_SQUARES    f_i(x) = 1/(2B) sum_k (a_k.x - y_k)^2;  batch = 0 means the whole shard
+ *   SOFTMAX          x = [W (C x F, row c = class c) | bias (C)], cross-entropy
+ *   MLP              x = [W1 (H x F) | b1 (H) | W2 (C x H) | b2 (C)], hidden = relu(W1 a + b1),
+ *                    cross-entropy; operands of the matrix products are rounded to bf16
+ *                    (round-to-nearest-even from fp32), accumulation in fp32
+ *   LOGISTIC_SPARSE  f_i(x) = 1/B sum_k log(1 + exp(-y_k a_k.x)), y in {-1,+1}, a_k sparse */
+enum {
+    RFAST_MODEL_QUAD_DIAG       = 0,
+    RFAST_MODEL_LEAST_SQUARES   = 1,
+    RFAST_MODEL_SOFTMAX         = 2,
+    RFAST_MODEL_MLP             = 3,
+    RFAST_MODEL_LOGISTIC_SPARSE = 4
+};
+
+typedef struct rfast_problem {
+    int32_t     n;            /* workers */
+    int32_t     root;         /* a common root of G(W) and G(A^T) (Assumption 2) */
+    int64_t     p;            /* dimension of x */
+    float       alpha;        /* constant step size gamma (Algorithm 1, S1) */
+    float       l2;           /* coefficient of the (l2/2)||x||^2 term in every f_i */
+    rfast_graph G_R;          /* W, row-stochastic    */
+    rfast_graph G_C;          /* A, column-stochastic */
+    int32_t     model;        /* RFAST_MODEL_* */
+    int32_t     batch;        /* B rows per activation (0: QUAD_DIAG, or whole shard for LEAST_SQUARES) */
+    int32_t     rows;         /* rows in every node's shard (0 for QUAD_DIAG) */
+    int32_t     n_features;   /* F (LEAST_SQUARES: F = p; LOGISTIC_SPARSE: F = p) */
+    int32_t     n_classes;    /* C (SOFTMAX, MLP) */
+    int32_t     n_hidden;     /* H (MLP) */
+    const float*   quad_d;    /* [n][p]            QUAD_DIAG */
+    const float*   quad_b;    /* [n][p]            QUAD_DIAG */
+    const float*   feat;      /* [n][rows][F]      dense features */
+    const float*   target;    /* [n][rows]         LEAST_SQUARES */
+    const int32_t* label;     /* [n][rows]         class id (SOFTMAX, MLP) or -1/+1 (LOGISTIC_SPARSE) */
+    const int64_t* sp_rowptr; /* [n*rows+1]        LOGISTIC_SPARSE, CSR over all shards, */
+    const int32_t* sp_col;    /*                   columns strictly ascending inside a row */
+    const float*   sp_val;
+    const float*   x0;        /* [n][p] initial iterates, or NULL for zeros */
+} rfast_problem;
+
+/* Raw schedule (value independent).  Round r activates the nodes
+ * act_node[act_ptr[r] .. act_ptr[r+1]) (strictly ascending).  Every activation is an
+ * "event"; events are numbered in array order.  All members of a round read the state and
+ * packets as of the start of the round.
+ * send_r / send_c hold one code per (event, out-edge of its node) for G_R / G_C, events in
+ * order, the out-edges of a node by ascending receiver id:  -1 = packet lost;  d >= 0 = the
+ * packet sent in round r is usable from round r + 1 + d on.  A receiver always uses, per
+ * in-edge, the packet with the largest sender stamp among those usable (Algorithm 1, S2).
+ * batch_idx: minibatch row indices into the node's shard, B per sample: first the initial
+ * samples zeta_i^0 of nodes 0..n-1 (used for z_i^0 = grad f_i(x_i^0; zeta_i^0)), then one
+ * sample per event.  Ignored (may be NULL) when the problem's batch is 0. */
+typedef struct rfast_schedule {
+    int32_t        K;
+    const int32_t* act_ptr;     /* [K+1] */
+    const int32_t* act_node;    /* [act_ptr[K]] */
+    int64_t        n_send_r;
+    const int8_t*  send_r;      /* [n_send_r] */
+    int64_t        n_send_c;
+    const int8_t*  send_c;      /* [n_send_c] */
+    int64_t        n_batch_idx;
+    const int32_t* batch_idx;   /* [(n + events) * B] */
+} rfast_schedule;
+
+/* Views for rfast_read_state.  Float views are fp32 row-major, unpadded. */
+enum {
+    RFAST_STATE_X            = 0,  /* float [n][p]     x_i                                        */
+    RFAST_STATE_Y            = 1,  /* float [n][p]     tracker z_i (the "y" of push-pull methods)  */
+    RFAST_STATE_G_LAST       = 2,  /* float [n][p]     remembered sample gradient                  */
+    RFAST_STATE_RHO_LATEST   = 3,  /* float [|E_C|][p] sender running sums rho, G_C edge order      */
+    RFAST_STATE_RHO_BUF      = 4,  /* float [|E_C|][p] receiver buffers rho~, G_C edge order        */
+    RFAST_STATE_T_LOCAL      = 5,  /* int32 [n]        local counters t_i after the rounds run      */
+    RFAST_STATE_USED_TAU_V   = 6,  /* int32 per (event, in-edge of G_R): stamp mixed in at S2a,     */
+                                   /*       whole loaded schedule, events in order                  */
+    RFAST_STATE_USED_TAU_RHO = 7,  /* int32 per (event, in-edge of G_C): stamp consumed at S2b      */
+    RFAST_STATE_TAU_V_END    = 8,  /* int32 [|E_R|]    tau_v at the end of the loaded schedule      */
+    RFAST_STATE_TAU_RHO_END  = 9,  /* int32 [|E_C|]    tau_rho at the end of the loaded schedule    */
+    RFAST_STATE_ROUND        = 10  /* int32 [1]        rounds run so far                            */
+};
+
+/* Counters for rfast_query. */
+enum {
+    RFAST_Q_ROUND          = 0,  /* rounds run so far */
+    RFAST_Q_EVENTS_TOTAL   = 1,  /* activation events in the loaded schedule */
+    RFAST_Q_EVENTS_RUN     = 2,  /* activation events run so far */
+    RFAST_Q_LAUNCHES       = 3,  /* kernels launched by rfast_run since create */
+    RFAST_Q_BYTES_RUN      = 4,  /* algorithmic bytes of the rounds run since the last reset:     */
+                                 /* every fp32 stream the compiled schedule makes a kernel read  */
+                                 /* or write, 4 bytes per coordinate                             */
+    RFAST_Q_V_SLOTS        = 5,  /* version rows allocated for v packets   */
+    RFAST_Q_RHO_SLOTS      = 6,  /* version rows allocated for rho packets */
+    RFAST_Q_DEVICE_BYTES   = 7,  /* device memory held by the handle */
+    RFAST_Q_N_USED_TAU_V   = 8,  /* element count of RFAST_STATE_USED_TAU_V   */
+    RFAST_Q_N_USED_TAU_RHO = 9,  /* element count of RFAST_STATE_USED_TAU_RHO */
+    RFAST_Q_BYTES_TOTAL    = 10  /* algorithmic bytes of the whole loaded schedule */
+};
+
+/* Problem statement -> device (eq. (1), Assumptions 1-2).  Validates Assumption 1
+ * (positive diagonal, W rows and A columns sum to 1 within 1e-5) and Assumption 2 (root
+ * reaches every node along G(W) and along G(A^T)); RFAST_EGRAPH otherwise.  Copies the
+ * shards to the device and sets x = x0, v = rho = rho~ = 0, t = 0 (initialisation line of
+ * Algorithm 1).  The trackers z_i^0 = grad f_i(x_i^0; zeta_i^0) need the initial samples
+ * and are set by rfast_load_schedule.  *out is NULL on failure. */
+int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out);
+
+/* Compiles a schedule (Algorithm 2, S.0) for the handle and resets the state to the
+ * initial one (round 0).  Host side, integers only: for every event and in-edge the stamp
+ * that is consumed (tau_v, tau_rho of Algorithm 1, i.e. the delays d_v, d_rho of
+ * Algorithm 2), then the lifetime of every packet version and a version row for each.
+ * Uploads the per-round descriptors.  RFAST_ESCHED if the arrays are inconsistent (sizes,
+ * order, ids, codes < -1). */
+int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s);
+
+/* Runs the next `rounds` rounds: for every active node S1 (v = x - alpha z), S2a (mix over
+ * G_R), the sample gradient at the new x, S2b/S2c (tracking over G_C with the running sums
+ * rho and the buffers rho~), S3/S4/S5 as compiled (Algorithm 1).  Asynchronous unless
+ * sync != 0.  RFAST_ESTATE without a schedule or past its end. */
+int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync);
+
+/* Stream-ordered copy of one view into a caller-owned HOST buffer of exactly `bytes` bytes
+ * (RFAST_EINVAL on mismatch); returns after the copy has completed. */
+int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes);
+
+/* Back to the initial state of the loaded schedule (x0, z^0, zero packets, round 0). */
+int rfast_reset(rfast_ctx* ctx);
+
+/* A counter (>= 0), or a negative status for an unknown id / NULL handle. */
+int64_t rfast_query(rfast_ctx* ctx, int what);
+
+/* Waits for the handle's stream; reports a pending asynchronous error. */
+int rfast_sync(rfast_ctx* ctx);
+
+/* Host-only companion of rfast_load_schedule (needs no CUDA device): compiles the schedule
+ * for the two graphs of `prob` (only n, root, batch, rows, model, G_R, G_C are read) and
+ * writes the integer artefacts into caller-owned HOST arrays, any of which may be NULL:
+ *   used_tau_v   [sum over events of indeg_R(node)]   stamp mixed in per (event, in-edge)
+ *   used_tau_rho [sum over events of indeg_C(node)]   stamp consumed per (event, in-edge)
+ *   v_ver        [events][3]       per v packet version:   row (-1: never leaves the node),
+ *   rho_ver      [n_send_c][3]     per rho packet version: write round, last round read
+ *   counts       [4]               v rows, rho rows, events, algorithmic floats per coordinate
+ * Two versions may share a row only if the earlier one is last read strictly before the round
+ * the later one is written (or, for rho, the later one is the same sender's in-place update). */
+int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s,
+                       int32_t* used_tau_v, int32_t* used_tau_rho,
+                       int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
+                       char* err, size_t err_len);
+
+void        rfast_destroy(rfast_ctx* ctx);
+const char* rfast_last_error(const rfast_ctx* ctx);   /* ctx may be NULL: last create error */
+const char* rfast_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RFAST_H */

@@ -1,0 +1,372 @@
+// Host-side schedule compiler: integers only.
+//
+// From the raw schedule (who is active when; which packets are lost or late) it derives what
+// Algorithm 1 calls tau_v / tau_rho -- per activation and in-edge, the largest stamp among the
+// packets usable by then -- which is the same information as the delays d_v, d_rho that
+// Algorithm 2 picks in step S.0.  Every packet payload that some later activation reads is a
+// "version"; the compiler computes each version's lifetime and gives it a row in a pool, so
+// that the kernels find a delayed payload by row id and a stale payload survives the sender's
+// later overwrites without any copy.
+#include <algorithm>
+#include <climits>
+#include <cmath>
+#include <cstdio>
+
+#include "rfast_internal.h"
+
+namespace rfast {
+
+static int fail(std::string& err, int code, const char* fmt, long long a = 0, long long b = 0,
+                long long c = 0) {
+    char buf[256];
+    std::snprintf(buf, sizeof buf, fmt, a, b, c);
+    err = buf;
+    return code;
+}
+
+int build_host_graph(const rfast_graph& g, int n, bool row_stochastic, HostGraph& H,
+                     std::string& err) {
+    if (n <= 0 || g.n_edges < 0 || !g.rowptr || !g.diag || (g.n_edges > 0 && (!g.col || !g.w)))
+        return fail(err, RFAST_EINVAL, "graph: null array or bad size");
+    H.n = n;
+    H.E = g.n_edges;
+    H.rowptr.assign(g.rowptr, g.rowptr + n + 1);
+    if (H.rowptr[0] != 0 || H.rowptr[n] != H.E)
+        return fail(err, RFAST_EGRAPH, "graph: rowptr must run from 0 to n_edges");
+    H.col.assign(g.col, g.col + H.E);
+    H.w.assign(g.w, g.w + H.E);
+    H.diag.assign(g.diag, g.diag + n);
+    H.recv.resize(H.E);
+    for (int i = 0; i < n; ++i) {
+        if (H.rowptr[i + 1] < H.rowptr[i])
+            return fail(err, RFAST_EGRAPH, "graph: rowptr decreases at node %lld", i);
+        if (!(H.diag[i] > 0.f))
+            return fail(err, RFAST_EGRAPH, "Assumption 1: diagonal entry of node %lld not positive", i);
+        for (int e = H.rowptr[i]; e < H.rowptr[i + 1]; ++e) {
+            int j = H.col[e];
+            if (j < 0 || j >= n || j == i)
+                return fail(err, RFAST_EGRAPH, "graph: bad sender %lld in row %lld", j, i);
+            if (e > H.rowptr[i] && H.col[e - 1] >= j)
+                return fail(err, RFAST_EGRAPH, "graph: senders of row %lld not strictly ascending", i);
+            if (!(H.w[e] > 0.f))
+                return fail(err, RFAST_EGRAPH, "Assumption 1: weight of edge %lld not positive", e);
+            H.recv[e] = i;
+        }
+    }
+    // Assumption 1 ii): W 1 = 1 (rows), 1^T A = 1^T (columns)
+    std::vector<double> sum(n);
+    for (int i = 0; i < n; ++i) sum[i] = H.diag[i];
+    for (int e = 0; e < H.E; ++e) sum[row_stochastic ? H.recv[e] : H.col[e]] += H.w[e];
+    for (int i = 0; i < n; ++i)
+        if (std::fabs(sum[i] - 1.0) > 1e-5)
+            return fail(err, RFAST_EGRAPH,
+                        row_stochastic ? "Assumption 1: row %lld of W does not sum to 1"
+                                       : "Assumption 1: column %lld of A does not sum to 1", i);
+    // sender-side lists, receivers ascending
+    H.optr.assign(n + 1, 0);
+    for (int e = 0; e < H.E; ++e) H.optr[H.col[e] + 1]++;
+    for (int i = 0; i < n; ++i) H.optr[i + 1] += H.optr[i];
+    H.oeid.resize(H.E);
+    H.opos.resize(H.E);
+    std::vector<int> fill(H.optr.begin(), H.optr.end() - 1);
+    for (int e = 0; e < H.E; ++e) {           // edge ids ascend with the receiver
+        int j = H.col[e];
+        H.opos[e] = fill[j] - H.optr[j];
+        H.oeid[fill[j]++] = e;
+    }
+    return RFAST_OK;
+}
+
+// Assumption 2: the root reaches every node along G(W) and along G(A^T).
+int check_roots(const HostGraph& R, const HostGraph& C, int root, std::string& err) {
+    const int n = R.n;
+    if (root < 0 || root >= n) return fail(err, RFAST_EINVAL, "root %lld out of range", root);
+    std::vector<char> seen(n, 0);
+    std::vector<int> todo;
+    auto bfs = [&](bool along_W) {
+        std::fill(seen.begin(), seen.end(), 0);
+        todo.assign(1, root);
+        seen[root] = 1;
+        int cnt = 1;
+        while (!todo.empty()) {
+            int u = todo.back();
+            todo.pop_back();
+            if (along_W) {                       // u sends to the receivers of its out-edges
+                for (int k = R.optr[u]; k < R.optr[u + 1]; ++k) {
+                    int v = R.recv[R.oeid[k]];
+                    if (!seen[v]) { seen[v] = 1; ++cnt; todo.push_back(v); }
+                }
+            } else {                             // G(A^T): u -> j whenever A_uj > 0
+                for (int e = C.rowptr[u]; e < C.rowptr[u + 1]; ++e) {
+                    int v = C.col[e];
+                    if (!seen[v]) { seen[v] = 1; ++cnt; todo.push_back(v); }
+                }
+            }
+        }
+        return cnt;
+    };
+    if (bfs(true) != n)
+        return fail(err, RFAST_EGRAPH, "Assumption 2: node %lld is not a root of a spanning tree of G(W)", root);
+    if (bfs(false) != n)
+        return fail(err, RFAST_EGRAPH, "Assumption 2: node %lld is not a root of a spanning tree of G(A^T)", root);
+    return RFAST_OK;
+}
+
+namespace {
+struct Pend { int arrival, stamp; };
+
+// Largest usable stamp on one edge at round r; drops what has arrived from the pending list.
+inline int deliver(std::vector<Pend>& q, int r, int tau) {
+    size_t keep = 0;
+    for (size_t k = 0; k < q.size(); ++k) {
+        if (q[k].arrival <= r) tau = std::max(tau, q[k].stamp);
+        else q[keep++] = q[k];
+    }
+    q.resize(keep);
+    return tau;
+}
+}  // namespace
+
+int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedule* s, int batch,
+                     int rows, const ModelTraffic& mt, Compiled& out, std::string& err) {
+    const int n = R.n;
+    if (!s || s->K < 0 || !s->act_ptr) return fail(err, RFAST_ESCHED, "schedule: null or K < 0");
+    const int K = s->K;
+    if (s->act_ptr[0] != 0) return fail(err, RFAST_ESCHED, "schedule: act_ptr[0] != 0");
+    for (int r = 0; r < K; ++r)
+        if (s->act_ptr[r + 1] < s->act_ptr[r])
+            return fail(err, RFAST_ESCHED, "schedule: act_ptr decreases at round %lld", r);
+    const int64_t nE = s->act_ptr[K];
+    if (nE > 0 && !s->act_node) return fail(err, RFAST_ESCHED, "schedule: act_node is null");
+    Compiled c;
+    c.K = K;
+    c.n_events = nE;
+    c.act_ptr.assign(s->act_ptr, s->act_ptr + K + 1);
+    c.act_node.assign(s->act_node, s->act_node + nE);
+    c.in_r_off.assign(nE + 1, 0);
+    c.in_c_off.assign(nE + 1, 0);
+    c.out_r_off.assign(nE + 1, 0);
+    c.out_c_off.assign(nE + 1, 0);
+    for (int r = 0; r < K; ++r)
+        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+            int i = c.act_node[ev];
+            if (i < 0 || i >= n) return fail(err, RFAST_ESCHED, "schedule: node id %lld out of range (event %lld)", i, ev);
+            if (ev > c.act_ptr[r] && c.act_node[ev - 1] >= i)
+                return fail(err, RFAST_ESCHED, "schedule: nodes of round %lld not strictly ascending", r);
+            c.in_r_off[ev + 1] = c.in_r_off[ev] + R.indeg(i);
+            c.in_c_off[ev + 1] = c.in_c_off[ev] + C.indeg(i);
+            c.out_r_off[ev + 1] = c.out_r_off[ev] + R.outdeg(i);
+            c.out_c_off[ev + 1] = c.out_c_off[ev] + C.outdeg(i);
+        }
+    if (s->n_send_r != c.out_r_off[nE] || s->n_send_c != c.out_c_off[nE])
+        return fail(err, RFAST_ESCHED, "schedule: send code counts (%lld, %lld) do not match the out-degrees",
+                    s->n_send_r, s->n_send_c);
+    if ((s->n_send_r > 0 && !s->send_r) || (s->n_send_c > 0 && !s->send_c))
+        return fail(err, RFAST_ESCHED, "schedule: send codes are null");
+    for (int64_t k = 0; k < s->n_send_r; ++k)
+        if (s->send_r[k] < -1) return fail(err, RFAST_ESCHED, "schedule: send_r code below -1 at %lld", k);
+    for (int64_t k = 0; k < s->n_send_c; ++k)
+        if (s->send_c[k] < -1) return fail(err, RFAST_ESCHED, "schedule: send_c code below -1 at %lld", k);
+    if (batch > 0) {
+        if (s->n_batch_idx != (int64_t)(n + nE) * batch || !s->batch_idx)
+            return fail(err, RFAST_ESCHED, "schedule: batch_idx must hold (n + events) * B = %lld entries",
+                        (long long)(n + nE) * batch);
+        for (int64_t k = 0; k < s->n_batch_idx; ++k)
+            if (s->batch_idx[k] < 0 || s->batch_idx[k] >= rows)
+                return fail(err, RFAST_ESCHED, "schedule: batch index out of the shard at %lld", k);
+    }
+
+    // ---- pass 1: consumed stamps, version lifetimes -----------------------------------------
+    const int INF = INT_MAX;
+    std::vector<std::vector<Pend>> pend_v(R.E), pend_c(C.E);
+    std::vector<int> tau_v(R.E, 0), tau_rho(C.E, 0), t(n, 0);
+    std::vector<std::vector<int>> ev_of(n);            // node -> event id of stamp s at [s-1]
+    c.used_tau_v.reserve(c.in_r_off[nE]);
+    c.used_tau_rho.reserve(c.in_c_off[nE]);
+    c.prev_tau_rho.reserve(c.in_c_off[nE]);
+    c.v_write.assign(nE, 0);
+    c.v_last.assign(nE, 0);
+    std::vector<char> v_sent(nE, 0);
+    const int64_t nRho = c.out_c_off[nE];
+    c.rho_write.assign(nRho, 0);
+    std::vector<int> rho_last_sender(nRho, 0), rho_last_recv(nRho, -1);
+    for (int r = 0; r < K; ++r) {
+        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+            const int i = c.act_node[ev];
+            for (int e = R.rowptr[i]; e < R.rowptr[i + 1]; ++e) {
+                int tau = deliver(pend_v[e], r, tau_v[e]);
+                tau_v[e] = tau;
+                c.used_tau_v.push_back(tau);
+                if (tau >= 1) {
+                    int pe = ev_of[R.col[e]][tau - 1];
+                    c.v_last[pe] = std::max(c.v_last[pe], r);
+                }
+            }
+            for (int e = C.rowptr[i]; e < C.rowptr[i + 1]; ++e) {
+                int prev = tau_rho[e];
+                int tau = deliver(pend_c[e], r, prev);
+                c.used_tau_rho.push_back(tau);
+                c.prev_tau_rho.push_back(prev);
+                if (tau > prev) {                      // news: rho[tau] - rho[prev] is read
+                    const auto& evs = ev_of[C.col[e]];
+                    int64_t vn = c.out_c_off[evs[tau - 1]] + C.opos[e];
+                    rho_last_recv[vn] = std::max(rho_last_recv[vn], r);
+                    if (prev >= 1) {
+                        int64_t vp = c.out_c_off[evs[prev - 1]] + C.opos[e];
+                        rho_last_recv[vp] = std::max(rho_last_recv[vp], r);
+                    }
+                }
+                tau_rho[e] = tau;
+            }
+            const int stamp = ++t[i];
+            if (stamp >= 2) {                          // S2c reads the sender's current running sums
+                int64_t base = c.out_c_off[ev_of[i][stamp - 2]];
+                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = r;
+            }
+            ev_of[i].push_back(ev);
+            c.v_write[ev] = r;
+            c.v_last[ev] = r;
+            for (int k = 0; k < R.outdeg(i); ++k) {
+                int d = s->send_r[c.out_r_off[ev] + k];
+                if (d >= 0) {
+                    v_sent[ev] = 1;
+                    pend_v[R.oeid[R.optr[i] + k]].push_back({r + 1 + d, stamp});
+                }
+            }
+            for (int k = 0; k < C.outdeg(i); ++k) {
+                int64_t vid = c.out_c_off[ev] + k;
+                c.rho_write[vid] = r;
+                rho_last_sender[vid] = r;
+                int d = s->send_c[vid];
+                if (d >= 0) pend_c[C.oeid[C.optr[i] + k]].push_back({r + 1 + d, stamp});
+            }
+        }
+    }
+    c.tau_v_end = tau_v;
+    c.tau_rho_end = tau_rho;
+    c.t_end = t;
+    // what is current at the end of the schedule stays readable: each sender's latest running
+    // sums and each receiver's buffered version
+    for (int i = 0; i < n; ++i)
+        if (t[i] >= 1) {
+            int64_t base = c.out_c_off[ev_of[i][t[i] - 1]];
+            for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = INF;
+        }
+    for (int e = 0; e < C.E; ++e)
+        if (tau_rho[e] >= 1)
+            rho_last_recv[c.out_c_off[ev_of[C.col[e]][tau_rho[e] - 1]] + C.opos[e]] = INF;
+    c.rho_last.resize(nRho);
+    for (int64_t v = 0; v < nRho; ++v) c.rho_last[v] = std::max(rho_last_sender[v], rho_last_recv[v]);
+
+    // ---- pass 2: rows.  A row is free again in the round after its version's last read -------
+    c.v_slot.assign(nE, -1);
+    c.rho_slot.assign(nRho, -1);
+    std::vector<std::vector<int64_t>> rel_v(K + 1), rel_c(K + 1);
+    std::vector<int> free_v, free_c;
+    std::vector<char> moved(nRho, 0);                  // row handed on to the next version in place
+    std::vector<int> stamp_of(nE, 0);
+    {
+        std::vector<int> tt(n, 0);
+        for (int64_t ev = 0; ev < nE; ++ev) stamp_of[ev] = ++tt[c.act_node[ev]];
+    }
+    for (int r = 0; r < K; ++r) {
+        for (int64_t id : rel_v[r]) free_v.push_back(c.v_slot[id]);
+        for (int64_t id : rel_c[r]) if (!moved[id]) free_c.push_back(c.rho_slot[id]);
+        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+            const int i = c.act_node[ev];
+            if (v_sent[ev]) {
+                int slot;
+                if (!free_v.empty()) { slot = free_v.back(); free_v.pop_back(); }
+                else slot = c.n_v_slots++;
+                c.v_slot[ev] = slot;
+                if (c.v_last[ev] + 1 < K) rel_v[c.v_last[ev] + 1].push_back(ev);
+            }
+            for (int k = 0; k < C.outdeg(i); ++k) {
+                int64_t vid = c.out_c_off[ev] + k;
+                int slot = -1;
+                if (stamp_of[ev] >= 2) {
+                    // in place: the previous version is read for the last time here, by this
+                    // very update, and no receiver reads it in this round or later
+                    int64_t cur = c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k;
+                    if (c.rho_last[cur] == r && rho_last_recv[cur] < r) {
+                        slot = c.rho_slot[cur];
+                        moved[cur] = 1;
+                    }
+                }
+                if (slot < 0) {
+                    if (!free_c.empty()) { slot = free_c.back(); free_c.pop_back(); }
+                    else slot = c.n_rho_slots++;
+                }
+                c.rho_slot[vid] = slot;
+                if (c.rho_last[vid] != INF && c.rho_last[vid] + 1 < K)
+                    rel_c[c.rho_last[vid] + 1].push_back(vid);
+            }
+        }
+    }
+
+    // ---- pass 3: device descriptors and the method's traffic ---------------------------------
+    c.ev.resize(nE);
+    c.round_streams.assign(K + 1, 0);
+    for (int r = 0; r < K; ++r) {
+        int64_t streams = 0;
+        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+            const int i = c.act_node[ev];
+            EvDesc d{};
+            d.node = i;
+            d.v_out = c.v_slot[ev];
+            d.w_self = R.diag[i];
+            d.a_self = C.diag[i];
+            d.stamp = stamp_of[ev];
+            d.g_par = (stamp_of[ev] - 1) & 1;
+            d.sample = (int32_t)(n + ev);
+            d.mix_beg = (int32_t)c.mix_slot.size();
+            for (int e = R.rowptr[i], k = 0; e < R.rowptr[i + 1]; ++e, ++k) {
+                int tau = c.used_tau_v[c.in_r_off[ev] + k];
+                if (tau < 1) continue;                 // stamp 0 is the zero vector: nothing to read
+                int slot = c.v_slot[ev_of[R.col[e]][tau - 1]];
+                if (slot < 0) return fail(err, RFAST_ESCHED, "internal: consumed v version without a row (event %lld)", ev);
+                c.mix_slot.push_back(slot);
+                c.mix_w.push_back(R.w[e]);
+            }
+            d.mix_cnt = (int32_t)c.mix_slot.size() - d.mix_beg;
+            d.news_beg = (int32_t)c.news_new.size();
+            int news_streams = 0;
+            for (int e = C.rowptr[i], k = 0; e < C.rowptr[i + 1]; ++e, ++k) {
+                int tau = c.used_tau_rho[c.in_c_off[ev] + k];
+                int prev = c.prev_tau_rho[c.in_c_off[ev] + k];
+                if (tau <= prev) continue;             // nothing newer: rho[tau] - rho~ = 0
+                const auto& evs = ev_of[C.col[e]];
+                c.news_new.push_back(c.rho_slot[c.out_c_off[evs[tau - 1]] + C.opos[e]]);
+                c.news_prev.push_back(prev >= 1 ? c.rho_slot[c.out_c_off[evs[prev - 1]] + C.opos[e]] : -1);
+                c.news_edge.push_back(e);
+                news_streams += 1 + (prev >= 1);
+            }
+            d.news_cnt = (int32_t)c.news_new.size() - d.news_beg;
+            d.out_beg = (int32_t)c.out_new.size();
+            int out_streams = 0;
+            for (int k = 0; k < C.outdeg(i); ++k) {
+                int e = C.oeid[C.optr[i] + k];
+                int cur = -1;
+                if (stamp_of[ev] >= 2) cur = c.rho_slot[c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k];
+                c.out_cur.push_back(cur);
+                c.out_new.push_back(c.rho_slot[c.out_c_off[ev] + k]);
+                c.out_a.push_back(C.w[e]);
+                c.out_edge.push_back(e);
+                out_streams += 1 + (cur >= 0);
+            }
+            d.out_cnt = (int32_t)c.out_new.size() - d.out_beg;
+            c.ev[ev] = d;
+            // fp32 streams per coordinate: S1/S2a read x, z, the neighbours' v, write v (if a
+            // packet leaves) and x; S2b/S2c read the news, write z and the running sums
+            int64_t st = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
+            if (mt.elementwise) st += mt.data_streams;
+            else st += 1 /*gradient reads x*/ + 1 /*writes g*/ + 3 /*track re-reads z, g_old, g_new*/;
+            streams += st;
+        }
+        c.round_streams[r + 1] = c.round_streams[r] + streams;
+    }
+    out = std::move(c);
+    return RFAST_OK;
+}
+
+}  // namespace rfast

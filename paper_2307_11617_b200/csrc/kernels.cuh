@@ -1,0 +1,461 @@
+// Device kernels of the R-FAST activation step (sm_100a).
+//
+// State layout: every per-node / per-version vector is one row of `stride` floats
+// (stride = p rounded up to 32 floats, so rows start on 128-byte boundaries and can be
+// walked with 128-bit accesses); the padding stays zero.  All passes over coordinates are
+// pure streaming: each byte is touched once per activation, so loads and stores carry the
+// streaming (evict-first) hint.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rfast_internal.h"
+
+namespace rfast {
+
+struct RoundArgs {
+    const EvDesc* ev;            // events of this round
+    const int*    mix_slot;  const float* mix_w;
+    const int*    news_new;  const int*   news_prev;
+    const int*    out_cur;   const int*   out_new;   const float* out_a;
+    float* x;  float* z;         // [n][stride]
+    float* vbuf;                 // [v rows][stride]   published v versions
+    float* rbuf;                 // [rho rows][stride] running-sum versions
+    int64_t stride;              // floats per row
+    int     n4;                  // float4 per row (stride / 4)
+    float   alpha;
+};
+
+__device__ __forceinline__ float4 ld_stream(const float* row, int i4) {
+    return __ldcs(reinterpret_cast<const float4*>(row) + i4);
+}
+__device__ __forceinline__ void st_stream(float* row, int i4, float4 v) {
+    __stcs(reinterpret_cast<float4*>(row) + i4, v);
+}
+__device__ __forceinline__ float4 f4_axpy(float a, float4 x, float4 y) {   // a*x + y
+    return make_float4(fmaf(a, x.x, y.x), fmaf(a, x.y, y.y), fmaf(a, x.z, y.z), fmaf(a, x.w, y.w));
+}
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) {
+    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+__device__ __forceinline__ float4 f4_sub(float4 a, float4 b) {
+    return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w);
+}
+__device__ __forceinline__ float4 f4_scale(float a, float4 x) {
+    return make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
+}
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------------------------------------
+// Fused activation for the element-wise objective f_i(x) = 0.5 || d_i .* (x - b_i) ||^2:
+// S1 v = x - alpha z;  S2a x' = w_ii v + sum_j w_ij v_j[tau];  g' = d^2 (x' - b), g = d^2 (x - b)
+// (the remembered gradient is recomputed from the unchanged x instead of being stored);
+// S2b z^ = z + sum_news (rho[tau'] - rho[tau_prev]) + g' - g;  S2c z' = a_ii z^, rho' = rho + a_ji z^.
+// The buffer update S4 is a change of row id done by the host compiler (rho~ is the version
+// last consumed, kept alive instead of copied).  One HBM pass per activation.
+// grid = (tiles, events of the round)
+// ---------------------------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+k_fused_quad(RoundArgs a, const float* __restrict__ qd, const float* __restrict__ qb) {
+    const EvDesc e = a.ev[blockIdx.y];
+    const int64_t row = (int64_t)e.node * a.stride;
+    float* xr = a.x + row;
+    float* zr = a.z + row;
+    const float* dr = qd + row;
+    const float* br = qb + row;
+    const int base = blockIdx.x * (kThreads * U) + threadIdx.x;
+
+    float4 xv[U], zv[U], dv[U], bv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int i4 = base + u * kThreads;
+        xv[u] = zv[u] = dv[u] = bv[u] = make_float4(0, 0, 0, 0);
+        if (i4 < a.n4) {
+            xv[u] = ld_stream(xr, i4);
+            zv[u] = ld_stream(zr, i4);
+            dv[u] = ld_stream(dr, i4);
+            bv[u] = ld_stream(br, i4);
+        }
+    }
+    float4 acc[U], v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        v[u] = f4_axpy(-a.alpha, zv[u], xv[u]);                    // S1
+        acc[u] = f4_scale(e.w_self, v[u]);                          // S2a, own term first
+    }
+    if (e.v_out >= 0) {
+        float* vr = a.vbuf + (int64_t)e.v_out * a.stride;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) st_stream(vr, i4, v[u]);
+        }
+    }
+    for (int m = 0; m < e.mix_cnt; ++m) {                           // ascending sender id
+        const float* nr = a.vbuf + (int64_t)a.mix_slot[e.mix_beg + m] * a.stride;
+        const float w = a.mix_w[e.mix_beg + m];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) acc[u] = f4_axpy(w, ld_stream(nr, i4), acc[u]);
+        }
+    }
+    float4 zh[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int i4 = base + u * kThreads;
+        if (i4 < a.n4) st_stream(xr, i4, acc[u]);
+        zh[u] = zv[u];
+    }
+    for (int m = 0; m < e.news_cnt; ++m) {                          // S2b, ascending sender id
+        const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
+        const int prev = a.news_prev[e.news_beg + m];
+        const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) {
+                float4 dl = ld_stream(nr, i4);
+                if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
+                zh[u] = f4_add(zh[u], dl);
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float4 d2 = make_float4(dv[u].x * dv[u].x, dv[u].y * dv[u].y, dv[u].z * dv[u].z, dv[u].w * dv[u].w);
+        const float4 gn = make_float4(d2.x * (acc[u].x - bv[u].x), d2.y * (acc[u].y - bv[u].y),
+                                      d2.z * (acc[u].z - bv[u].z), d2.w * (acc[u].w - bv[u].w));
+        const float4 go = make_float4(d2.x * (xv[u].x - bv[u].x), d2.y * (xv[u].y - bv[u].y),
+                                      d2.z * (xv[u].z - bv[u].z), d2.w * (xv[u].w - bv[u].w));
+        zh[u] = f4_sub(f4_add(zh[u], gn), go);
+        const int i4 = base + u * kThreads;
+        if (i4 < a.n4) st_stream(zr, i4, f4_scale(e.a_self, zh[u]));       // S2c keep
+    }
+    for (int m = 0; m < e.out_cnt; ++m) {                           // S2c accumulate
+        const int cur = a.out_cur[e.out_beg + m];
+        const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
+        float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
+        const float aw = a.out_a[e.out_beg + m];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) {
+                float4 r = f4_scale(aw, zh[u]);
+                if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
+                st_stream(wr, i4, r);
+            }
+        }
+    }
+}
+
+// z_i^0 = grad f_i(x_i^0) for the element-wise objective.  grid = (tiles, n)
+__global__ void __launch_bounds__(kThreads)
+k_quad_grad(const float* __restrict__ x, const float* __restrict__ qd, const float* __restrict__ qb,
+            float* __restrict__ out, int64_t stride, int n4) {
+    const int64_t row = (int64_t)blockIdx.y * stride;
+    const int i4 = blockIdx.x * kThreads + threadIdx.x;
+    if (i4 >= n4) return;
+    const float4 xv = ld_stream(x + row, i4), d = ld_stream(qd + row, i4), b = ld_stream(qb + row, i4);
+    st_stream(out + row, i4, make_float4(d.x * d.x * (xv.x - b.x), d.y * d.y * (xv.y - b.y),
+                                         d.z * d.z * (xv.z - b.z), d.w * d.w * (xv.w - b.w)));
+}
+
+// ---------------------------------------------------------------------------------------------
+// S1 + S2a for objectives whose gradient needs the whole new x first.  Optionally leaves a
+// bf16 copy of the new x (operand of the MLP's matrix products).  grid = (tiles, events)
+// ---------------------------------------------------------------------------------------------
+template <int U, bool BF16>
+__global__ void __launch_bounds__(kThreads)
+k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
+    const EvDesc e = a.ev[blockIdx.y];
+    const int64_t row = (int64_t)e.node * a.stride;
+    float* xr = a.x + row;
+    const float* zr = a.z + row;
+    const int base = blockIdx.x * (kThreads * U) + threadIdx.x;
+    float4 acc[U], v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int i4 = base + u * kThreads;
+        float4 xv = make_float4(0, 0, 0, 0), zv = xv;
+        if (i4 < a.n4) { xv = ld_stream(xr, i4); zv = ld_stream(zr, i4); }
+        v[u] = f4_axpy(-a.alpha, zv, xv);
+        acc[u] = f4_scale(e.w_self, v[u]);
+    }
+    if (e.v_out >= 0) {
+        float* vr = a.vbuf + (int64_t)e.v_out * a.stride;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) st_stream(vr, i4, v[u]);
+        }
+    }
+    for (int m = 0; m < e.mix_cnt; ++m) {
+        const float* nr = a.vbuf + (int64_t)a.mix_slot[e.mix_beg + m] * a.stride;
+        const float w = a.mix_w[e.mix_beg + m];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) acc[u] = f4_axpy(w, ld_stream(nr, i4), acc[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int i4 = base + u * kThreads;
+        if (i4 < a.n4) {
+            // the gradient kernels re-read x soon: keep it cacheable
+            reinterpret_cast<float4*>(xr)[i4] = acc[u];
+            if (BF16) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(acc[u].x, acc[u].y);
+                __nv_bfloat162 hi = __floats2bfloat162_rn(acc[u].z, acc[u].w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                reinterpret_cast<uint2*>(xb + row)[i4] = pk;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// S2b + S2c (+ S4 by row id) with the gradients taken from the two gradient buffers:
+// g_old = gbuf[par][node], g_new = gbuf[par^1][node].  grid = (tiles, events)
+// ---------------------------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
+    const EvDesc e = a.ev[blockIdx.y];
+    const int64_t row = (int64_t)e.node * a.stride;
+    float* zr = a.z + row;
+    const float* go = gbuf + (int64_t)e.g_par * gplane + row;
+    const float* gn = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
+    const int base = blockIdx.x * (kThreads * U) + threadIdx.x;
+    float4 zh[U], gnv[U], gov[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int i4 = base + u * kThreads;
+        zh[u] = gnv[u] = gov[u] = make_float4(0, 0, 0, 0);
+        if (i4 < a.n4) { zh[u] = ld_stream(zr, i4); gnv[u] = ld_stream(gn, i4); gov[u] = ld_stream(go, i4); }
+    }
+    for (int m = 0; m < e.news_cnt; ++m) {
+        const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
+        const int prev = a.news_prev[e.news_beg + m];
+        const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) {
+                float4 dl = ld_stream(nr, i4);
+                if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
+                zh[u] = f4_add(zh[u], dl);
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        zh[u] = f4_sub(f4_add(zh[u], gnv[u]), gov[u]);
+        const int i4 = base + u * kThreads;
+        if (i4 < a.n4) st_stream(zr, i4, f4_scale(e.a_self, zh[u]));
+    }
+    for (int m = 0; m < e.out_cnt; ++m) {
+        const int cur = a.out_cur[e.out_beg + m];
+        const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
+        float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
+        const float aw = a.out_a[e.out_beg + m];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) {
+                float4 r = f4_scale(aw, zh[u]);
+                if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
+                st_stream(wr, i4, r);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sample gradients.  Every kernel takes the round's events; x_i is the freshly mixed row and
+// the result goes to gbuf[par^1][node].  Reductions run in a fixed order (run-to-run identical).
+// ---------------------------------------------------------------------------------------------
+struct GradArgs {
+    const EvDesc* ev;
+    const float*  x;          // [n][stride]
+    float*        gbuf;       // [2][n][stride]
+    int64_t stride, gplane;
+    const int*    batch_idx;  // [(n + events) * B]
+    int B, rows, F, C, H;
+    int64_t p;
+    float l2;
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Least squares, phase 1: residual r_k = a_k . x - y_k, one warp per sampled row.
+// grid = (ceil(B / 8), events), 256 threads.  res: [events][B]
+__global__ void __launch_bounds__(256)
+k_ls_residual(GradArgs g, const float* __restrict__ feat, const float* __restrict__ target,
+              float* __restrict__ res, int use_all) {
+    const EvDesc e = g.ev[blockIdx.y];
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (k >= g.B) return;
+    const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+    const float* a = feat + ((int64_t)e.node * g.rows + rrow) * g.F;
+    const float* x = g.x + (int64_t)e.node * g.stride;
+    float s = 0.f;
+    for (int c = lane; c < g.F; c += 32) s = fmaf(a[c], x[c], s);
+    s = warp_sum(s);
+    if (lane == 0) res[(int64_t)blockIdx.y * g.B + k] = s - target[(int64_t)e.node * g.rows + rrow];
+}
+
+// Least squares, phase 2: g_c = (1/B) sum_k a_k[c] r_k + l2 x_c.  grid = (ceil(p/256), events)
+__global__ void __launch_bounds__(256)
+k_ls_grad(GradArgs g, const float* __restrict__ feat, const float* __restrict__ res, int use_all) {
+    const EvDesc e = g.ev[blockIdx.y];
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    if (c >= g.F) return;
+    const float* abase = feat + (int64_t)e.node * g.rows * g.F;
+    float s = 0.f;
+    for (int k = 0; k < g.B; ++k) {
+        const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+        s = fmaf(abase[(int64_t)rrow * g.F + c], res[(int64_t)blockIdx.y * g.B + k], s);
+    }
+    const int64_t row = (int64_t)e.node * g.stride;
+    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + row + c] = s / (float)g.B + g.l2 * g.x[row + c];
+}
+
+// Softmax regression, phase 1: logits[k][c] = W_c . a_k + bias_c; one block per sampled row,
+// one warp per class (round-robin).  grid = (B, events).  logit: [events][B][C]
+__global__ void __launch_bounds__(256)
+k_softmax_logits(GradArgs g, const float* __restrict__ feat, float* __restrict__ logit) {
+    const EvDesc e = g.ev[blockIdx.y];
+    const int k = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
+    const float* a = feat + ((int64_t)e.node * g.rows + rrow) * g.F;
+    const float* x = g.x + (int64_t)e.node * g.stride;
+    for (int c = warp; c < g.C; c += 8) {
+        const float* w = x + (int64_t)c * g.F;
+        float s = 0.f;
+        for (int f = lane; f < g.F; f += 32) s = fmaf(a[f], w[f], s);
+        s = warp_sum(s);
+        if (lane == 0) logit[((int64_t)blockIdx.y * g.B + k) * g.C + c] = s + x[(int64_t)g.C * g.F + c];
+    }
+}
+
+// Softmax regression, phase 2: delta = (softmax(logits) - onehot) / B (recomputed per block in
+// shared memory), then g[c][f] = sum_k delta[k][c] a_k[f] + l2 W[c][f] and the bias gradient.
+// grid = (ceil(p / 256), events); dynamic shared memory: B*C floats + B ints
+__global__ void __launch_bounds__(256)
+k_softmax_grad(GradArgs g, const float* __restrict__ feat, const int* __restrict__ label,
+               const float* __restrict__ logit) {
+    extern __shared__ float sm[];
+    float* delta = sm;                                   // [B][C]
+    int* rowid = reinterpret_cast<int*>(sm + g.B * g.C); // [B]
+    const EvDesc e = g.ev[blockIdx.y];
+    for (int k = threadIdx.x; k < g.B; k += 256) {
+        const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
+        rowid[k] = rrow;
+        const float* lg = logit + ((int64_t)blockIdx.y * g.B + k) * g.C;
+        float m = lg[0];
+        for (int c = 1; c < g.C; ++c) m = fmaxf(m, lg[c]);
+        float den = 0.f;
+        for (int c = 0; c < g.C; ++c) den += expf(lg[c] - m);
+        const int lab = label[(int64_t)e.node * g.rows + rrow];
+        for (int c = 0; c < g.C; ++c)
+            delta[k * g.C + c] = (expf(lg[c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)g.B;
+    }
+    __syncthreads();
+    const int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (q >= g.p) return;
+    const int64_t row = (int64_t)e.node * g.stride;
+    float s = 0.f;
+    if (q < (int64_t)g.C * g.F) {
+        const int c = (int)(q / g.F), f = (int)(q % g.F);
+        const float* abase = feat + (int64_t)e.node * g.rows * g.F;
+        for (int k = 0; k < g.B; ++k) s = fmaf(delta[k * g.C + c], abase[(int64_t)rowid[k] * g.F + f], s);
+    } else {
+        const int c = (int)(q - (int64_t)g.C * g.F);
+        for (int k = 0; k < g.B; ++k) s += delta[k * g.C + c];
+    }
+    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + row + q] = s + g.l2 * g.x[row + q];
+}
+
+// Sparse logistic regression, phase 1: coef_k = -y_k / (1 + exp(y_k a_k.x)) / B, one warp per
+// sampled row.  grid = (ceil(B / 8), events).  coef: [events][B]
+__global__ void __launch_bounds__(256)
+k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col,
+             const float* __restrict__ sp_val, const int* __restrict__ label, float* __restrict__ coef) {
+    const EvDesc e = g.ev[blockIdx.y];
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (k >= g.B) return;
+    const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
+    const int64_t r = (int64_t)e.node * g.rows + rrow;
+    const float* x = g.x + (int64_t)e.node * g.stride;
+    float s = 0.f;
+    for (int64_t q = sp_ptr[r] + lane; q < sp_ptr[r + 1]; q += 32) s = fmaf(sp_val[q], x[sp_col[q]], s);
+    s = warp_sum(s);
+    if (lane == 0) {
+        const float y = (float)label[r];
+        coef[(int64_t)blockIdx.y * g.B + k] = -y / (1.f + expf(y * s)) / (float)g.B;
+    }
+}
+
+// Sparse logistic regression, phase 2: g = l2 x + sum_k coef_k a_k on a tile of kTile
+// coordinates held in shared memory; rows are added one after the other (fixed order), the
+// entries of one row land on distinct coordinates.  grid = (ceil(p / kTile), events)
+constexpr int kLogitTile = 2048;
+__global__ void __launch_bounds__(256)
+k_logit_grad(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col,
+             const float* __restrict__ sp_val, const float* __restrict__ coef) {
+    __shared__ float tile[kLogitTile];
+    __shared__ int64_t lo_s, hi_s;
+    const EvDesc e = g.ev[blockIdx.y];
+    const int64_t c0 = (int64_t)blockIdx.x * kLogitTile;
+    const int64_t c1 = min(c0 + (int64_t)kLogitTile, g.p);
+    const int64_t row = (int64_t)e.node * g.stride;
+    for (int c = threadIdx.x; c < kLogitTile; c += 256)
+        tile[c] = (c0 + c < c1) ? g.l2 * g.x[row + c0 + c] : 0.f;
+    __syncthreads();
+    for (int k = 0; k < g.B; ++k) {
+        const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
+        const int64_t r = (int64_t)e.node * g.rows + rrow;
+        if (threadIdx.x == 0) {                      // entries of row r with c0 <= col < c1
+            int64_t lo = sp_ptr[r], hi = sp_ptr[r + 1], end = hi;
+            while (lo < hi) { int64_t m = (lo + hi) >> 1; if (sp_col[m] < c0) lo = m + 1; else hi = m; }
+            lo_s = lo;
+            hi = end;
+            while (lo < hi) { int64_t m = (lo + hi) >> 1; if (sp_col[m] < c1) lo = m + 1; else hi = m; }
+            hi_s = lo;
+        }
+        __syncthreads();
+        const float ck = coef[(int64_t)blockIdx.y * g.B + k];
+        for (int64_t q = lo_s + threadIdx.x; q < hi_s; q += 256)
+            tile[sp_col[q] - c0] = fmaf(ck, sp_val[q], tile[sp_col[q] - c0]);
+        __syncthreads();
+    }
+    float* out = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row;
+    for (int c = threadIdx.x; c0 + c < c1; c += 256) out[c0 + c] = tile[c];
+}
+
+// row copy helpers ----------------------------------------------------------------------------
+// dst[r][0..n4) = src[idx ? idx[r] : r][0..n4); a negative index gives a zero row.  grid = (tiles, rows)
+__global__ void __launch_bounds__(kThreads)
+k_gather_rows(const float* __restrict__ src, const int* __restrict__ idx, float* __restrict__ dst,
+              int64_t src_stride, int64_t dst_stride, int n4) {
+    const int i4 = blockIdx.x * kThreads + threadIdx.x;
+    if (i4 >= n4) return;
+    const int r = idx ? idx[blockIdx.y] : (int)blockIdx.y;
+    float4 v = make_float4(0, 0, 0, 0);
+    if (r >= 0) v = reinterpret_cast<const float4*>(src + (int64_t)r * src_stride)[i4];
+    reinterpret_cast<float4*>(dst + (int64_t)blockIdx.y * dst_stride)[i4] = v;
+}
+
+}  // namespace rfast
