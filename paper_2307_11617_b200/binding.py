@@ -1,0 +1,271 @@
+"""ctypes binding of librfast.so: argument marshalling only.
+
+Every step of the R-FAST activation path runs inside the CUDA library; this module turns
+numpy arrays into the plain pointers of include/rfast.h and back.  The functions carry the
+names of the C entry points.  There is no fallback: if the shared library is missing, or no
+CUDA device is present, the calls raise.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librfast.so")
+
+OK, EINVAL, EGRAPH, ESCHED, ENOMEM, ECUDA, ETIMEOUT, ESTATE = 0, -1, -2, -3, -4, -5, -6, -7
+_ERRNAMES = {-1: "EINVAL", -2: "EGRAPH", -3: "ESCHED", -4: "ENOMEM", -5: "ECUDA", -6: "ETIMEOUT", -7: "ESTATE"}
+
+MODEL_IDS = {"quad_diag": 0, "least_squares": 1, "softmax": 2, "mlp": 3, "logistic_sparse": 4}
+
+STATE_X, STATE_Y, STATE_G_LAST, STATE_RHO_LATEST, STATE_RHO_BUF = 0, 1, 2, 3, 4
+STATE_T_LOCAL, STATE_USED_TAU_V, STATE_USED_TAU_RHO, STATE_TAU_V_END, STATE_TAU_RHO_END, STATE_ROUND = 5, 6, 7, 8, 9, 10
+Q_ROUND, Q_EVENTS_TOTAL, Q_EVENTS_RUN, Q_LAUNCHES, Q_BYTES_RUN, Q_V_SLOTS, Q_RHO_SLOTS = 0, 1, 2, 3, 4, 5, 6
+Q_DEVICE_BYTES, Q_N_USED_TAU_V, Q_N_USED_TAU_RHO, Q_BYTES_TOTAL = 7, 8, 9, 10
+
+
+class RFastError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"rfast: {_ERRNAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+class _Graph(C.Structure):
+    _fields_ = [("n_edges", C.c_int32), ("rowptr", C.c_void_p), ("col", C.c_void_p),
+                ("w", C.c_void_p), ("diag", C.c_void_p)]
+
+
+class _Problem(C.Structure):
+    _fields_ = [("n", C.c_int32), ("root", C.c_int32), ("p", C.c_int64), ("alpha", C.c_float),
+                ("l2", C.c_float), ("G_R", _Graph), ("G_C", _Graph), ("model", C.c_int32),
+                ("batch", C.c_int32), ("rows", C.c_int32), ("n_features", C.c_int32),
+                ("n_classes", C.c_int32), ("n_hidden", C.c_int32),
+                ("quad_d", C.c_void_p), ("quad_b", C.c_void_p), ("feat", C.c_void_p),
+                ("target", C.c_void_p), ("label", C.c_void_p), ("sp_rowptr", C.c_void_p),
+                ("sp_col", C.c_void_p), ("sp_val", C.c_void_p), ("x0", C.c_void_p)]
+
+
+class _Schedule(C.Structure):
+    _fields_ = [("K", C.c_int32), ("act_ptr", C.c_void_p), ("act_node", C.c_void_p),
+                ("n_send_r", C.c_int64), ("send_r", C.c_void_p), ("n_send_c", C.c_int64),
+                ("send_c", C.c_void_p), ("n_batch_idx", C.c_int64), ("batch_idx", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it first "
+                               "(python -m paper_2307_11617_b200.build); there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        L.rfast_create.argtypes = [C.POINTER(_Problem), C.c_void_p, C.POINTER(C.c_void_p)]
+        L.rfast_load_schedule.argtypes = [C.c_void_p, C.POINTER(_Schedule)]
+        L.rfast_run.argtypes = [C.c_void_p, C.c_int32, C.c_int]
+        L.rfast_read_state.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t]
+        L.rfast_reset.argtypes = [C.c_void_p]
+        L.rfast_sync.argtypes = [C.c_void_p]
+        L.rfast_query.argtypes = [C.c_void_p, C.c_int]
+        L.rfast_query.restype = C.c_int64
+        L.rfast_destroy.argtypes = [C.c_void_p]
+        L.rfast_destroy.restype = None
+        L.rfast_last_error.argtypes = [C.c_void_p]
+        L.rfast_last_error.restype = C.c_char_p
+        L.rfast_version.restype = C.c_char_p
+        L.rfast_compile_host.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule)] + [C.c_void_p] * 5 + \
+            [C.c_char_p, C.c_size_t]
+        _lib = L
+    return _lib
+
+
+def _arr(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _graph(g, keep):
+    rowptr, col = _arr(g.rowptr, np.int32), _arr(g.col, np.int32)
+    w, diag = _arr(g.w, np.float32), _arr(g.diag, np.float32)
+    keep += [rowptr, col, w, diag]
+    return _Graph(len(col), _ptr(rowptr), _ptr(col), _ptr(w), _ptr(diag))
+
+
+def _problem(wl, keep):
+    """wl: object with n, p, root, alpha, l2, G_R, G_C, model (name), batch, rows, dims, data, x0."""
+    P = _Problem()
+    P.n, P.root, P.p, P.alpha, P.l2 = int(wl.n), int(wl.root), int(wl.p), float(wl.alpha), float(wl.l2)
+    P.G_R, P.G_C = _graph(wl.G_R, keep), _graph(wl.G_C, keep)
+    P.model = MODEL_IDS[wl.model] if isinstance(wl.model, str) else int(wl.model)
+    P.batch, P.rows = int(wl.batch), int(wl.rows)
+    dims = getattr(wl, "dims", {}) or {}
+    P.n_features = int(dims.get("n_features", 0))
+    P.n_classes = int(dims.get("n_classes", 0))
+    P.n_hidden = int(dims.get("n_hidden", 0))
+    data = getattr(wl, "data", {}) or {}
+    spec = {"quad_d": ("d", np.float32), "quad_b": ("b", np.float32), "feat": ("feat", np.float32),
+            "target": ("target", np.float32), "label": ("label", np.int32),
+            "sp_rowptr": ("sp_rowptr", np.int64), "sp_col": ("sp_col", np.int32),
+            "sp_val": ("sp_val", np.float32)}
+    for field, (key, dt) in spec.items():
+        if key in data and data[key] is not None:
+            a = _arr(data[key], dt)
+            keep.append(a)
+            setattr(P, field, _ptr(a))
+    if getattr(wl, "x0", None) is not None:
+        a = _arr(wl.x0, np.float32)
+        keep.append(a)
+        P.x0 = _ptr(a)
+    return P
+
+
+def _schedule(s, keep):
+    S = _Schedule()
+    act_ptr, act_node = _arr(s.act_ptr, np.int32), _arr(s.act_node, np.int32)
+    send_r, send_c = _arr(s.send_r, np.int8), _arr(s.send_c, np.int8)
+    bidx = _arr(s.batch_idx, np.int32)
+    keep += [act_ptr, act_node, send_r, send_c, bidx]
+    S.K = int(s.K)
+    S.act_ptr, S.act_node = _ptr(act_ptr), _ptr(act_node)
+    S.n_send_r, S.send_r = len(send_r), _ptr(send_r)
+    S.n_send_c, S.send_c = len(send_c), _ptr(send_c)
+    S.n_batch_idx, S.batch_idx = len(bidx), _ptr(bidx)
+    return S
+
+
+def _check(rc, handle=None):
+    if rc != OK:
+        raise RFastError(rc, lib().rfast_last_error(handle).decode())
+
+
+def rfast_version() -> str:
+    return lib().rfast_version().decode()
+
+
+def rfast_create(wl, cuda_stream: int = 0) -> int:
+    """Returns an opaque handle.  cuda_stream: a cudaStream_t as an integer (0: default stream)."""
+    keep = []
+    P = _problem(wl, keep)
+    h = C.c_void_p()
+    _check(lib().rfast_create(C.byref(P), C.c_void_p(cuda_stream), C.byref(h)))
+    return h.value
+
+
+def rfast_load_schedule(handle, s) -> None:
+    keep = []
+    S = _schedule(s, keep)
+    _check(lib().rfast_load_schedule(handle, C.byref(S)), handle)
+
+
+def rfast_run(handle, rounds: int, sync: bool = True) -> None:
+    _check(lib().rfast_run(handle, int(rounds), 1 if sync else 0), handle)
+
+
+def rfast_reset(handle) -> None:
+    _check(lib().rfast_reset(handle), handle)
+
+
+def rfast_sync(handle) -> None:
+    _check(lib().rfast_sync(handle), handle)
+
+
+def rfast_query(handle, what: int) -> int:
+    v = lib().rfast_query(handle, int(what))
+    if v < 0:
+        _check(int(v), handle)
+    return int(v)
+
+
+def rfast_read_state(handle, which: int, shape, out=None) -> np.ndarray:
+    """shape: the view's shape; float views are float32, integer views int32."""
+    dt = np.float32 if which <= STATE_RHO_BUF else np.int32
+    if out is None:
+        out = np.empty(shape, dtype=dt)
+    assert out.dtype == dt and out.flags.c_contiguous
+    _check(lib().rfast_read_state(handle, int(which), _ptr(out), out.nbytes), handle)
+    return out
+
+
+def rfast_destroy(handle) -> None:
+    lib().rfast_destroy(handle)
+
+
+def rfast_compile_host(wl, s):
+    """Host-only schedule compilation (no device needed).  Returns a dict of int arrays."""
+    keep = []
+    P, S = _problem(wl, keep), _schedule(s, keep)
+    indeg_r = np.diff(np.asarray(wl.G_R.rowptr)).astype(np.int64)
+    indeg_c = np.diff(np.asarray(wl.G_C.rowptr)).astype(np.int64)
+    nodes = np.clip(np.asarray(s.act_node, dtype=np.int64), 0, int(wl.n) - 1)   # bad ids are the library's to reject
+    ev = len(nodes)
+    used_v = np.empty(int(indeg_r[nodes].sum()), np.int32)
+    used_r = np.empty(int(indeg_c[nodes].sum()), np.int32)
+    v_ver = np.empty((ev, 3), np.int32)
+    rho_ver = np.empty((len(s.send_c), 3), np.int32)
+    counts = np.zeros(4, np.int64)
+    err = C.create_string_buffer(512)
+    rc = lib().rfast_compile_host(C.byref(P), C.byref(S), _ptr(used_v), _ptr(used_r), _ptr(v_ver),
+                                  _ptr(rho_ver), _ptr(counts), err, 512)
+    if rc != OK:
+        raise RFastError(rc, err.value.decode())
+    return {"used_tau_v": used_v, "used_tau_rho": used_r, "v_ver": v_ver, "rho_ver": rho_ver,
+            "v_rows": int(counts[0]), "rho_rows": int(counts[1]), "events": int(counts[2]),
+            "streams": int(counts[3])}
+
+
+class Engine:
+    """Convenience wrapper owning one handle."""
+
+    def __init__(self, wl, cuda_stream: int = 0):
+        self.n, self.p = int(wl.n), int(wl.p)
+        self.n_edges_c = len(wl.G_C.col)
+        self.n_edges_r = len(wl.G_R.col)
+        self.h = rfast_create(wl, cuda_stream)
+        self.K = 0
+
+    def load_schedule(self, s):
+        rfast_load_schedule(self.h, s)
+        self.K = int(s.K)
+
+    def run(self, rounds=None, sync=True):
+        rfast_run(self.h, self.K - self.query(Q_ROUND) if rounds is None else rounds, sync)
+
+    def reset(self):
+        rfast_reset(self.h)
+
+    def sync(self):
+        rfast_sync(self.h)
+
+    def query(self, what):
+        return rfast_query(self.h, what)
+
+    def read(self, which, out=None):
+        n, p = self.n, self.p
+        shape = {STATE_X: (n, p), STATE_Y: (n, p), STATE_G_LAST: (n, p),
+                 STATE_RHO_LATEST: (self.n_edges_c, p), STATE_RHO_BUF: (self.n_edges_c, p),
+                 STATE_T_LOCAL: (n,), STATE_TAU_V_END: (self.n_edges_r,),
+                 STATE_TAU_RHO_END: (self.n_edges_c,), STATE_ROUND: (1,)}.get(which)
+        if which == STATE_USED_TAU_V:
+            shape = (self.query(Q_N_USED_TAU_V),)
+        if which == STATE_USED_TAU_RHO:
+            shape = (self.query(Q_N_USED_TAU_RHO),)
+        return rfast_read_state(self.h, which, shape, out)
+
+    def close(self):
+        if self.h:
+            rfast_destroy(self.h)
+            self.h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()

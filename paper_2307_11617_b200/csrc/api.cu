@@ -1,0 +1,586 @@
+// C ABI of librfast: handle life cycle, uploads, per-round launches, state read-back.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+#include "rfast_internal.h"
+
+using namespace rfast;
+
+namespace rfast {
+// MLP gradient (tensor-core path), defined in grad_mlp.cu
+struct MlpPlan;
+int  mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride, int max_events,
+                     const float* d_feat, MlpPlan** out, size_t* dev_bytes, std::string& err);
+void mlp_plan_destroy(MlpPlan* plan);
+int  mlp_grad_launch(MlpPlan* plan, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
+                     int n_events, cudaStream_t st, int64_t* launches, std::string& err);
+}  // namespace rfast
+
+static std::string g_create_error;
+
+struct rfast_ctx {
+    cudaStream_t stream = nullptr;
+    int n = 0, root = 0, model = 0, batch = 0, rows = 0, F = 0, C = 0, H = 0;
+    int64_t p = 0, stride = 0;
+    float alpha = 0, l2 = 0;
+    HostGraph R, Cg;
+    // device state
+    float *x = nullptr, *z = nullptr, *gbuf = nullptr, *x0 = nullptr;
+    float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
+    int* label = nullptr;
+    int64_t* sp_ptr = nullptr;
+    int* sp_col = nullptr;
+    float* sp_val = nullptr;
+    __nv_bfloat16* xb = nullptr;
+    float *vbuf = nullptr, *rbuf = nullptr, *scratch = nullptr;
+    MlpPlan* mlp = nullptr;
+    // compiled schedule
+    bool has_sched = false;
+    Compiled comp;
+    EvDesc *d_ev = nullptr, *d_init_ev = nullptr;
+    int *d_mix_slot = nullptr, *d_news_new = nullptr, *d_news_prev = nullptr, *d_out_cur = nullptr,
+        *d_out_new = nullptr, *d_batch_idx = nullptr;
+    float *d_mix_w = nullptr, *d_out_a = nullptr;
+    std::vector<void*> sched_allocs;
+    int max_round_events = 0;
+    int round = 0;
+    int64_t launches = 0;
+    size_t dev_bytes = 0, sched_bytes = 0;
+    std::string err;
+};
+
+namespace {
+
+int set_err(rfast_ctx* c, int code, const std::string& msg) {
+    if (c) c->err = msg; else g_create_error = msg;
+    return code;
+}
+
+#define CK(call)                                                                               \
+    do {                                                                                       \
+        cudaError_t e_ = (call);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return set_err(ctx, e_ == cudaErrorMemoryAllocation ? RFAST_ENOMEM : RFAST_ECUDA, \
+                           std::string(#call) + ": " + cudaGetErrorString(e_));                \
+    } while (0)
+
+template <class T>
+cudaError_t dev_alloc(rfast_ctx* c, T** ptr, size_t count, bool sched = false) {
+    *ptr = nullptr;
+    if (count == 0) count = 1;
+    cudaError_t e = cudaMalloc((void**)ptr, count * sizeof(T));
+    if (e == cudaSuccess) {
+        c->dev_bytes += count * sizeof(T);
+        if (sched) { c->sched_allocs.push_back(*ptr); c->sched_bytes += count * sizeof(T); }
+    }
+    return e;
+}
+
+template <class T>
+int upload(rfast_ctx* ctx, T** dptr, const std::vector<T>& h) {
+    CK(dev_alloc(ctx, dptr, h.size(), true));
+    if (!h.empty())
+        CK(cudaMemcpyAsync(*dptr, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice, ctx->stream));
+    return RFAST_OK;
+}
+
+// host [rows][p] -> device [rows][stride], padding zeroed
+int upload_rows(rfast_ctx* ctx, float* dst, const float* src, int64_t rows) {
+    CK(cudaMemsetAsync(dst, 0, (size_t)rows * ctx->stride * sizeof(float), ctx->stream));
+    CK(cudaMemcpy2DAsync(dst, ctx->stride * sizeof(float), src, ctx->p * sizeof(float),
+                         ctx->p * sizeof(float), rows, cudaMemcpyHostToDevice, ctx->stream));
+    return RFAST_OK;
+}
+
+void free_schedule(rfast_ctx* c) {
+    for (void* q : c->sched_allocs) cudaFree(q);
+    c->sched_allocs.clear();
+    c->dev_bytes -= c->sched_bytes;
+    c->sched_bytes = 0;
+    c->d_ev = c->d_init_ev = nullptr;
+    c->vbuf = c->rbuf = c->scratch = nullptr;
+    c->has_sched = false;
+}
+
+ModelTraffic traffic_of(int model) {
+    ModelTraffic mt;
+    mt.elementwise = (model == RFAST_MODEL_QUAD_DIAG);
+    mt.data_streams = mt.elementwise ? 2 : 0;
+    return mt;
+}
+
+int validate_problem(const rfast_problem* p, std::string& err) {
+    auto bad = [&](const char* m) { err = m; return RFAST_EINVAL; };
+    if (!p) return bad("problem is null");
+    if (p->n <= 0 || p->n > 65535) return bad("n must be in [1, 65535]");
+    if (p->p <= 0) return bad("p must be positive");
+    if (!(p->alpha == p->alpha)) return bad("alpha is NaN");
+    switch (p->model) {
+        case RFAST_MODEL_QUAD_DIAG:
+            if (!p->quad_d || !p->quad_b) return bad("QUAD_DIAG needs quad_d and quad_b");
+            if (p->batch != 0) return bad("QUAD_DIAG takes batch = 0");
+            break;
+        case RFAST_MODEL_LEAST_SQUARES:
+            if (!p->feat || !p->target || p->rows <= 0) return bad("LEAST_SQUARES needs feat, target, rows");
+            if (p->n_features != p->p) return bad("LEAST_SQUARES needs n_features = p");
+            if (p->batch < 0 || p->batch > 4096 || p->rows > (p->batch ? 1 << 30 : 4096))
+                return bad("LEAST_SQUARES: batch (or the whole shard when batch = 0) is limited to 4096 rows");
+            break;
+        case RFAST_MODEL_SOFTMAX:
+            if (!p->feat || !p->label || p->rows <= 0 || p->batch <= 0) return bad("SOFTMAX needs feat, label, rows, batch");
+            if (p->n_classes < 2 || p->n_features <= 0 || p->p != (int64_t)p->n_classes * p->n_features + p->n_classes)
+                return bad("SOFTMAX needs p = C*F + C");
+            if ((int64_t)p->batch * p->n_classes > 8192) return bad("SOFTMAX: batch * classes limited to 8192");
+            break;
+        case RFAST_MODEL_MLP:
+            if (!p->feat || !p->label || p->rows <= 0 || p->batch <= 0) return bad("MLP needs feat, label, rows, batch");
+            if (p->p != (int64_t)p->n_hidden * p->n_features + p->n_hidden + (int64_t)p->n_classes * p->n_hidden + p->n_classes)
+                return bad("MLP needs p = H*F + H + C*H + C");
+            break;
+        case RFAST_MODEL_LOGISTIC_SPARSE:
+            if (!p->sp_rowptr || !p->sp_col || !p->sp_val || !p->label || p->rows <= 0 || p->batch <= 0)
+                return bad("LOGISTIC_SPARSE needs sp_rowptr, sp_col, sp_val, label, rows, batch");
+            if (p->p > 0x7fffffff) return bad("LOGISTIC_SPARSE: p limited to 2^31 - 1");
+            break;
+        default:
+            return bad("unknown model");
+    }
+    return RFAST_OK;
+}
+
+dim3 tile_grid(int n4, int U, int events) { return dim3((n4 + kThreads * U - 1) / (kThreads * U), events); }
+
+// sample gradients of `nev` events (descriptors on the device) into gbuf[par^1]
+int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
+    GradArgs g{};
+    g.ev = d_ev; g.x = ctx->x; g.gbuf = ctx->gbuf; g.stride = ctx->stride;
+    g.gplane = (int64_t)ctx->n * ctx->stride;
+    g.batch_idx = ctx->d_batch_idx; g.rows = ctx->rows; g.F = ctx->F; g.C = ctx->C; g.H = ctx->H;
+    g.p = ctx->p; g.l2 = ctx->l2;
+    cudaStream_t st = ctx->stream;
+    switch (ctx->model) {
+        case RFAST_MODEL_LEAST_SQUARES: {
+            const int use_all = ctx->batch == 0;
+            g.B = use_all ? ctx->rows : ctx->batch;
+            k_ls_residual<<<dim3((g.B + 7) / 8, nev), 256, 0, st>>>(g, ctx->feat, ctx->target, ctx->scratch, use_all);
+            k_ls_grad<<<dim3((g.F + 255) / 256, nev), 256, 0, st>>>(g, ctx->feat, ctx->scratch, use_all);
+            ctx->launches += 2;
+            break;
+        }
+        case RFAST_MODEL_SOFTMAX: {
+            g.B = ctx->batch;
+            k_softmax_logits<<<dim3(g.B, nev), 256, 0, st>>>(g, ctx->feat, ctx->scratch);
+            const size_t sm = (size_t)g.B * g.C * sizeof(float) + (size_t)g.B * sizeof(int);
+            k_softmax_grad<<<dim3((unsigned)((g.p + 255) / 256), nev), 256, sm, st>>>(g, ctx->feat, ctx->label, ctx->scratch);
+            ctx->launches += 2;
+            break;
+        }
+        case RFAST_MODEL_LOGISTIC_SPARSE: {
+            g.B = ctx->batch;
+            k_logit_coef<<<dim3((g.B + 7) / 8, nev), 256, 0, st>>>(g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->label, ctx->scratch);
+            k_logit_grad<<<dim3((unsigned)((g.p + kLogitTile - 1) / kLogitTile), nev), 256, 0, st>>>(
+                g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->scratch);
+            ctx->launches += 2;
+            break;
+        }
+        case RFAST_MODEL_MLP: {
+            g.B = ctx->batch;
+            int rc = mlp_grad_launch(ctx->mlp, g, ctx->xb, ctx->label, nev, st, &ctx->launches, ctx->err);
+            if (rc != RFAST_OK) return rc;
+            break;
+        }
+        default:
+            break;
+    }
+    CK(cudaGetLastError());
+    return RFAST_OK;
+}
+
+int reset_state(rfast_ctx* ctx) {
+    const size_t plane = (size_t)ctx->n * ctx->stride * sizeof(float);
+    if (ctx->x0) CK(cudaMemcpyAsync(ctx->x, ctx->x0, plane, cudaMemcpyDeviceToDevice, ctx->stream));
+    else CK(cudaMemsetAsync(ctx->x, 0, plane, ctx->stream));
+    const int n4 = (int)(ctx->stride / 4);
+    if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
+        k_quad_grad<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
+            ctx->x, ctx->quad_d, ctx->quad_b, ctx->z, ctx->stride, n4);
+        CK(cudaGetLastError());
+    } else {
+        CK(cudaMemsetAsync(ctx->gbuf, 0, 2 * plane, ctx->stream));
+        if (ctx->model == RFAST_MODEL_MLP) {      // bf16 copy of x0 for the matrix products
+            k_rows_to_bf16<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
+                ctx->x, ctx->xb, ctx->stride, n4);
+            CK(cudaGetLastError());
+        }
+        // z_i^0 = g_i^0 = grad f_i(x_i^0; zeta_i^0)  (initialisation line of Algorithm 1)
+        int rc = launch_gradients(ctx, ctx->d_init_ev, ctx->n);
+        if (rc != RFAST_OK) return rc;
+        CK(cudaMemcpyAsync(ctx->z, ctx->gbuf, plane, cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    ctx->round = 0;
+    return RFAST_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rfast_version(void) { return "rfast-b200 0.1 (sm_100a)"; }
+
+const char* rfast_last_error(const rfast_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+void rfast_destroy(rfast_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    free_schedule(c);
+    if (c->mlp) mlp_plan_destroy(c->mlp);
+    void* ptrs[] = {c->x, c->z, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
+                    c->sp_ptr, c->sp_col, c->sp_val, c->xb};
+    for (void* q : ptrs) if (q) cudaFree(q);
+    delete c;
+}
+
+int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) try {
+    if (!out) return set_err(nullptr, RFAST_EINVAL, "out is null");
+    *out = nullptr;
+    std::string err;
+    int rc = validate_problem(prob, err);
+    if (rc != RFAST_OK) return set_err(nullptr, rc, err);
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+        cudaGetLastError();
+        return set_err(nullptr, RFAST_ECUDA, "no CUDA device: this library has no CPU path");
+    }
+    rfast_ctx* ctx = new rfast_ctx();
+    struct Guard { rfast_ctx* c; ~Guard() { if (c) { g_create_error = c->err; rfast_destroy(c); } } } guard{ctx};
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->n = prob->n; ctx->root = prob->root; ctx->p = prob->p; ctx->alpha = prob->alpha; ctx->l2 = prob->l2;
+    ctx->model = prob->model; ctx->batch = prob->batch; ctx->rows = prob->rows;
+    ctx->F = prob->n_features; ctx->C = prob->n_classes; ctx->H = prob->n_hidden;
+    ctx->stride = (prob->p + 31) / 32 * 32;
+    if (ctx->stride / 4 > 0x7fffffff) return set_err(ctx, RFAST_EINVAL, "p too large");
+    if ((rc = build_host_graph(prob->G_R, ctx->n, true, ctx->R, err)) != RFAST_OK) return set_err(ctx, rc, "G_R: " + err);
+    if ((rc = build_host_graph(prob->G_C, ctx->n, false, ctx->Cg, err)) != RFAST_OK) return set_err(ctx, rc, "G_C: " + err);
+    if ((rc = check_roots(ctx->R, ctx->Cg, ctx->root, err)) != RFAST_OK) return set_err(ctx, rc, err);
+
+    const size_t plane = (size_t)ctx->n * ctx->stride;
+    CK(dev_alloc(ctx, &ctx->x, plane));
+    CK(dev_alloc(ctx, &ctx->z, plane));
+    if (prob->x0) {
+        CK(dev_alloc(ctx, &ctx->x0, plane));
+        if ((rc = upload_rows(ctx, ctx->x0, prob->x0, ctx->n)) != RFAST_OK) return rc;
+    }
+    const size_t nrows = (size_t)ctx->n * ctx->rows;
+    switch (ctx->model) {
+        case RFAST_MODEL_QUAD_DIAG:
+            CK(dev_alloc(ctx, &ctx->quad_d, plane));
+            CK(dev_alloc(ctx, &ctx->quad_b, plane));
+            if ((rc = upload_rows(ctx, ctx->quad_d, prob->quad_d, ctx->n)) != RFAST_OK) return rc;
+            if ((rc = upload_rows(ctx, ctx->quad_b, prob->quad_b, ctx->n)) != RFAST_OK) return rc;
+            break;
+        case RFAST_MODEL_LEAST_SQUARES:
+        case RFAST_MODEL_SOFTMAX:
+        case RFAST_MODEL_MLP:
+            CK(dev_alloc(ctx, &ctx->feat, nrows * ctx->F));
+            CK(cudaMemcpyAsync(ctx->feat, prob->feat, nrows * ctx->F * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+            if (ctx->model == RFAST_MODEL_LEAST_SQUARES) {
+                CK(dev_alloc(ctx, &ctx->target, nrows));
+                CK(cudaMemcpyAsync(ctx->target, prob->target, nrows * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+            } else {
+                for (size_t k = 0; k < nrows; ++k)
+                    if (prob->label[k] < 0 || prob->label[k] >= ctx->C) return set_err(ctx, RFAST_EINVAL, "label out of range");
+                CK(dev_alloc(ctx, &ctx->label, nrows));
+                CK(cudaMemcpyAsync(ctx->label, prob->label, nrows * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+            }
+            break;
+        case RFAST_MODEL_LOGISTIC_SPARSE: {
+            const int64_t nnz = prob->sp_rowptr[nrows];
+            if (prob->sp_rowptr[0] != 0 || nnz < 0) return set_err(ctx, RFAST_EINVAL, "sp_rowptr must start at 0");
+            for (size_t r = 0; r < nrows; ++r) {
+                if (prob->sp_rowptr[r + 1] < prob->sp_rowptr[r]) return set_err(ctx, RFAST_EINVAL, "sp_rowptr decreases");
+                for (int64_t q = prob->sp_rowptr[r]; q < prob->sp_rowptr[r + 1]; ++q) {
+                    if (prob->sp_col[q] < 0 || prob->sp_col[q] >= ctx->p ||
+                        (q > prob->sp_rowptr[r] && prob->sp_col[q - 1] >= prob->sp_col[q]))
+                        return set_err(ctx, RFAST_EINVAL, "sp_col must be strictly ascending inside a row and below p");
+                }
+                if (prob->label[r] != 1 && prob->label[r] != -1) return set_err(ctx, RFAST_EINVAL, "labels must be -1 or +1");
+            }
+            CK(dev_alloc(ctx, &ctx->sp_ptr, nrows + 1));
+            CK(dev_alloc(ctx, &ctx->sp_col, (size_t)nnz));
+            CK(dev_alloc(ctx, &ctx->sp_val, (size_t)nnz));
+            CK(dev_alloc(ctx, &ctx->label, nrows));
+            CK(cudaMemcpyAsync(ctx->sp_ptr, prob->sp_rowptr, (nrows + 1) * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream));
+            CK(cudaMemcpyAsync(ctx->sp_col, prob->sp_col, (size_t)nnz * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+            CK(cudaMemcpyAsync(ctx->sp_val, prob->sp_val, (size_t)nnz * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+            CK(cudaMemcpyAsync(ctx->label, prob->label, nrows * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+            break;
+        }
+    }
+    if (ctx->model != RFAST_MODEL_QUAD_DIAG) CK(dev_alloc(ctx, &ctx->gbuf, 2 * plane));
+    if (ctx->model == RFAST_MODEL_MLP) {
+        CK(dev_alloc(ctx, &ctx->xb, plane));
+        CK(cudaMemsetAsync(ctx->xb, 0, plane * sizeof(__nv_bfloat16), ctx->stream));
+        size_t mb = 0;
+        rc = mlp_plan_create(ctx->n, ctx->rows, ctx->F, ctx->H, ctx->C, ctx->batch, ctx->stride, ctx->n,
+                             ctx->feat, &ctx->mlp, &mb, err);
+        if (rc != RFAST_OK) return set_err(ctx, rc, err);
+        ctx->dev_bytes += mb;
+    }
+    CK(cudaStreamSynchronize(ctx->stream));    // the caller's arrays may go away now
+    guard.c = nullptr;
+    *out = ctx;
+    return RFAST_OK;
+} catch (const std::bad_alloc&) {
+    return set_err(nullptr, RFAST_ENOMEM, "host allocation failed");
+} catch (...) {
+    return set_err(nullptr, RFAST_EINVAL, "unexpected failure in rfast_create");
+}
+
+int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
+    if (!ctx) return RFAST_EINVAL;
+    CK(cudaStreamSynchronize(ctx->stream));
+    Compiled comp;
+    std::string err;
+    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model), comp, err);
+    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+    free_schedule(ctx);
+    ctx->comp = std::move(comp);
+    Compiled& c = ctx->comp;
+    ctx->max_round_events = 0;
+    for (int r = 0; r < c.K; ++r) ctx->max_round_events = std::max(ctx->max_round_events, c.act_ptr[r + 1] - c.act_ptr[r]);
+    if ((rc = upload(ctx, &ctx->d_ev, c.ev))) return rc;
+    if ((rc = upload(ctx, &ctx->d_mix_slot, c.mix_slot))) return rc;
+    if ((rc = upload(ctx, &ctx->d_mix_w, c.mix_w))) return rc;
+    if ((rc = upload(ctx, &ctx->d_news_new, c.news_new))) return rc;
+    if ((rc = upload(ctx, &ctx->d_news_prev, c.news_prev))) return rc;
+    if ((rc = upload(ctx, &ctx->d_out_cur, c.out_cur))) return rc;
+    if ((rc = upload(ctx, &ctx->d_out_new, c.out_new))) return rc;
+    if ((rc = upload(ctx, &ctx->d_out_a, c.out_a))) return rc;
+    std::vector<int> bidx;
+    if (ctx->batch > 0) bidx.assign(s->batch_idx, s->batch_idx + s->n_batch_idx);
+    if ((rc = upload(ctx, &ctx->d_batch_idx, bidx))) return rc;
+    std::vector<EvDesc> init(ctx->n);
+    for (int i = 0; i < ctx->n; ++i) {
+        EvDesc d{};
+        d.node = i; d.v_out = -1; d.g_par = 1; d.sample = i;     // result lands in gradient buffer 0
+        init[i] = d;
+    }
+    if ((rc = upload(ctx, &ctx->d_init_ev, init))) return rc;
+    CK(dev_alloc(ctx, &ctx->vbuf, (size_t)c.n_v_slots * ctx->stride, true));
+    CK(dev_alloc(ctx, &ctx->rbuf, (size_t)c.n_rho_slots * ctx->stride, true));
+    CK(cudaMemsetAsync(ctx->vbuf, 0, std::max<size_t>(1, (size_t)c.n_v_slots * ctx->stride) * sizeof(float), ctx->stream));
+    CK(cudaMemsetAsync(ctx->rbuf, 0, std::max<size_t>(1, (size_t)c.n_rho_slots * ctx->stride) * sizeof(float), ctx->stream));
+    // scratch of the two-phase gradients: residuals / logits / coefficients per (event, row[, class])
+    size_t per_ev = 0;
+    if (ctx->model == RFAST_MODEL_LEAST_SQUARES) per_ev = ctx->batch ? ctx->batch : ctx->rows;
+    if (ctx->model == RFAST_MODEL_SOFTMAX) per_ev = (size_t)ctx->batch * ctx->C;
+    if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) per_ev = ctx->batch;
+    CK(dev_alloc(ctx, &ctx->scratch, per_ev * std::max(ctx->n, ctx->max_round_events), true));
+    ctx->has_sched = true;
+    rc = reset_state(ctx);
+    if (rc != RFAST_OK) return rc;
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+} catch (const std::bad_alloc&) {
+    return set_err(ctx, RFAST_ENOMEM, "host allocation failed");
+} catch (...) {
+    return set_err(ctx, RFAST_EINVAL, "unexpected failure in rfast_load_schedule");
+}
+
+int rfast_reset(rfast_ctx* ctx) {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    return reset_state(ctx);
+}
+
+int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (rounds < 0 || ctx->round + (int64_t)rounds > ctx->comp.K)
+        return set_err(ctx, RFAST_ESTATE, "run would pass the end of the schedule");
+    const Compiled& c = ctx->comp;
+    RoundArgs a{};
+    a.mix_slot = ctx->d_mix_slot; a.mix_w = ctx->d_mix_w;
+    a.news_new = ctx->d_news_new; a.news_prev = ctx->d_news_prev;
+    a.out_cur = ctx->d_out_cur; a.out_new = ctx->d_out_new; a.out_a = ctx->d_out_a;
+    a.x = ctx->x; a.z = ctx->z; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
+    a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
+    const bool big = a.n4 >= kThreads * 4;
+    for (int r = ctx->round; r < ctx->round + rounds; ++r) {
+        const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
+        if (nev == 0) continue;
+        a.ev = ctx->d_ev + c.act_ptr[r];
+        if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
+            if (big) k_fused_quad<2><<<tile_grid(a.n4, 2, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
+            else k_fused_quad<1><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
+            ctx->launches += 1;
+        } else {
+            if (ctx->model == RFAST_MODEL_MLP) k_mix<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb);
+            else k_mix<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr);
+            ctx->launches += 1;
+            int rc = launch_gradients(ctx, a.ev, nev);
+            if (rc != RFAST_OK) return rc;
+            k_track<1><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
+            ctx->launches += 1;
+        }
+    }
+    CK(cudaGetLastError());
+    ctx->round += rounds;
+    if (sync) CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
+int rfast_sync(rfast_ctx* ctx) {
+    if (!ctx) return RFAST_EINVAL;
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
+int64_t rfast_query(rfast_ctx* ctx, int what) {
+    if (!ctx) return RFAST_EINVAL;
+    const Compiled& c = ctx->comp;
+    const bool hs = ctx->has_sched;
+    switch (what) {
+        case RFAST_Q_ROUND: return ctx->round;
+        case RFAST_Q_EVENTS_TOTAL: return hs ? c.n_events : 0;
+        case RFAST_Q_EVENTS_RUN: return hs ? c.act_ptr[ctx->round] : 0;
+        case RFAST_Q_LAUNCHES: return ctx->launches;
+        case RFAST_Q_BYTES_RUN: return hs ? c.round_streams[ctx->round] * 4 * ctx->p : 0;
+        case RFAST_Q_BYTES_TOTAL: return hs ? c.round_streams[c.K] * 4 * ctx->p : 0;
+        case RFAST_Q_V_SLOTS: return hs ? c.n_v_slots : 0;
+        case RFAST_Q_RHO_SLOTS: return hs ? c.n_rho_slots : 0;
+        case RFAST_Q_DEVICE_BYTES: return (int64_t)ctx->dev_bytes;
+        case RFAST_Q_N_USED_TAU_V: return hs ? (int64_t)c.used_tau_v.size() : 0;
+        case RFAST_Q_N_USED_TAU_RHO: return hs ? (int64_t)c.used_tau_rho.size() : 0;
+        default: return set_err(ctx, RFAST_EINVAL, "unknown counter");
+    }
+}
+
+int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
+    if (!ctx || !dst) return RFAST_EINVAL;
+    const Compiled& c = ctx->comp;
+    auto ints = [&](const int* src, size_t cnt) {
+        if (bytes != cnt * sizeof(int)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
+        std::memcpy(dst, src, bytes);
+        return RFAST_OK;
+    };
+    const int n = ctx->n, n4 = (int)(ctx->stride / 4);
+    auto rows_out = [&](const float* dev, int64_t rows) -> int {
+        if (bytes != (size_t)rows * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
+        if (rows == 0) return RFAST_OK;
+        CK(cudaMemcpy2DAsync(dst, ctx->p * sizeof(float), dev, ctx->stride * sizeof(float), ctx->p * sizeof(float),
+                             rows, cudaMemcpyDeviceToHost, ctx->stream));
+        CK(cudaStreamSynchronize(ctx->stream));
+        return RFAST_OK;
+    };
+    // rows picked by index from a pool, staged through a temporary
+    auto gathered = [&](const float* pool, const std::vector<int>& idx) -> int {
+        const int64_t rows = (int64_t)idx.size();
+        if (bytes != (size_t)rows * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
+        if (rows == 0) return RFAST_OK;
+        float* tmp = nullptr; int* didx = nullptr;
+        CK(cudaMalloc((void**)&tmp, (size_t)rows * ctx->stride * sizeof(float)));
+        cudaError_t e = cudaMalloc((void**)&didx, rows * sizeof(int));
+        if (e != cudaSuccess) { cudaFree(tmp); return set_err(ctx, RFAST_ENOMEM, "read_state: temporary"); }
+        cudaMemcpyAsync(didx, idx.data(), rows * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
+        k_gather_rows<<<dim3((n4 + kThreads - 1) / kThreads, (unsigned)rows), kThreads, 0, ctx->stream>>>(
+            pool, didx, tmp, ctx->stride, ctx->stride, n4);
+        int rc = rows_out(tmp, rows);
+        cudaStreamSynchronize(ctx->stream);
+        cudaFree(tmp); cudaFree(didx);
+        return rc;
+    };
+    switch (which) {
+        case RFAST_STATE_X: return rows_out(ctx->x, n);
+        case RFAST_STATE_Y: return rows_out(ctx->z, n);
+        case RFAST_STATE_ROUND: return ints(&ctx->round, 1);
+        default: break;
+    }
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    // replay of the integer bookkeeping up to the current round
+    std::vector<int> t(n, 0);
+    const int ev_end = c.act_ptr[ctx->round];
+    for (int ev = 0; ev < ev_end; ++ev) t[c.act_node[ev]]++;
+    switch (which) {
+        case RFAST_STATE_T_LOCAL: return ints(t.data(), n);
+        case RFAST_STATE_USED_TAU_V: return ints(c.used_tau_v.data(), c.used_tau_v.size());
+        case RFAST_STATE_USED_TAU_RHO: return ints(c.used_tau_rho.data(), c.used_tau_rho.size());
+        case RFAST_STATE_TAU_V_END: return ints(c.tau_v_end.data(), c.tau_v_end.size());
+        case RFAST_STATE_TAU_RHO_END: return ints(c.tau_rho_end.data(), c.tau_rho_end.size());
+        case RFAST_STATE_G_LAST: {
+            if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
+                if (bytes != (size_t)n * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
+                float* tmp = nullptr;
+                CK(cudaMalloc((void**)&tmp, (size_t)n * ctx->stride * sizeof(float)));
+                k_quad_grad<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(
+                    ctx->x, ctx->quad_d, ctx->quad_b, tmp, ctx->stride, n4);
+                int rc = rows_out(tmp, n);
+                cudaStreamSynchronize(ctx->stream);
+                cudaFree(tmp);
+                return rc;
+            }
+            std::vector<int> idx(n);
+            for (int i = 0; i < n; ++i) idx[i] = (t[i] & 1) * n + i;
+            return gathered(ctx->gbuf, idx);
+        }
+        case RFAST_STATE_RHO_LATEST:
+        case RFAST_STATE_RHO_BUF: {
+            std::vector<int> idx(ctx->Cg.E, -1);
+            for (int ev = 0; ev < ev_end; ++ev) {
+                const EvDesc& d = c.ev[ev];
+                if (which == RFAST_STATE_RHO_LATEST)
+                    for (int k = 0; k < d.out_cnt; ++k) idx[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
+                else
+                    for (int k = 0; k < d.news_cnt; ++k) idx[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
+            }
+            return gathered(ctx->rbuf, idx);
+        }
+        default: return set_err(ctx, RFAST_EINVAL, "read_state: unknown view");
+    }
+} catch (...) {
+    return set_err(ctx, RFAST_ENOMEM, "read_state: host allocation failed");
+}
+
+int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32_t* used_tau_v,
+                       int32_t* used_tau_rho, int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
+                       char* errbuf, size_t err_len) try {
+    std::string err;
+    auto done = [&](int rc) {
+        if (errbuf && err_len) { std::snprintf(errbuf, err_len, "%s", err.c_str()); }
+        return rc;
+    };
+    if (!prob || prob->n <= 0) { err = "problem is null or n <= 0"; return done(RFAST_EINVAL); }
+    HostGraph R, C;
+    int rc;
+    if ((rc = build_host_graph(prob->G_R, prob->n, true, R, err)) != RFAST_OK) return done(rc);
+    if ((rc = build_host_graph(prob->G_C, prob->n, false, C, err)) != RFAST_OK) return done(rc);
+    if ((rc = check_roots(R, C, prob->root, err)) != RFAST_OK) return done(rc);
+    Compiled c;
+    if ((rc = compile_schedule(R, C, s, prob->batch, prob->rows, traffic_of(prob->model), c, err)) != RFAST_OK) return done(rc);
+    if (used_tau_v) std::copy(c.used_tau_v.begin(), c.used_tau_v.end(), used_tau_v);
+    if (used_tau_rho) std::copy(c.used_tau_rho.begin(), c.used_tau_rho.end(), used_tau_rho);
+    if (v_ver)
+        for (int64_t ev = 0; ev < c.n_events; ++ev) {
+            v_ver[3 * ev] = c.v_slot[ev]; v_ver[3 * ev + 1] = c.v_write[ev]; v_ver[3 * ev + 2] = c.v_last[ev];
+        }
+    if (rho_ver)
+        for (size_t v = 0; v < c.rho_slot.size(); ++v) {
+            rho_ver[3 * v] = c.rho_slot[v]; rho_ver[3 * v + 1] = c.rho_write[v]; rho_ver[3 * v + 2] = c.rho_last[v];
+        }
+    if (counts) {
+        counts[0] = c.n_v_slots; counts[1] = c.n_rho_slots; counts[2] = c.n_events; counts[3] = c.round_streams[c.K];
+    }
+    return done(RFAST_OK);
+} catch (...) {
+    if (errbuf && err_len) std::snprintf(errbuf, err_len, "host allocation failed");
+    return RFAST_ENOMEM;
+}
+
+}  // extern "C"

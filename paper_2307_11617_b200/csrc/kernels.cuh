@@ -282,16 +282,6 @@ k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
 // Sample gradients.  Every kernel takes the round's events; x_i is the freshly mixed row and
 // the result goes to gbuf[par^1][node].  Reductions run in a fixed order (run-to-run identical).
 // ---------------------------------------------------------------------------------------------
-struct GradArgs {
-    const EvDesc* ev;
-    const float*  x;          // [n][stride]
-    float*        gbuf;       // [2][n][stride]
-    int64_t stride, gplane;
-    const int*    batch_idx;  // [(n + events) * B]
-    int B, rows, F, C, H;
-    int64_t p;
-    float l2;
-};
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -456,6 +446,20 @@ k_gather_rows(const float* __restrict__ src, const int* __restrict__ idx, float*
     float4 v = make_float4(0, 0, 0, 0);
     if (r >= 0) v = reinterpret_cast<const float4*>(src + (int64_t)r * src_stride)[i4];
     reinterpret_cast<float4*>(dst + (int64_t)blockIdx.y * dst_stride)[i4] = v;
+}
+
+// bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)
+__global__ void __launch_bounds__(kThreads)
+k_rows_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int n4) {
+    const int i4 = blockIdx.x * kThreads + threadIdx.x;
+    if (i4 >= n4) return;
+    const int64_t row = (int64_t)blockIdx.y * stride;
+    const float4 v = reinterpret_cast<const float4*>(src + row)[i4];
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(dst + row)[i4] = pk;
 }
 
 }  // namespace rfast

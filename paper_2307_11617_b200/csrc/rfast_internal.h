@@ -58,6 +58,18 @@ struct Compiled {
     std::vector<int64_t> round_streams;   // [K+1]
 };
 
+// Arguments shared by the sample-gradient kernels.
+struct GradArgs {
+    const EvDesc* ev;
+    const float*  x;          // [n][stride]
+    float*        gbuf;       // [2][n][stride]
+    int64_t stride, gplane;
+    const int*    batch_idx;  // [(n + events) * B]
+    int B, rows, F, C, H;
+    int64_t p;
+    float l2;
+};
+
 // What the byte accounting needs to know about the model.
 struct ModelTraffic {
     bool elementwise = false;   // one fused pass, gradient recomputed instead of stored

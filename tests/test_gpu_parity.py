@@ -1,0 +1,150 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bar: integer artefacts (consumed stamps, counters) bit-exact; x and y within 1e-5 relative L2
+after K rounds, the denominator floored at 1e-3 of the reference's initial norm."""
+
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from conftest import has_cuda
+from oracle import from_workload, make_model, rel_l2, run_schedule
+from workloads import build_config
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+# sizes the oracle finishes in seconds, spanning several tiles and a ragged tail
+CASES = [
+    ("quad_tree64", dict(n=16, p=70_001, K=30), "tiles+tail"),
+    ("quad_tree64", dict(n=64, p=3, K=100), "tiny p"),
+    ("quad_tree64", dict(n=1, p=33, K=5), "single node"),
+    ("quad_tree64", dict(n=64, p=4099, K=100, drop=0.6, max_delay=8), "heavy loss"),
+    ("quad_tree64", dict(n=32, p=2048, K=60, drop=0.0, max_delay=0), "no loss no delay"),
+    ("ls_ring4", {}, "config 1 as stated"),
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=150, batch=8), "reduced softmax"),
+    ("logistic_tree1024", dict(n=96, p=5000, rows=8, K=60, batch=4, nnz=50), "reduced sparse logistic"),
+]
+
+
+def _oracle(wl, K=None):
+    orc = from_workload(wl, make_model(wl).grad)
+    B = wl.batch
+    zeta0 = [wl.schedule.batch_idx[i * B:(i + 1) * B] for i in range(wl.n)] if B else None
+    orc.init_gradients(zeta0)
+    ref0 = (np.linalg.norm(orc.X()), np.linalg.norm(orc.Z()))
+    run_schedule(orc, wl.schedule, K=K)
+    return orc, ref0
+
+
+def _compare(eng, orc, ref0, tol=TOL):
+    from paper_2307_11617_b200 import binding as B
+    x, y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+    assert np.isfinite(x).all() and np.isfinite(y).all()
+    ex, ey = rel_l2(x, orc.X(), ref0[0]), rel_l2(y, orc.Z(), ref0[1])
+    assert ex <= tol and ey <= tol, (ex, ey)
+    g = eng.read(B.STATE_G_LAST)
+    assert rel_l2(g, orc.G(), ref0[1]) <= 10 * tol
+    if len(orc.rho):
+        rl, rb = eng.read(B.STATE_RHO_LATEST), eng.read(B.STATE_RHO_BUF)
+        scale = max(np.linalg.norm(orc.RHO()), ref0[1])
+        assert np.linalg.norm(rl - orc.RHO()) <= 10 * tol * scale
+        assert np.linalg.norm(rb - orc.RHO_TILDE()) <= 10 * tol * scale
+    return ex, ey
+
+
+@pytest.mark.parametrize("name,ov,why", CASES, ids=[c[2] for c in CASES])
+def test_parity_after_K_rounds(rfast_lib, name, ov, why):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config(name, seed=1, **ov)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        # integers: bit-exact
+        assert eng.read(B.STATE_USED_TAU_V).tolist() == orc.used_tau_v
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
+        assert eng.read(B.STATE_T_LOCAL).tolist() == orc.t
+        assert eng.read(B.STATE_TAU_V_END).tolist() == orc.tau_v
+        assert eng.read(B.STATE_TAU_RHO_END).tolist() == orc.tau_rho
+        assert eng.read(B.STATE_ROUND)[0] == wl.schedule.K
+        assert eng.query(B.Q_EVENTS_RUN) == orc.activations
+        assert eng.query(B.Q_LAUNCHES) > 0
+
+
+def test_parity_round_by_round_and_reset(rfast_lib):
+    """Stepping one round at a time gives the same state as one call, and reset + rerun is
+    bit-identical (no atomics, fixed summation order)."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("quad_tree64", seed=7, n=16, p=1500, K=25)
+    orc = from_workload(wl, make_model(wl).grad)
+    orc.init_gradients()
+    ref0 = (1.0, np.linalg.norm(orc.Z()))
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        for r in range(wl.schedule.K):
+            eng.run(1)
+            run_schedule(orc, wl.schedule, K=r + 1)
+            if r % 6 == 0 or r == wl.schedule.K - 1:
+                _compare(eng, orc, ref0)
+                assert eng.read(B.STATE_T_LOCAL).tolist() == orc.t
+        x1, y1 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        eng.reset()
+        assert eng.query(B.Q_ROUND) == 0
+        eng.run()
+        assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
+
+
+def test_conservation_on_the_device_state(rfast_lib):
+    """Lemma 3 on what the GPU holds: trackers plus undelivered mass equal the sum of the
+    latest gradients, up to fp32 rounding of the running sums."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("quad_tree64", seed=3, n=32, p=999, K=80, drop=0.4)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        y, g = eng.read(B.STATE_Y).astype(np.float64), eng.read(B.STATE_G_LAST).astype(np.float64)
+        rl, rb = eng.read(B.STATE_RHO_LATEST).astype(np.float64), eng.read(B.STATE_RHO_BUF).astype(np.float64)
+    res = y.sum(axis=0) + (rl - rb).sum(axis=0) - g.sum(axis=0)
+    scale = np.abs(g).sum(axis=0).max()
+    assert np.abs(res).max() <= 1e-5 * scale
+
+
+def test_run_past_the_schedule_is_refused(rfast_lib):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import ESTATE, RFastError
+    wl = build_config("quad_tree64", n=4, p=8, K=3)
+    with pkg.Engine(wl) as eng:
+        with pytest.raises(RFastError) as ei:
+            eng.run(1)                      # no schedule yet
+        assert ei.value.code == ESTATE
+        eng.load_schedule(wl.schedule)
+        eng.run(3)
+        with pytest.raises(RFastError) as ei:
+            eng.run(1)
+        assert ei.value.code == ESTATE
+
+
+def test_empty_rounds_and_x0(rfast_lib):
+    """Rounds without any active node are legal; a non-zero x0 is honoured."""
+    import paper_2307_11617_b200 as pkg
+    wl = build_config("quad_tree64", seed=9, n=8, p=40, K=12)
+    s = wl.schedule
+    # empty out rounds 2 and 5 (their events and codes are removed consistently)
+    from workloads import make_schedule
+    acts = [s.act_node[s.act_ptr[r]:s.act_ptr[r + 1]] for r in range(s.K)]
+    acts[2] = acts[2][:0]; acts[5] = acts[5][:0]
+    rng = np.random.default_rng(0)
+    wl.schedule = make_schedule(wl.G_R, wl.G_C, acts, 0.2, 3, rng)
+    wl.x0 = rng.standard_normal((wl.n, wl.p)).astype(np.float32)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)

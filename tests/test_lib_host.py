@@ -1,0 +1,166 @@
+"""Host-side logic of the CUDA library, checked without a GPU: exported symbols, the schedule
+compiler's integer artefacts against the oracle and against brute force, safety of the version
+rows, input validation."""
+
+from __future__ import annotations
+
+import copy
+import os
+import re
+
+import numpy as np
+import pytest
+
+from helpers import brute_force_stamps, out_edges
+from oracle import from_workload, make_model, run_schedule
+from workloads import build_config, graph_from_edges
+
+CASES = [
+    ("ls_ring4", {}),
+    ("softmax_exp16", dict(F=12, C=4, rows=16, K=120, batch=4)),
+    ("mlp_tree64", dict(F=10, H=6, C=3, rows=12, K=60, batch=4)),
+    ("quad_tree64", dict(p=19, K=100)),
+    ("logistic_tree1024", dict(n=150, p=300, rows=4, K=60, batch=2, nnz=6)),
+]
+
+
+def test_library_exports_every_declared_symbol(rfast_lib, repo_root):
+    text = open(os.path.join(repo_root, "include", "rfast.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = set(re.findall(r"\b(rfast_[a-z_]+)\s*\(", text))
+    assert {"rfast_create", "rfast_load_schedule", "rfast_run", "rfast_read_state"} <= names
+    for nm in names:
+        assert hasattr(rfast_lib, nm), nm
+
+
+@pytest.mark.parametrize("name,ov", CASES)
+def test_compiled_stamps_equal_oracle_and_brute_force(rfast_lib, name, ov):
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=2, **ov)
+    r = pkg.rfast_compile_host(wl, wl.schedule)
+    sv, _ = brute_force_stamps(wl.G_R, wl.schedule, wl.schedule.send_r)
+    sr, _ = brute_force_stamps(wl.G_C, wl.schedule, wl.schedule.send_c)
+    assert list(r["used_tau_v"]) == sv and list(r["used_tau_rho"]) == sr
+    if name != "mlp_tree64":                          # the oracle's MLP is slow; stamps are value-free
+        orc = from_workload(wl, make_model(wl).grad)
+        run_schedule(orc, wl.schedule)
+        assert list(r["used_tau_v"]) == orc.used_tau_v and list(r["used_tau_rho"]) == orc.used_tau_rho
+    assert r["events"] == wl.schedule.n_events
+
+
+@pytest.mark.parametrize("name,ov", CASES)
+def test_version_rows_never_alias_a_live_version(rfast_lib, name, ov):
+    """Two versions may share a row only if the first is dead before the second is written;
+    every consumed version is alive, in its own row, when it is read."""
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=5, **ov)
+    s = wl.schedule
+    r = pkg.rfast_compile_host(wl, s)
+    ev_round = np.repeat(np.arange(s.K), np.diff(s.act_ptr))
+    # --- v versions: one per event
+    v = r["v_ver"]
+    assert (v[:, 1] == ev_round).all()
+    by_row = {}
+    for ev in np.argsort(v[:, 1], kind="stable"):
+        row, wr, last = v[ev]
+        if row < 0:
+            continue
+        assert 0 <= row < r["v_rows"] and last >= wr
+        if row in by_row:
+            assert by_row[row] < wr, "row reused while its version was still to be read"
+        by_row[row] = last
+    # --- rho versions: one per (event, out-edge in G_C)
+    rho = r["rho_ver"]
+    outC = out_edges(wl.G_C)
+    edge_of, stamp_of = [], []
+    t = [0] * wl.n
+    for ev, i in enumerate(s.act_node):
+        t[i] += 1
+        for f in outC[i]:
+            edge_of.append(f); stamp_of.append(t[i])
+    assert len(edge_of) == len(rho)
+    owner = {}
+    for vid in np.argsort(rho[:, 1], kind="stable"):
+        row, wr, last = rho[vid]
+        assert 0 <= row < r["rho_rows"] and last >= wr
+        if row in owner:
+            pl, pe, ps = owner[row]
+            in_place = (pe == edge_of[vid] and ps + 1 == stamp_of[vid] and pl == wr)
+            assert pl < wr or in_place, "rho row reused while its version was still to be read"
+        owner[row] = (last, edge_of[vid], stamp_of[vid])
+    # --- every consumed version is inside its lifetime
+    sv, _ = brute_force_stamps(wl.G_R, s, s.send_r)
+    ev_of = [[] for _ in range(wl.n)]
+    for ev, i in enumerate(s.act_node):
+        ev_of[i].append(ev)
+    k = 0
+    for ev, i in enumerate(s.act_node):
+        for e in range(wl.G_R.rowptr[i], wl.G_R.rowptr[i + 1]):
+            tau = sv[k]; k += 1
+            if tau >= 1:
+                row, wr, last = v[ev_of[wl.G_R.col[e]][tau - 1]]
+                assert row >= 0 and wr < ev_round[ev] <= last
+    sr, _ = brute_force_stamps(wl.G_C, s, s.send_c)
+    off = np.concatenate([[0], np.cumsum([len(outC[i]) for i in s.act_node])])
+    pos = {f: k for i in range(wl.n) for k, f in enumerate(outC[i])}
+    k = 0
+    prev = [0] * wl.G_C.n_edges
+    for ev, i in enumerate(s.act_node):
+        for e in range(wl.G_C.rowptr[i], wl.G_C.rowptr[i + 1]):
+            tau = sr[k]; k += 1
+            if tau > prev[e]:
+                for st in (tau, prev[e]):
+                    if st >= 1:
+                        row, wr, last = rho[off[ev_of[wl.G_C.col[e]][st - 1]] + pos[e]]
+                        assert wr < ev_round[ev] <= last
+                prev[e] = tau
+
+
+def test_compile_rejects_bad_graphs_and_schedules(rfast_lib):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import EGRAPH, ESCHED, RFastError
+    wl = build_config("quad_tree64", n=8, p=5, K=10)
+    bad = copy.deepcopy(wl)
+    bad.G_R.w = bad.G_R.w * np.float32(0.9)                       # rows of W no longer sum to 1
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_host(bad, bad.schedule)
+    assert ei.value.code == EGRAPH and "Assumption 1" in str(ei.value)
+    bad = copy.deepcopy(wl)
+    bad.G_C.diag = bad.G_C.diag.copy(); bad.G_C.diag[3] = 0.0    # Assumption 1 i)
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_host(bad, bad.schedule)
+    assert ei.value.code == EGRAPH
+    # no common root: G_R a chain 0->1->...; G_C pushes away from node 0
+    n = 4
+    bad = build_config("quad_tree64", n=n, p=5, K=10)
+    bad.G_R = graph_from_edges(n, [(i, i + 1) for i in range(n - 1)], "row")
+    bad.G_C = graph_from_edges(n, [(i, i + 1) for i in range(n - 1)], "col")
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_host(bad, bad.schedule)
+    assert ei.value.code == EGRAPH and "Assumption 2" in str(ei.value)
+    for mutate in ("order", "code", "count", "node"):
+        s = copy.deepcopy(wl.schedule)
+        if mutate == "order":
+            r = int(np.argmax(np.diff(s.act_ptr) >= 2)); a = s.act_ptr[r]
+            s.act_node[a], s.act_node[a + 1] = s.act_node[a + 1], s.act_node[a]
+        elif mutate == "code":
+            s.send_c[0] = -2
+        elif mutate == "count":
+            s.send_r = s.send_r[:-1]
+        else:
+            s.act_node[0] = wl.n
+        with pytest.raises(RFastError) as ei:
+            pkg.rfast_compile_host(wl, s)
+        assert ei.value.code == ESCHED, mutate
+
+
+def test_create_fails_loudly_without_a_device(rfast_lib):
+    from conftest import has_cuda
+    if has_cuda():
+        pytest.skip("a CUDA device is present")
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import ECUDA, RFastError
+    wl = build_config("quad_tree64", n=4, p=5, K=3)
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_create(wl)
+    assert ei.value.code == ECUDA
