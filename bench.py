@@ -1,0 +1,285 @@
+#!/usr/bin/env python
+"""Benchmark of the R-FAST activation engine.
+
+A step is one pass of the whole hot path over one workload: the full seeded schedule
+(K rounds; every activation runs S1 descent, S2a mix, sample gradient, S2b/S2c tracking,
+S3-S5) from the initial state.  Headline metric: node activations per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config quad_tree64] [--impl reference]
+
+One JSON line on stdout (rank 0).  With N > 1 (torchrun) every rank runs an independent replica
+of the workload on its own GPU (the path does not shard: replicas only) and the time is the
+max over ranks.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "node_activations_per_s"
+UNIT = "activations/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.2 and len(r) >= 7] or \
+               [r for (_, r) in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [nm for k, nm in enumerate(names) if any(r[3 + k].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
+                "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
+
+
+def build_workload(name, small=False):
+    from workloads import build_config
+    if small:
+        ov = {"quad_tree64": dict(p=200_000, K=20), "softmax_exp16": dict(K=200, rows=128),
+              "logistic_tree1024": dict(K=20, rows=8), "mlp_tree64": dict(K=10, rows=128),
+              "ls_ring4": {}}[name]
+        return build_config(name, seed=0, **ov)
+    return build_config(name, seed=0)
+
+
+def oracle_sample(wl, budget_s=15.0):
+    """Times the oracle as it stands on a bounded sample of the workload and returns
+    (activations/s scaled to the full workload, description, seconds spent)."""
+    import copy
+    from oracle import from_workload, make_model, run_schedule
+    s = wl.schedule
+    if wl.model == "quad_diag":
+        # the element-wise objective makes coordinates independent: run all n nodes and all K
+        # rounds on a coordinate chunk and scale the time by p / chunk
+        chunk = min(wl.p, 100_000)
+        sub = copy.copy(wl)
+        sub.p = chunk
+        sub.data = {"d": wl.data["d"][:, :chunk], "b": wl.data["b"][:, :chunk]}
+        sub.x0 = None if wl.x0 is None else wl.x0[:, :chunk]
+        t0 = time.perf_counter()
+        orc = from_workload(sub, make_model(sub).grad)
+        run_schedule(orc, s)
+        dt = time.perf_counter() - t0
+        full = dt * (wl.p / chunk)
+        return orc.activations / full, f"all {s.K} rounds, {wl.n} nodes, coordinates [0,{chunk}) of {wl.p}, time scaled by p/chunk", dt
+    # other objectives: as many leading rounds as fit the budget
+    orc = from_workload(wl, make_model(wl).grad)
+    t0 = time.perf_counter()
+    done = 0
+    for r in range(s.K):
+        run_schedule(orc, s, K=r + 1)
+        done = r + 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return orc.activations / dt, f"first {done} of {s.K} rounds, full size", dt
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = build_workload(args.config, args.small)
+    vals, desc = [], ""
+    for _ in range(args.warmup + args.steps):
+        v, desc, _dt = oracle_sample(wl, budget_s=8.0)
+        vals.append(v)
+    v = float(np.mean(vals[args.warmup:]))
+    ev = wl.schedule.n_events
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * ev / v,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl.name, "n": wl.n, "p": wl.p, "rounds": wl.schedule.K},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--config", default="quad_tree64")
+    ap.add_argument("--small", action="store_true", help="reduced size (profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+
+    t_gen = time.perf_counter()
+    wl = build_workload(args.config, args.small)
+    t_gen = time.perf_counter() - t_gen
+    stream = torch.cuda.Stream()
+    t_create = time.perf_counter()
+    eng = pkg.Engine(wl, stream.cuda_stream)
+    t_create = time.perf_counter() - t_create
+    t_load = time.perf_counter()
+    eng.load_schedule(wl.schedule)
+    t_load = time.perf_counter() - t_load
+    events = eng.query(B.Q_EVENTS_TOTAL)
+    bytes_step = eng.query(B.Q_BYTES_TOTAL)
+    K_rounds = wl.schedule.K
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step(timed):
+        eng.reset()                                   # back to round 0; not part of the timed work
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        eng.run(sync=False)
+        e1.record(stream)
+        return (e0, e1)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step(False)
+    barrier()
+    l0 = eng.query(B.Q_LAUNCHES)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    w0 = time.time()
+    pairs = [one_step(True) for _ in range(args.steps)]
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1)
+    launches = eng.query(B.Q_LAUNCHES) - l0
+    ms = [a.elapsed_time(b) for a, b in pairs]
+    ms_step = float(sum(ms) / len(ms))
+    if world > 1:
+        t = torch.tensor([ms_step], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    value = world * events / (ms_step * 1e-3)
+
+    # end to end through the C ABI with host buffers: schedule arrays in (compiled and uploaded),
+    # the run, x and y back into pinned host memory
+    e2e = None
+    if not args.no_e2e:
+        xo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
+        yo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
+        s = wl.schedule
+        h2d = sum(a.nbytes for a in (s.act_ptr, s.act_node, s.send_r, s.send_c, s.batch_idx)) + \
+            64 * events
+        reps = max(1, min(args.steps, 3))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            eng.load_schedule(s)
+            eng.run(sync=False)
+            eng.read(B.STATE_X, xo)
+            eng.read(B.STATE_Y, yo)
+        barrier()
+        dt = (time.perf_counter() - t0) / reps
+        if world > 1:
+            t = torch.tensor([dt], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * events / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3}
+
+    peak, peak_kind = measured_peaks()
+    achieved = bytes_step / (ms_step * 1e-3) / 1e9
+    hbm_bound = wl.model in ("quad_diag", "logistic_sparse", "mlp")
+    roofline = {"bound": "hbm", "kernel": "k_fused_quad" if wl.model == "quad_diag" else "k_mix+gradient+k_track",
+                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
+                "algorithmic_bytes_per_launch": bytes_step / max(1, launches // max(1, args.steps)),
+                "traffic": None,
+                "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        v, desc, dt = oracle_sample(wl)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": wl.name, "n": wl.n, "p": wl.p, "rounds": K_rounds,
+                           "activations_per_step": events, "small": bool(args.small),
+                           "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
+                           "reset_between_steps": "untimed", "parallelism": f"replicas x{world}"},
+                "param_updates_per_s": value * wl.p, "gpu_launches": int(launches),
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+                "setup_s": {"generate": t_gen, "create": t_create, "load_schedule": t_load},
+                "device_bytes": eng.query(B.Q_DEVICE_BYTES),
+                "version_rows": {"v": eng.query(B.Q_V_SLOTS), "rho": eng.query(B.Q_RHO_SLOTS)}}
+        print(json.dumps(line), flush=True)
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
