@@ -83,7 +83,7 @@ class ClockSampler:
 def build_workload(name, small=False):
     from workloads import build_config
     if small:
-        ov = {"quad_tree64": dict(p=200_000, K=20), "softmax_exp16": dict(K=200, rows=128),
+        ov = {"quad_tree64": dict(p=1_500_000, K=20), "softmax_exp16": dict(K=200, rows=128),
               "logistic_tree1024": dict(K=20, rows=8), "mlp_tree64": dict(K=10, rows=128),
               "ls_ring4": {}}[name]
         return build_config(name, seed=0, **ov)
