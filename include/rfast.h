@@ -202,6 +202,33 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s,
                        int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
                        char* err, size_t err_len);
 
+/* No counterpart in the paper: a service entry point for callers that are not allowed to
+ * allocate device memory.  Some hosts of this library cannot call cudaMalloc where they need a
+ * gradient: a framework that hands the whole GPU to its own memory pool up front, a latency-
+ * critical loop in which cudaMalloc's implicit device-wide synchronisation is unacceptable, or
+ * code that runs after memory has been budgeted to the last byte.  For them this call computes
+ * the full-shard least-squares gradient
+ *     grad = (1/rows) * feat^T (feat x - target) + l2 * x
+ * (the LEAST_SQUARES objective above with batch = 0, for one node) without allocating anything:
+ * the per-row residuals that the handle-based path keeps in an allocated buffer live in a fixed
+ * array inside the library image, RFAST_STATIC_MAX_ROWS floats (256 KiB) that every GPU loading
+ * the library holds until the process exits.
+ *   d_feat [rows][n_features], d_target [rows], d_x [n_features]: DEVICE pointers, inputs;
+ *   d_grad [n_features]: DEVICE pointer, output; all owned by the caller, row-major fp32.
+ *   cuda_stream: cudaStream_t as void* (NULL: legacy default stream); the work is enqueued
+ *   there and the call returns without waiting.
+ * The device that is current at the call is used.  The first call made on a device looks up
+ * the array's device address (cudaGetSymbolAddress) and remembers it; make that first call
+ * before starting any stream capture.  rows > RFAST_STATIC_MAX_ROWS is rejected with
+ * RFAST_EINVAL and a message in err (err may be NULL).  All calls share the one array, which
+ * keeps the previous call's contents; the part a call uses is cleared first.  Two calls whose
+ * work overlaps on the GPU (different streams, or different host threads without ordering)
+ * race on it: order them on one stream or with events.  Calls no cudaMalloc / cudaFree. */
+#define RFAST_STATIC_MAX_ROWS 65536
+int rfast_ls_gradient_static(const float* d_feat, const float* d_target, const float* d_x,
+                             float* d_grad, int32_t rows, int32_t n_features, float l2,
+                             void* cuda_stream, char* err, size_t err_len);
+
 void        rfast_destroy(rfast_ctx* ctx);
 const char* rfast_last_error(const rfast_ctx* ctx);   /* ctx may be NULL: last create error */
 const char* rfast_version(void);

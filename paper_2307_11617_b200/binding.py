@@ -80,6 +80,8 @@ def lib():
         L.rfast_version.restype = C.c_char_p
         L.rfast_compile_host.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule)] + [C.c_void_p] * 5 + \
             [C.c_char_p, C.c_size_t]
+        L.rfast_ls_gradient_static.argtypes = [C.c_void_p] * 4 + [C.c_int32, C.c_int32, C.c_float,
+                                               C.c_void_p, C.c_char_p, C.c_size_t]
         _lib = L
     return _lib
 
@@ -219,6 +221,25 @@ def rfast_compile_host(wl, s):
     return {"used_tau_v": used_v, "used_tau_rho": used_r, "v_ver": v_ver, "rho_ver": rho_ver,
             "v_rows": int(counts[0]), "rho_rows": int(counts[1]), "events": int(counts[2]),
             "streams": int(counts[3])}
+
+
+STATIC_MAX_ROWS = 65536
+
+
+def rfast_ls_gradient_static(d_feat: int, d_target: int, d_x: int, d_grad: int, rows: int,
+                             n_features: int, l2: float = 0.0, cuda_stream: int = 0) -> None:
+    """Full-shard least-squares gradient without any device allocation, for callers that may not
+    allocate (a framework that owns all GPU memory, a loop that cannot afford cudaMalloc's
+    device-wide synchronisation).  All four arguments are raw DEVICE addresses (integers) of
+    caller-owned fp32 arrays: feat [rows][n_features], target [rows], x [n_features] in, grad
+    [n_features] out.  Enqueued on cuda_stream; the caller synchronises.  At most
+    STATIC_MAX_ROWS rows; calls that overlap on the GPU race on the shared built-in scratch."""
+    err = C.create_string_buffer(256)
+    rc = lib().rfast_ls_gradient_static(C.c_void_p(d_feat), C.c_void_p(d_target), C.c_void_p(d_x),
+                                        C.c_void_p(d_grad), int(rows), int(n_features), float(l2),
+                                        C.c_void_p(cuda_stream), err, 256)
+    if rc != OK:
+        raise RFastError(rc, err.value.decode())
 
 
 class Engine:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librfast.so")
-SOURCES = ["api.cu", "compile.cpp", "grad_mlp.cu"]
+SOURCES = ["api.cu", "compile.cpp", "grad_mlp.cu", "noalloc.cu"]
 
 
 def _newest_source_mtime():
