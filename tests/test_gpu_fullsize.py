@@ -53,3 +53,48 @@ def test_quad_tree64_full_size_sampled_chunks(rfast_lib):
     d, b = wl.data["d"][:, :width].astype(np.float64), wl.data["b"][:, :width].astype(np.float64)
     xs = (d * d * b).sum(axis=0) / (d * d).sum(axis=0)
     assert np.linalg.norm(x[:, :width] - xs) < np.linalg.norm(xs) * np.sqrt(wl.n)
+
+
+def _run_both(wl, K=None):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    orc = from_workload(wl, make_model(wl).grad)
+    Bsz = wl.batch
+    orc.init_gradients([wl.schedule.batch_idx[i * Bsz:(i + 1) * Bsz] for i in range(wl.n)] if Bsz else None)
+    x0n, z0n = np.linalg.norm(orc.X()), np.linalg.norm(orc.Z())
+    run_schedule(orc, wl.schedule, K=K)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run(K)
+        x, y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        used_v, used_r = eng.read(B.STATE_USED_TAU_V), eng.read(B.STATE_USED_TAU_RHO)
+        t_loc = eng.read(B.STATE_T_LOCAL)
+    ex, ey = rel_l2(x, orc.X(), x0n), rel_l2(y, orc.Z(), z0n)
+    nv, nr = len(orc.used_tau_v), len(orc.used_tau_rho)       # the oracle saw only the first K rounds
+    assert used_v[:nv].tolist() == orc.used_tau_v and used_r[:nr].tolist() == orc.used_tau_rho
+    assert t_loc.tolist() == orc.t
+    return ex, ey
+
+
+def test_softmax_exp16_full_size_5000_rounds(rfast_lib):
+    """Config 2 as stated: n=16, 784x10 softmax (p=7850), minibatch 32, one straggler, 5000 rounds."""
+    wl = build_config("softmax_exp16", seed=0)
+    assert (wl.n, wl.p, wl.batch, wl.schedule.K) == (16, 7850, 32, 5000)
+    ex, ey = _run_both(wl)
+    assert ex <= 1e-5 and ey <= 1e-5, (ex, ey)
+
+
+def test_logistic_tree1024_full_size_first_rounds(rfast_lib):
+    """Config 5 at full size (n=1024, p=100k, 1 % density); the oracle needs ~4 ms per
+    activation there, so the comparison covers the first 6 rounds (about 5.6k activations)."""
+    wl = build_config("logistic_tree1024", seed=0)
+    assert (wl.n, wl.p, wl.batch) == (1024, 100_000, 16)
+    ex, ey = _run_both(wl, K=6)
+    assert ex <= 1e-5 and ey <= 1e-5, (ex, ey)
+
+
+def test_logistic_long_horizon_reduced_dimension(rfast_lib):
+    """All 300 rounds of config 5's schedule shape (stragglers, 30 % loss) at reduced n and p."""
+    wl = build_config("logistic_tree1024", seed=0, n=256, p=2000, nnz=20, rows=16, K=300)
+    ex, ey = _run_both(wl)
+    assert ex <= 1e-5 and ey <= 1e-5, (ex, ey)
