@@ -94,6 +94,10 @@ typedef struct rfast_problem {
     const int32_t* sp_col;    /*                   columns strictly ascending inside a row */
     const float*   sp_val;
     const float*   x0;        /* [n][p] initial iterates, or NULL for zeros */
+    int32_t     compensated;  /* tracker arithmetic of S2b/S2c: 0 = plain fp32; 1 = the tracker is  */
+                              /* carried as a sum of two floats and the rounding errors of the      */
+                              /* mass-moving operations are fed back (keeps the conservation of      */
+                              /* Lemma 3 over long horizons; one more fp32 stream read and written) */
 } rfast_problem;
 
 /* Raw schedule (value independent).  Round r activates the nodes

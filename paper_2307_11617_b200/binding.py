@@ -45,7 +45,8 @@ class _Problem(C.Structure):
                 ("n_classes", C.c_int32), ("n_hidden", C.c_int32),
                 ("quad_d", C.c_void_p), ("quad_b", C.c_void_p), ("feat", C.c_void_p),
                 ("target", C.c_void_p), ("label", C.c_void_p), ("sp_rowptr", C.c_void_p),
-                ("sp_col", C.c_void_p), ("sp_val", C.c_void_p), ("x0", C.c_void_p)]
+                ("sp_col", C.c_void_p), ("sp_val", C.c_void_p), ("x0", C.c_void_p),
+                ("compensated", C.c_int32)]
 
 
 class _Schedule(C.Structure):
@@ -108,6 +109,7 @@ def _problem(wl, keep):
     P.G_R, P.G_C = _graph(wl.G_R, keep), _graph(wl.G_C, keep)
     P.model = MODEL_IDS[wl.model] if isinstance(wl.model, str) else int(wl.model)
     P.batch, P.rows = int(wl.batch), int(wl.rows)
+    P.compensated = 1 if getattr(wl, "compensated", False) else 0
     dims = getattr(wl, "dims", {}) or {}
     P.n_features = int(dims.get("n_features", 0))
     P.n_classes = int(dims.get("n_classes", 0))

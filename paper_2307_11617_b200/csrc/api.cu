@@ -32,7 +32,8 @@ struct rfast_ctx {
     float alpha = 0, l2 = 0;
     HostGraph R, Cg;
     // device state
-    float *x = nullptr, *z = nullptr, *gbuf = nullptr, *x0 = nullptr;
+    float *x = nullptr, *z = nullptr, *zc = nullptr, *gbuf = nullptr, *x0 = nullptr;
+    bool compensated = false;
     float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
     int* label = nullptr;
     int64_t* sp_ptr = nullptr;
@@ -109,10 +110,10 @@ void free_schedule(rfast_ctx* c) {
     c->has_sched = false;
 }
 
-ModelTraffic traffic_of(int model) {
+ModelTraffic traffic_of(int model, bool compensated) {
     ModelTraffic mt;
     mt.elementwise = (model == RFAST_MODEL_QUAD_DIAG);
-    mt.data_streams = mt.elementwise ? 2 : 0;
+    mt.data_streams = (mt.elementwise ? 2 : 0) + (compensated ? 2 : 0);
     return mt;
 }
 
@@ -208,6 +209,7 @@ int reset_state(rfast_ctx* ctx) {
     if (ctx->x0) CK(cudaMemcpyAsync(ctx->x, ctx->x0, plane, cudaMemcpyDeviceToDevice, ctx->stream));
     else CK(cudaMemsetAsync(ctx->x, 0, plane, ctx->stream));
     const int n4 = (int)(ctx->stride / 4);
+    if (ctx->zc) CK(cudaMemsetAsync(ctx->zc, 0, plane, ctx->stream));
     if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
         k_quad_grad<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
             ctx->x, ctx->quad_d, ctx->quad_b, ctx->z, ctx->stride, n4);
@@ -241,7 +243,7 @@ void rfast_destroy(rfast_ctx* c) {
     cudaStreamSynchronize(c->stream);
     free_schedule(c);
     if (c->mlp) mlp_plan_destroy(c->mlp);
-    void* ptrs[] = {c->x, c->z, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
+    void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
                     c->sp_ptr, c->sp_col, c->sp_val, c->xb};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete c;
@@ -264,6 +266,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
     ctx->n = prob->n; ctx->root = prob->root; ctx->p = prob->p; ctx->alpha = prob->alpha; ctx->l2 = prob->l2;
     ctx->model = prob->model; ctx->batch = prob->batch; ctx->rows = prob->rows;
     ctx->F = prob->n_features; ctx->C = prob->n_classes; ctx->H = prob->n_hidden;
+    ctx->compensated = prob->compensated != 0;
     ctx->stride = (prob->p + 31) / 32 * 32;
     if (ctx->stride / 4 > 0x7fffffff) return set_err(ctx, RFAST_EINVAL, "p too large");
     if ((rc = build_host_graph(prob->G_R, ctx->n, true, ctx->R, err)) != RFAST_OK) return set_err(ctx, rc, "G_R: " + err);
@@ -273,6 +276,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
     const size_t plane = (size_t)ctx->n * ctx->stride;
     CK(dev_alloc(ctx, &ctx->x, plane));
     CK(dev_alloc(ctx, &ctx->z, plane));
+    if (ctx->compensated) CK(dev_alloc(ctx, &ctx->zc, plane));
     if (prob->x0) {
         CK(dev_alloc(ctx, &ctx->x0, plane));
         if ((rc = upload_rows(ctx, ctx->x0, prob->x0, ctx->n)) != RFAST_OK) return rc;
@@ -348,7 +352,7 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     CK(cudaStreamSynchronize(ctx->stream));
     Compiled comp;
     std::string err;
-    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model), comp, err);
+    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated), comp, err);
     if (rc != RFAST_OK) return set_err(ctx, rc, err);
     free_schedule(ctx);
     ctx->comp = std::move(comp);
@@ -410,7 +414,7 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
     a.mix_slot = ctx->d_mix_slot; a.mix_w = ctx->d_mix_w;
     a.news_new = ctx->d_news_new; a.news_prev = ctx->d_news_prev;
     a.out_cur = ctx->d_out_cur; a.out_new = ctx->d_out_new; a.out_a = ctx->d_out_a;
-    a.x = ctx->x; a.z = ctx->z; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
+    a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
     a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
     const bool big = a.n4 >= kThreads * 4;
     for (int r = ctx->round; r < ctx->round + rounds; ++r) {
@@ -418,8 +422,9 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         if (nev == 0) continue;
         a.ev = ctx->d_ev + c.act_ptr[r];
         if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
-            if (big) k_fused_quad<2><<<tile_grid(a.n4, 2, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
-            else k_fused_quad<1><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
+            if (ctx->compensated) k_fused_quad<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
+            else if (big) k_fused_quad<2, false><<<tile_grid(a.n4, 2, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
+            else k_fused_quad<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             ctx->launches += 1;
         } else {
             if (ctx->model == RFAST_MODEL_MLP) k_mix<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb);
@@ -427,7 +432,8 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
             ctx->launches += 1;
             int rc = launch_gradients(ctx, a.ev, nev);
             if (rc != RFAST_OK) return rc;
-            k_track<1><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
+            if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
+            else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
             ctx->launches += 1;
         }
     }
@@ -563,7 +569,7 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32
     if ((rc = build_host_graph(prob->G_C, prob->n, false, C, err)) != RFAST_OK) return done(rc);
     if ((rc = check_roots(R, C, prob->root, err)) != RFAST_OK) return done(rc);
     Compiled c;
-    if ((rc = compile_schedule(R, C, s, prob->batch, prob->rows, traffic_of(prob->model), c, err)) != RFAST_OK) return done(rc);
+    if ((rc = compile_schedule(R, C, s, prob->batch, prob->rows, traffic_of(prob->model, prob->compensated != 0), c, err)) != RFAST_OK) return done(rc);
     if (used_tau_v) std::copy(c.used_tau_v.begin(), c.used_tau_v.end(), used_tau_v);
     if (used_tau_rho) std::copy(c.used_tau_rho.begin(), c.used_tau_rho.end(), used_tau_rho);
     if (v_ver)

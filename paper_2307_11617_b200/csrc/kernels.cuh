@@ -21,6 +21,7 @@ struct RoundArgs {
     const int*    news_new;  const int*   news_prev;
     const int*    out_cur;   const int*   out_new;   const float* out_a;
     float* x;  float* z;         // [n][stride]
+    float* zc;                   // [n][stride] low-order part of the tracker (compensated mode), else null
     float* vbuf;                 // [v rows][stride]   published v versions
     float* rbuf;                 // [rho rows][stride] running-sum versions
     int64_t stride;              // floats per row
@@ -47,7 +48,159 @@ __device__ __forceinline__ float4 f4_scale(float a, float4 x) {
     return make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
 }
 
+
+// Error-free addition (Knuth): s + err == a + b exactly.
+__device__ __forceinline__ void two_sum(float a, float b, float& s, float& err) {
+    s = __fadd_rn(a, b);
+    const float bb = __fsub_rn(s, a);
+    err = __fadd_rn(__fsub_rn(a, __fsub_rn(s, bb)), __fsub_rn(b, bb));
+}
+__device__ __forceinline__ float& comp(float4& v, int c) { return reinterpret_cast<float*>(&v)[c]; }
+__device__ __forceinline__ float comp(const float4& v, int c) { return reinterpret_cast<const float*>(&v)[c]; }
+
 constexpr int kThreads = 256;
+
+
+// ---------------------------------------------------------------------------------------------
+// S2b + S2c on U float4 per thread, shared by the fused and the split kernels.
+//   z^ = z + sum over in-edges with news (rho[tau'] - rho[tau_prev]) + g_new - g_old
+//   z' = a_ii z^ ;  rho'_ji = rho_ji + a_ji z^  for every out-edge
+// COMP = false: plain fp32, in the order written above.
+// COMP = true: the tracker is carried as an unevaluated sum of two floats (z + zc) and every
+// rounding error of the mass-moving operations (the additions into z^, the products with the
+// weights, the additions into the running sums) is captured with error-free transformations
+// and kept in the node's own low-order part, so that the tracked mass of Lemma 3 is conserved
+// to second order instead of drifting with every fp32 rounding.  The running sums stay fp32.
+// ---------------------------------------------------------------------------------------------
+template <int U, bool COMP>
+__device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc& e, int base, float* zr,
+                                               const float4 (&zv)[U], const float4 (&gn)[U],
+                                               const float4 (&go)[U]) {
+    if (!COMP) {
+        float4 zh[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) zh[u] = zv[u];
+        for (int m = 0; m < e.news_cnt; ++m) {                          // ascending sender id
+            const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
+            const int prev = a.news_prev[e.news_beg + m];
+            const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i4 = base + u * kThreads;
+                if (i4 < a.n4) {
+                    float4 dl = ld_stream(nr, i4);
+                    if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
+                    zh[u] = f4_add(zh[u], dl);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            zh[u] = f4_sub(f4_add(zh[u], gn[u]), go[u]);
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) st_stream(zr, i4, f4_scale(e.a_self, zh[u]));   // S2c keep
+        }
+        for (int m = 0; m < e.out_cnt; ++m) {                           // S2c accumulate
+            const int cur = a.out_cur[e.out_beg + m];
+            const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
+            float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
+            const float aw = a.out_a[e.out_beg + m];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i4 = base + u * kThreads;
+                if (i4 < a.n4) {
+                    float4 r = f4_scale(aw, zh[u]);
+                    if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
+                    st_stream(wr, i4, r);
+                }
+            }
+        }
+    } else {
+        float* cr_ = a.zc + (zr - a.z);
+        float4 hi[U], lo[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            hi[u] = zv[u];
+            lo[u] = make_float4(0, 0, 0, 0);
+            if (i4 < a.n4) lo[u] = ld_stream(cr_, i4);
+        }
+        for (int m = 0; m < e.news_cnt; ++m) {
+            const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
+            const int prev = a.news_prev[e.news_beg + m];
+            const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i4 = base + u * kThreads;
+                if (i4 < a.n4) {
+                    const float4 nv = ld_stream(nr, i4);
+                    const float4 pv = prev >= 0 ? ld_stream(pr, i4) : make_float4(0, 0, 0, 0);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float d, de, s, se;
+                        two_sum(comp(nv, c), -comp(pv, c), d, de);
+                        two_sum(comp(hi[u], c), d, s, se);
+                        comp(hi[u], c) = s;
+                        comp(lo[u], c) += se + de;
+                    }
+                }
+            }
+        }
+        float4 zh_hi[U], zh_lo[U], k_hi[U], k_lo[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float s, se, t, te;
+                two_sum(comp(hi[u], c), comp(gn[u], c), s, se);
+                two_sum(s, -comp(go[u], c), t, te);
+                const float l = comp(lo[u], c) + (se + te);
+                float zh, zl;
+                two_sum(t, l, zh, zl);
+                comp(zh_hi[u], c) = zh;
+                comp(zh_lo[u], c) = zl;
+                const float kh = __fmul_rn(e.a_self, zh);
+                comp(k_hi[u], c) = kh;
+                comp(k_lo[u], c) = __fmaf_rn(e.a_self, zh, -kh) + e.a_self * zl;
+            }
+        }
+        for (int m = 0; m < e.out_cnt; ++m) {
+            const int cur = a.out_cur[e.out_beg + m];
+            const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
+            float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
+            const float aw = a.out_a[e.out_beg + m];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i4 = base + u * kThreads;
+                if (i4 < a.n4) {
+                    const float4 cv = cur >= 0 ? ld_stream(cr, i4) : make_float4(0, 0, 0, 0);
+                    float4 r;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float inc = __fmul_rn(aw, comp(zh_hi[u], c));
+                        const float ierr = __fmaf_rn(aw, comp(zh_hi[u], c), -inc) + aw * comp(zh_lo[u], c);
+                        float s, se;
+                        two_sum(comp(cv, c), inc, s, se);
+                        comp(r, c) = s;
+                        comp(k_lo[u], c) += se + ierr;       // what did not fit stays with the sender
+                    }
+                    st_stream(wr, i4, r);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i4 = base + u * kThreads;
+            if (i4 < a.n4) {
+                float4 zf, cf;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) two_sum(comp(k_hi[u], c), comp(k_lo[u], c), comp(zf, c), comp(cf, c));
+                st_stream(zr, i4, zf);
+                st_stream(cr_, i4, cf);
+            }
+        }
+    }
+}
 
 // ---------------------------------------------------------------------------------------------
 // Fused activation for the element-wise objective f_i(x) = 0.5 || d_i .* (x - b_i) ||^2:
@@ -58,7 +211,7 @@ constexpr int kThreads = 256;
 // last consumed, kept alive instead of copied).  One HBM pass per activation.
 // grid = (tiles, events of the round)
 // ---------------------------------------------------------------------------------------------
-template <int U>
+template <int U, bool COMP>
 __global__ void __launch_bounds__(kThreads)
 k_fused_quad(RoundArgs a, const float* __restrict__ qd, const float* __restrict__ qb) {
     const EvDesc e = a.ev[blockIdx.y];
@@ -104,53 +257,18 @@ k_fused_quad(RoundArgs a, const float* __restrict__ qd, const float* __restrict_
             if (i4 < a.n4) acc[u] = f4_axpy(w, ld_stream(nr, i4), acc[u]);
         }
     }
-    float4 zh[U];
+    float4 gn[U], go[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const int i4 = base + u * kThreads;
         if (i4 < a.n4) st_stream(xr, i4, acc[u]);
-        zh[u] = zv[u];
-    }
-    for (int m = 0; m < e.news_cnt; ++m) {                          // S2b, ascending sender id
-        const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
-        const int prev = a.news_prev[e.news_beg + m];
-        const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i4 = base + u * kThreads;
-            if (i4 < a.n4) {
-                float4 dl = ld_stream(nr, i4);
-                if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
-                zh[u] = f4_add(zh[u], dl);
-            }
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
         const float4 d2 = make_float4(dv[u].x * dv[u].x, dv[u].y * dv[u].y, dv[u].z * dv[u].z, dv[u].w * dv[u].w);
-        const float4 gn = make_float4(d2.x * (acc[u].x - bv[u].x), d2.y * (acc[u].y - bv[u].y),
-                                      d2.z * (acc[u].z - bv[u].z), d2.w * (acc[u].w - bv[u].w));
-        const float4 go = make_float4(d2.x * (xv[u].x - bv[u].x), d2.y * (xv[u].y - bv[u].y),
-                                      d2.z * (xv[u].z - bv[u].z), d2.w * (xv[u].w - bv[u].w));
-        zh[u] = f4_sub(f4_add(zh[u], gn), go);
-        const int i4 = base + u * kThreads;
-        if (i4 < a.n4) st_stream(zr, i4, f4_scale(e.a_self, zh[u]));       // S2c keep
+        gn[u] = make_float4(d2.x * (acc[u].x - bv[u].x), d2.y * (acc[u].y - bv[u].y),
+                            d2.z * (acc[u].z - bv[u].z), d2.w * (acc[u].w - bv[u].w));
+        go[u] = make_float4(d2.x * (xv[u].x - bv[u].x), d2.y * (xv[u].y - bv[u].y),
+                            d2.z * (xv[u].z - bv[u].z), d2.w * (xv[u].w - bv[u].w));
     }
-    for (int m = 0; m < e.out_cnt; ++m) {                           // S2c accumulate
-        const int cur = a.out_cur[e.out_beg + m];
-        const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
-        float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
-        const float aw = a.out_a[e.out_beg + m];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i4 = base + u * kThreads;
-            if (i4 < a.n4) {
-                float4 r = f4_scale(aw, zh[u]);
-                if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
-                st_stream(wr, i4, r);
-            }
-        }
-    }
+    track_and_push<U, COMP>(a, e, base, zr, zv, gn, go);
 }
 
 // z_i^0 = grad f_i(x_i^0) for the element-wise objective.  grid = (tiles, n)
@@ -225,7 +343,7 @@ k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
 // S2b + S2c (+ S4 by row id) with the gradients taken from the two gradient buffers:
 // g_old = gbuf[par][node], g_new = gbuf[par^1][node].  grid = (tiles, events)
 // ---------------------------------------------------------------------------------------------
-template <int U>
+template <int U, bool COMP>
 __global__ void __launch_bounds__(kThreads)
 k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
     const EvDesc e = a.ev[blockIdx.y];
@@ -241,41 +359,7 @@ k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
         zh[u] = gnv[u] = gov[u] = make_float4(0, 0, 0, 0);
         if (i4 < a.n4) { zh[u] = ld_stream(zr, i4); gnv[u] = ld_stream(gn, i4); gov[u] = ld_stream(go, i4); }
     }
-    for (int m = 0; m < e.news_cnt; ++m) {
-        const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
-        const int prev = a.news_prev[e.news_beg + m];
-        const float* pr = a.rbuf + (int64_t)(prev < 0 ? 0 : prev) * a.stride;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i4 = base + u * kThreads;
-            if (i4 < a.n4) {
-                float4 dl = ld_stream(nr, i4);
-                if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
-                zh[u] = f4_add(zh[u], dl);
-            }
-        }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        zh[u] = f4_sub(f4_add(zh[u], gnv[u]), gov[u]);
-        const int i4 = base + u * kThreads;
-        if (i4 < a.n4) st_stream(zr, i4, f4_scale(e.a_self, zh[u]));
-    }
-    for (int m = 0; m < e.out_cnt; ++m) {
-        const int cur = a.out_cur[e.out_beg + m];
-        const float* cr = a.rbuf + (int64_t)(cur < 0 ? 0 : cur) * a.stride;
-        float* wr = a.rbuf + (int64_t)a.out_new[e.out_beg + m] * a.stride;
-        const float aw = a.out_a[e.out_beg + m];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int i4 = base + u * kThreads;
-            if (i4 < a.n4) {
-                float4 r = f4_scale(aw, zh[u]);
-                if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
-                st_stream(wr, i4, r);
-            }
-        }
-    }
+    track_and_push<U, COMP>(a, e, base, zr, zh, gnv, gov);
 }
 
 // ---------------------------------------------------------------------------------------------

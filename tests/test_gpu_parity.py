@@ -100,6 +100,27 @@ def test_parity_round_by_round_and_reset(rfast_lib):
         assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
 
 
+@pytest.mark.parametrize("name,ov", [
+    ("quad_tree64", dict(n=32, p=4099, K=80, drop=0.4)),
+    ("quad_tree64", dict(n=16, p=70_001, K=30)),
+    ("ls_ring4", {}),
+    ("logistic_tree1024", dict(n=96, p=5000, rows=8, K=60, batch=4, nnz=50)),
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=150, batch=8, compensated=False)),
+], ids=["quad", "quad tiles", "ls", "logistic", "softmax plain"])
+def test_parity_in_the_other_tracker_arithmetic(rfast_lib, name, ov):
+    """Every objective in the tracker arithmetic its configuration does not use by default
+    (compensated two-float tracker <-> plain fp32)."""
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=2, **ov)
+    if name != "softmax_exp16":
+        wl.compensated = True
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+
+
 def test_conservation_on_the_device_state(rfast_lib):
     """Lemma 3 on what the GPU holds: trackers plus undelivered mass equal the sum of the
     latest gradients, up to fp32 rounding of the running sums."""

@@ -48,6 +48,7 @@ class Workload:
     x0: np.ndarray | None = None    # float32 [n, p] or None (zeros)
     schedule: Schedule | None = None
     meta: dict = field(default_factory=dict)
+    compensated: bool = False       # ask the engine for compensated tracker arithmetic (long horizons)
 
     def __post_init__(self):
         # scalars are handed to every consumer as the fp32-representable value
@@ -132,7 +133,8 @@ def _softmax_exp(seed, ov):
     return Workload("softmax_exp16", n, p, 0, alpha, G_R, G_C, MODEL_SOFTMAX, B, 1e-4, rows,
                     dims={"n_features": F, "n_classes": C}, data={"feat": feat, "label": label},
                     schedule=sch, meta={"K": K, "drop": drop, "max_delay": max_delay,
-                                        "straggler": straggler})
+                                        "straggler": straggler},
+                    compensated=ov.get("compensated", True))
 
 
 # -- config 3: n=64 random trees, MLP F-H-C ReLU, lognormal compute times -----------------------
