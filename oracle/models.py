@@ -101,8 +101,10 @@ class Softmax:
 
 class MLP:
     """One hidden ReLU layer, softmax cross-entropy.  With round_inputs=True the operands of
-    every matrix product (weights, activations, deltas) are first rounded to bf16; sums,
-    biases, ReLU, softmax and the products' accumulation stay in full precision."""
+    the two GEMM-shaped products -- the hidden pre-activations A W1^T and the weight gradient
+    dpre^T A -- are first rounded to bf16 ("fp32 state / bf16 GEMM inputs").  The products
+    with the n_classes-wide output layer are a few columns thin, not GEMM work, and stay in
+    full precision, as do sums, biases, ReLU, softmax and all accumulation."""
 
     def __init__(self, feat, label, n_hidden, n_classes, l2=0.0, round_inputs=True):
         self.A, self.lab = feat, label
@@ -124,7 +126,7 @@ class MLP:
         W1, b1, W2, b2 = self._split(x)
         pre = A @ q(W1).T + b1
         h = np.maximum(pre, 0.0)
-        logits = q(h) @ q(W2).T + b2
+        logits = h @ W2.T + b2
         return A, lab, pre, h, logits
 
     def loss(self, i, x, idx):
@@ -139,9 +141,9 @@ class MLP:
         P, _ = _softmax_rows(logits)
         P[np.arange(len(lab)), lab] -= 1.0
         dlog = P / len(lab)                       # d loss / d logits          [B, C]
-        gW2 = q(dlog).T @ q(h)                    #                            [C, H]
+        gW2 = dlog.T @ h                          #                            [C, H]
         gb2 = dlog.sum(axis=0)
-        dh = q(dlog) @ q(W2)                      #                            [B, H]
+        dh = dlog @ W2                            #                            [B, H]
         dpre = dh * (pre > 0.0)
         gW1 = q(dpre).T @ A                       # A already rounded          [H, F]
         gb1 = dpre.sum(axis=0)

@@ -17,7 +17,9 @@ namespace rfast {
 // MLP gradient (tensor-core path), defined in grad_mlp.cu
 struct MlpPlan;
 int  mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride, int max_events,
-                     const float* d_feat, MlpPlan** out, size_t* dev_bytes, std::string& err);
+                     const float* d_feat, const __nv_bfloat16* xb, cudaStream_t st, MlpPlan** out,
+                     size_t* dev_bytes, std::string& err);
+int  mlp_plan_status(MlpPlan* plan, cudaStream_t st);
 void mlp_plan_destroy(MlpPlan* plan);
 int  mlp_grad_launch(MlpPlan* plan, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
                      int n_events, cudaStream_t st, int64_t* launches, std::string& err);
@@ -204,6 +206,16 @@ int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
     return RFAST_OK;
 }
 
+// after a synchronisation: did a bounded device-side wait run out?
+int check_device_status(rfast_ctx* ctx) {
+    if (ctx->mlp) {
+        const int st = mlp_plan_status(ctx->mlp, ctx->stream);
+        if (st < 0) return set_err(ctx, RFAST_ECUDA, "reading the device status word failed");
+        if (st > 0) return set_err(ctx, RFAST_ETIMEOUT, "a bounded wait in the MLP gradient kernels ran out (role " + std::to_string(st) + ")");
+    }
+    return RFAST_OK;
+}
+
 int reset_state(rfast_ctx* ctx) {
     const size_t plane = (size_t)ctx->n * ctx->stride * sizeof(float);
     if (ctx->x0) CK(cudaMemcpyAsync(ctx->x, ctx->x0, plane, cudaMemcpyDeviceToDevice, ctx->stream));
@@ -333,7 +345,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
         CK(cudaMemsetAsync(ctx->xb, 0, plane * sizeof(__nv_bfloat16), ctx->stream));
         size_t mb = 0;
         rc = mlp_plan_create(ctx->n, ctx->rows, ctx->F, ctx->H, ctx->C, ctx->batch, ctx->stride, ctx->n,
-                             ctx->feat, &ctx->mlp, &mb, err);
+                             ctx->feat, ctx->xb, ctx->stream, &ctx->mlp, &mb, err);
         if (rc != RFAST_OK) return set_err(ctx, rc, err);
         ctx->dev_bytes += mb;
     }
@@ -439,14 +451,17 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
     }
     CK(cudaGetLastError());
     ctx->round += rounds;
-    if (sync) CK(cudaStreamSynchronize(ctx->stream));
+    if (sync) {
+        CK(cudaStreamSynchronize(ctx->stream));
+        return check_device_status(ctx);
+    }
     return RFAST_OK;
 }
 
 int rfast_sync(rfast_ctx* ctx) {
     if (!ctx) return RFAST_EINVAL;
     CK(cudaStreamSynchronize(ctx->stream));
-    return RFAST_OK;
+    return check_device_status(ctx);
 }
 
 int64_t rfast_query(rfast_ctx* ctx, int what) {
@@ -503,6 +518,10 @@ int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
         cudaFree(tmp); cudaFree(didx);
         return rc;
     };
+    if (which <= RFAST_STATE_RHO_BUF) {
+        int rc = check_device_status(ctx);
+        if (rc != RFAST_OK) return rc;
+    }
     switch (which) {
         case RFAST_STATE_X: return rows_out(ctx->x, n);
         case RFAST_STATE_Y: return rows_out(ctx->z, n);

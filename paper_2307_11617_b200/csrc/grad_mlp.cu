@@ -1,27 +1,571 @@
-// MLP sample gradient (placeholder until the tensor-core path lands).
+// Sample gradient of the one-hidden-layer MLP (softmax cross-entropy), sm_100a.
+//
+// Per activation (batch of B = 64 sampled rows A, parameters W1 [H x F], b1, W2 [C x H], b2):
+//   pre = q(A) q(W1)^T + b1,  h = relu(pre),  logits = h W2^T + b2,  dlog = (softmax - onehot) / B
+//   gW2 = dlog^T h,  gb2 = sum_k dlog,  dh = dlog W2,  dpre = dh .* (pre > 0)
+//   gW1 = q(dpre)^T q(A),  gb1 = sum_k dpre                      (q = round to bf16)
+// The two products that carry the work, pre (H x B x F) and gW1 (H x F x B), are dense
+// contractions and run on the 5th-generation tensor cores: operands are brought into shared
+// memory by TMA (128-byte swizzle), tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) accumulates in
+// tensor memory, and the epilogue reads the accumulator back with tcgen05.ld.  Both are
+// computed transposed (M = a 128-row slab of hidden units) so that M is the tensor core's
+// native 128.  The C <= 16 wide products in between are far too thin for an MMA tile and run
+// in fp32 on the CUDA cores of one CTA per activation.
+//
+// Every wait on an mbarrier is bounded: when it runs out the CTA records a code in a status
+// word, leaves its loops, frees its tensor memory and returns.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstdio>
 #include <string>
 
 #include "rfast_internal.h"
 
 namespace rfast {
 
-struct MlpPlan { int unused; };
+namespace {
 
-int mlp_plan_create(int, int, int, int, int, int, int64_t, int, const float*, MlpPlan** out,
+constexpr int kBatch = 64;          // rows per minibatch the tensor-core path is built for
+constexpr int kMTile = 128;         // hidden units per CTA (UMMA M)
+constexpr int kKBlock = 64;         // bf16 elements per 128-byte swizzle row
+constexpr int kStagesFwd = 4;
+constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait; false when the limit ran out (the caller records it and bails out).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+        uint64_t now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (it == 0) t0 = now;
+        else if (now - t0 > kWaitLimitNs) return false;
+    }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {     // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {         // whole warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate; one thread issues.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The barrier gets one arrival when all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory operand descriptor: K-major tile of rows x 64 bf16 as written by TMA with the
+// 128-byte swizzle (row pitch 128 B, groups of 8 rows = 1024 B), tile base 1024-byte aligned.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);        // start address
+    d |= (uint64_t)1 << 16;                          // leading-dimension byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, shape M x N.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+enum { kErrNone = 0, kErrProducer = 1, kErrMma = 2, kErrEpilogue = 3 };
+
+}  // namespace
+
+struct MlpPlan;
+void mlp_plan_destroy(MlpPlan* p);
+
+struct MlpPlan {
+    int n = 0, rows = 0, F = 0, H = 0, C = 0, B = 0, Fp = 0, NT = 0, maxev = 0;
+    int64_t stride = 0;
+    __nv_bfloat16 *featb = nullptr, *Ab = nullptr, *AbT = nullptr, *dpqT = nullptr;
+    float* hf = nullptr;               // [ev][B][H] hidden activations
+    int* status = nullptr;
+    CUtensorMap tmW1, tmA, tmD, tmAT;
+};
+
+// ---------------------------------------------------------------------------------------------
+// kernels
+// ---------------------------------------------------------------------------------------------
+
+// fp32 -> bf16 (nearest even), flat
+__global__ void k_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t count) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// Sampled rows of one activation, as the two GEMMs want them:
+//   Ab  [ev][B][Fp]  row k = features of sample k, zero beyond F (K-major operand of pre)
+//   AbT [ev][F][B]   the transpose                      (K-major operand of gW1, K = batch)
+__global__ void __launch_bounds__(256)
+k_mlp_gather(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx,
+             const __nv_bfloat16* __restrict__ featb, __nv_bfloat16* __restrict__ Ab,
+             __nv_bfloat16* __restrict__ AbT, int rows, int F, int Fp) {
+    const EvDesc e = evs[blockIdx.x];
+    const int* idx = batch_idx + (int64_t)e.sample * kBatch;
+    const __nv_bfloat16* shard = featb + (int64_t)e.node * rows * F;
+    __nv_bfloat16* ab = Ab + (int64_t)blockIdx.x * kBatch * Fp;
+    __nv_bfloat16* abt = AbT + (int64_t)blockIdx.x * F * kBatch;
+    for (int q = threadIdx.x; q < kBatch * Fp; q += 256) {
+        const int k = q / Fp, f = q % Fp;
+        ab[q] = f < F ? shard[(int64_t)idx[k] * F + f] : __float2bfloat16_rn(0.f);
+    }
+    for (int q = threadIdx.x; q < F * kBatch; q += 256) {
+        const int f = q / kBatch, k = q % kBatch;
+        abt[q] = shard[(int64_t)idx[k] * F + f];
+    }
+}
+
+// pre^T slab = W1[h0 .. h0+128) x A^T, then h = relu(pre + b1), stored in hf[ev][k][j].
+// grid = (H / 128, events)
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmA,
+          const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
+          float* __restrict__ hf, int F, int H, int kblocks, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr int kABytes = kMTile * kKBlock * 2, kBBytes = kBatch * kKBlock * 2;
+    uint8_t* sA = smem;                                   // [stages][128][64] bf16
+    uint8_t* sB = smem + kStagesFwd * kABytes;            // [stages][64][64] bf16
+    __shared__ uint64_t full[kStagesFwd], empty[kStagesFwd], acc_full;
+    __shared__ uint32_t tmem_base;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ev = blockIdx.y, h0 = blockIdx.x * kMTile;
+    const EvDesc e = evs[ev];
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStagesFwd; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(&acc_full, 1);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&tmem_base, 64);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tacc = tmem_base;
+
+    if (warp == 0 && lane == 0) {                          // ---- TMA producer
+        int issued = 0;
+        bool ok = true;
+        for (int kb = 0; kb < kblocks && ok; ++kb) {
+            const int s = kb % kStagesFwd;
+            if (kb >= kStagesFwd) ok = mbar_wait(&empty[s], ((kb / kStagesFwd) - 1) & 1);
+            if (!ok) break;
+            mbar_expect_tx(&full[s], kABytes + kBBytes);
+            tma_load_3d(sA + s * kABytes, &tmW1, &full[s], kb * kKBlock, h0, e.node);
+            tma_load_2d(sB + s * kBBytes, &tmA, &full[s], kb * kKBlock, ev * kBatch);
+            ++issued;
+        }
+        if (!ok) {
+            atomicExch(status, kErrProducer);
+            // let the copies already issued land before the CTA's shared memory goes away
+            for (int q = (issued > kStagesFwd ? issued - kStagesFwd : 0); q < issued; ++q)
+                mbar_wait(&full[q % kStagesFwd], (q / kStagesFwd) & 1);
+        }
+    } else if (warp == 1 && lane == 0) {                   // ---- MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(kMTile, kBatch);
+        bool ok = true;
+        for (int kb = 0; kb < kblocks; ++kb) {
+            const int s = kb % kStagesFwd;
+            ok = mbar_wait(&full[s], (kb / kStagesFwd) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t ad = umma_desc_sw128(smem_u32(sA + s * kABytes));
+            const uint64_t bd = umma_desc_sw128(smem_u32(sB + s * kBBytes));
+#pragma unroll
+            for (int k = 0; k < kKBlock / 16; ++k)          // 16 bf16 = 32 bytes per step inside the swizzle row
+                umma_bf16(tacc, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, (kb | k) ? 1u : 0u);
+            umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(&acc_full);
+        else { atomicExch(status, kErrMma); mbar_arrive(&acc_full); }
+    } else if (warp >= 2) {                                // ---- epilogue: TMEM -> relu -> hf
+        const bool ok = mbar_wait(&acc_full, 0);
+        tc_fence_after();
+        if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
+        else if (atomicAdd(status, 0) == kErrNone) {
+            const int q = warp & 3;                         // this warp owns tensor-memory lanes 32q .. 32q+31
+            const int j = h0 + q * 32 + lane;               // hidden unit
+            const float b1 = x[(int64_t)e.node * stride + (int64_t)H * F + j];
+            float* out = hf + (int64_t)ev * kBatch * H + j;
+#pragma unroll
+            for (int c0 = 0; c0 < kBatch; c0 += 16) {
+                float v[16];
+                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    out[(int64_t)(c0 + i) * H] = fmaxf(v[i] + b1, 0.f);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 64); }
+}
+
+// Everything between the two big products, one CTA per activation (CUDA cores):
+// logits, softmax, dlog; gW2, gb2, dh, dpre, gb1; q(dpre)^T for the second product.
+// grid = events, 512 threads; dynamic shared memory: 2 * B * C floats
+__global__ void __launch_bounds__(512)
+k_mlp_mid(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
+          const float* __restrict__ x, int64_t stride,
+          const float* __restrict__ hf, __nv_bfloat16* __restrict__ dpqT,
+          float* __restrict__ gbuf, int64_t gplane, int rows, int F, int H, int C, float l2) {
+    extern __shared__ float sm[];
+    float* logit = sm;                     // [B][C]
+    float* dl = sm + kBatch * C;           // [B][C] dlog
+    const int ev = blockIdx.x;
+    const EvDesc e = evs[ev];
+    const int64_t row = (int64_t)e.node * stride;
+    const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
+    const float* h = hf + (int64_t)ev * kBatch * H;
+    const float* W2 = x + row + oW2;
+    float* g = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    for (int k = warp; k < kBatch; k += nwarp)
+        for (int c = 0; c < C; ++c) {
+            float s = 0.f;
+            for (int j = lane; j < H; j += 32)
+                s = fmaf(h[(int64_t)k * H + j], W2[(int64_t)c * H + j], s);
+            s = warp_sum(s);
+            if (lane == 0) logit[k * C + c] = s + x[row + ob2 + c];
+        }
+    __syncthreads();
+    if (threadIdx.x < kBatch) {
+        const int k = threadIdx.x;
+        const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
+        float m = logit[k * C];
+        for (int c = 1; c < C; ++c) m = fmaxf(m, logit[k * C + c]);
+        float den = 0.f;
+        for (int c = 0; c < C; ++c) den += expf(logit[k * C + c] - m);
+        for (int c = 0; c < C; ++c) {
+            const float d = (expf(logit[k * C + c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)kBatch;
+            dl[k * C + c] = d;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < C) {
+        float s = 0.f;
+        for (int k = 0; k < kBatch; ++k) s += dl[k * C + threadIdx.x];
+        g[ob2 + threadIdx.x] = s + l2 * x[row + ob2 + threadIdx.x];
+    }
+    for (int j = threadIdx.x; j < H; j += blockDim.x) {
+        float w2[16], gw2[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
+        float gb1 = 0.f;
+        __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch;
+        for (int k0 = 0; k0 < kBatch; k0 += 8) {
+            __align__(16) __nv_bfloat16 pack[8];
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const int k = k0 + kk;
+                const float hv = h[(int64_t)k * H + j];
+                float dh = 0.f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) if (c < C) dh = fmaf(dl[k * C + c], w2[c], dh);
+                const float dp = hv > 0.f ? dh : 0.f;
+                gb1 += dp;
+                pack[kk] = __float2bfloat16_rn(dp);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) if (c < C) gw2[c] = fmaf(dl[k * C + c], hv, gw2[c]);
+            }
+            *reinterpret_cast<uint4*>(drow + k0) = *reinterpret_cast<const uint4*>(pack);
+        }
+        g[(int64_t)H * F + j] = gb1 + l2 * x[row + (int64_t)H * F + j];
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+            if (c < C) g[oW2 + (int64_t)c * H + j] = gw2[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
+    }
+}
+
+// gW1 slab [h0 .. h0+128) x F = q(dpre)^T (K = batch) x A, N tiles of NT features, accumulators
+// double-buffered in tensor memory.  grid = (H / 128, events)
+constexpr int kStagesB = 3;
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmAT,
+          const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
+          float* __restrict__ gbuf, int64_t gplane, int F, int H, int NT, float l2, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr int kABytes = kMTile * kKBlock * 2;          // q(dpre)^T slab, loaded once
+    constexpr int kBMax = 128 * kKBlock * 2;               // room for one N tile of A^T
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kABytes;                          // [stages][NT][64] bf16, stage pitch kBMax
+    __shared__ uint64_t a_full, b_full[kStagesB], b_empty[kStagesB], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ev = blockIdx.y, h0 = blockIdx.x * kMTile;
+    const EvDesc e = evs[ev];
+    const int ntiles = F / NT;
+    if (threadIdx.x == 0) {
+        mbar_init(&a_full, 1);
+        for (int s = 0; s < kStagesB; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&tmem_base, 256);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tacc = tmem_base;
+
+    if (warp == 0 && lane == 0) {                          // ---- TMA producer
+        bool ok = true;
+        mbar_expect_tx(&a_full, kABytes);
+        tma_load_2d(sA, &tmD, &a_full, 0, ev * H + h0);
+        for (int t = 0; t < ntiles; ++t) {
+            const int s = t % kStagesB;
+            if (t >= kStagesB) ok = mbar_wait(&b_empty[s], ((t / kStagesB) - 1) & 1);
+            if (!ok) break;
+            mbar_expect_tx(&b_full[s], NT * kKBlock * 2);
+            tma_load_2d(sB + s * kBMax, &tmAT, &b_full[s], 0, ev * F + t * NT);
+        }
+        if (!ok) atomicExch(status, kErrProducer);
+    } else if (warp == 1 && lane == 0) {                   // ---- MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(kMTile, NT);
+        bool ok = mbar_wait(&a_full, 0);
+        const uint64_t ad = umma_desc_sw128(smem_u32(sA));
+        for (int t = 0; t < ntiles && ok; ++t) {
+            const int s = t % kStagesB, a = t & 1;
+            if (t >= 2) ok = mbar_wait(&acc_empty[a], ((t >> 1) - 1) & 1);
+            if (ok) ok = mbar_wait(&b_full[s], (t / kStagesB) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t bd = umma_desc_sw128(smem_u32(sB + s * kBMax));
+#pragma unroll
+            for (int k = 0; k < kKBlock / 16; ++k)
+                umma_bf16(tacc + a * 128, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, k ? 1u : 0u);
+            umma_commit(&b_empty[s]);
+            umma_commit(&acc_full[a]);
+        }
+        if (!ok) { atomicExch(status, kErrMma); mbar_arrive(&acc_full[0]); mbar_arrive(&acc_full[1]); }
+    } else if (warp >= 2) {                                // ---- epilogue: TMEM -> global
+        const int q = warp & 3;
+        const int j = h0 + q * 32 + lane;
+        const int64_t row = (int64_t)e.node * stride;
+        float* grow = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row + (int64_t)j * F;
+        const float* xrow = x + row + (int64_t)j * F;
+        for (int t = 0; t < ntiles; ++t) {
+            const int a = t & 1;
+            const bool ok = mbar_wait(&acc_full[a], (t >> 1) & 1);
+            tc_fence_after();
+            if (!ok || atomicAdd(status, 0) != kErrNone) { if (!ok && lane == 0) atomicExch(status, kErrEpilogue); break; }
+            for (int c0 = 0; c0 < NT; c0 += 16) {
+                float v[16];
+                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + a * 128 + c0, v);
+                const int f0 = t * NT + c0;
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                    float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                    if (l2 != 0.f) {
+                        const float4 xv = *reinterpret_cast<const float4*>(xrow + f0 + i);
+                        o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
+                    }
+                    *reinterpret_cast<float4*>(grow + f0 + i) = o;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[a]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 256); }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 tensor, innermost dimension first; strides in bytes for dimensions 1.. ; 128-byte swizzle
+bool make_map(CUtensorMap* m, void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+              const uint32_t* box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t d[3], s[2];
+    cuuint32_t b[3], es[3] = {1, 1, 1};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, base, d, s, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 1024;
+constexpr size_t kDw1Smem = kMTile * kKBlock * 2 + kStagesB * (128 * kKBlock * 2) + 1024;
+
+}  // namespace
+
+int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride, int max_events,
+                    const float* d_feat, const __nv_bfloat16* xb, cudaStream_t st, MlpPlan** out,
                     size_t* dev_bytes, std::string& err) {
     *out = nullptr;
     *dev_bytes = 0;
-    err = "MLP objective is not available in this build";
-    return RFAST_EINVAL;
+    if (B != kBatch || H % kMTile != 0 || H <= 0 || F % 16 != 0 || F <= 0 || C < 2 || C > 16) {
+        err = "MLP: the tensor-core path needs batch = 64, n_hidden a multiple of 128, n_features a multiple of 16, 2 <= n_classes <= 16";
+        return RFAST_EINVAL;
+    }
+    MlpPlan* p = new MlpPlan();
+    p->n = n; p->rows = rows; p->F = F; p->H = H; p->C = C; p->B = B; p->stride = stride; p->maxev = max_events;
+    p->Fp = (F + kKBlock - 1) / kKBlock * kKBlock;
+    p->NT = 16;
+    for (int nt = 128; nt >= 16; nt -= 16) if (F % nt == 0) { p->NT = nt; break; }
+    size_t total = 0;
+    auto alloc = [&](__nv_bfloat16** q, size_t cnt) {
+        cudaError_t e = cudaMalloc((void**)q, cnt * sizeof(__nv_bfloat16));
+        if (e == cudaSuccess) total += cnt * sizeof(__nv_bfloat16);
+        return e == cudaSuccess;
+    };
+    const size_t nfeat = (size_t)n * rows * F;
+    bool ok = alloc(&p->featb, nfeat) && alloc(&p->Ab, (size_t)max_events * kBatch * p->Fp) &&
+              alloc(&p->AbT, (size_t)max_events * F * kBatch) &&
+              alloc(&p->dpqT, (size_t)max_events * H * kBatch) &&
+              cudaMalloc((void**)&p->hf, (size_t)max_events * kBatch * H * sizeof(float)) == cudaSuccess &&
+              cudaMalloc((void**)&p->status, sizeof(int)) == cudaSuccess;
+    if (!ok) { mlp_plan_destroy(p); err = "MLP: device allocation failed"; return RFAST_ENOMEM; }
+    cudaMemsetAsync(p->status, 0, sizeof(int), st);
+    k_to_bf16<<<(unsigned)((nfeat + 255) / 256), 256, 0, st>>>(d_feat, p->featb, (int64_t)nfeat);
+    {
+        const uint64_t dW[3] = {(uint64_t)F, (uint64_t)H, (uint64_t)n};
+        const uint64_t sW[2] = {(uint64_t)F * 2, (uint64_t)stride * 2};
+        const uint32_t bW[3] = {kKBlock, kMTile, 1};
+        const uint64_t dA[2] = {(uint64_t)p->Fp, (uint64_t)max_events * kBatch};
+        const uint64_t sA[1] = {(uint64_t)p->Fp * 2};
+        const uint32_t bA[2] = {kKBlock, kBatch};
+        const uint64_t dD[2] = {(uint64_t)kBatch, (uint64_t)max_events * H};
+        const uint64_t sD[1] = {(uint64_t)kBatch * 2};
+        const uint32_t bD[2] = {kKBlock, kMTile};
+        const uint64_t dT[2] = {(uint64_t)kBatch, (uint64_t)max_events * F};
+        const uint32_t bT[2] = {kKBlock, (uint32_t)p->NT};
+        if (!make_map(&p->tmW1, (void*)xb, 3, dW, sW, bW) || !make_map(&p->tmA, p->Ab, 2, dA, sA, bA) ||
+            !make_map(&p->tmD, p->dpqT, 2, dD, sD, bD) || !make_map(&p->tmAT, p->AbT, 2, dT, sD, bT)) {
+            mlp_plan_destroy(p);
+            err = "MLP: cuTensorMapEncodeTiled failed";
+            return RFAST_ECUDA;
+        }
+    }
+    if (cudaFuncSetAttribute(k_mlp_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDw1Smem) != cudaSuccess) {
+        mlp_plan_destroy(p);
+        err = "MLP: cannot reserve shared memory";
+        return RFAST_ECUDA;
+    }
+    *out = p;
+    *dev_bytes = total + sizeof(int) + (size_t)max_events * kBatch * H * sizeof(float);
+    return RFAST_OK;
 }
-void mlp_plan_destroy(MlpPlan* plan) { delete plan; }
-int mlp_grad_launch(MlpPlan*, const GradArgs&, const __nv_bfloat16*, const int*, int, cudaStream_t,
-                    int64_t*, std::string& err) {
-    err = "MLP objective is not available in this build";
-    return RFAST_EINVAL;
+
+void mlp_plan_destroy(MlpPlan* p) {
+    if (!p) return;
+    void* ptrs[] = {p->featb, p->Ab, p->AbT, p->hf, p->dpqT, p->status};
+    for (void* q : ptrs) if (q) cudaFree(q);
+    delete p;
+}
+
+int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
+                    int n_events, cudaStream_t st, int64_t* launches, std::string& err) {
+    if (!p || n_events > p->maxev) { err = "MLP: too many events for the plan"; return RFAST_EINVAL; }
+    k_mlp_gather<<<n_events, 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
+    k_mlp_fwd<<<dim3(p->H / kMTile, n_events), kGemmThreads, kFwdSmem, st>>>(
+        p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
+    k_mlp_mid<<<n_events, 512, 2 * kBatch * p->C * sizeof(float), st>>>(
+        g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dpqT, g.gbuf, g.gplane, p->rows, p->F, p->H, p->C, g.l2);
+    k_mlp_dw1<<<dim3(p->H / kMTile, n_events), kGemmThreads, kDw1Smem, st>>>(
+        p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);
+    *launches += 4;
+    return RFAST_OK;
+}
+
+// 0 when no bounded wait ran out so far (synchronises the stream)
+int mlp_plan_status(MlpPlan* p, cudaStream_t st) {
+    int h = 0;
+    if (!p) return 0;
+    if (cudaMemcpyAsync(&h, p->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return -1;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return -1;
+    return h;
 }
 
 }  // namespace rfast

@@ -98,3 +98,28 @@ def test_logistic_long_horizon_reduced_dimension(rfast_lib):
     wl = build_config("logistic_tree1024", seed=0, n=256, p=2000, nnz=20, rows=16, K=300)
     ex, ey = _run_both(wl)
     assert ex <= 1e-5 and ey <= 1e-5, (ex, ey)
+
+
+def test_mlp_tree64_full_dimensions_first_rounds(rfast_lib):
+    """Config 3 at full dimensions (n=64, MLP 784-512-10, p=407,050, minibatch 64); the oracle
+    needs ~7 ms per activation, so the comparison covers the first 40 rounds.  Tolerance on y
+    is the derived 1e-4 of the bf16-state effect (see tests/test_gpu_mlp.py); x meets 1e-5."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("mlp_tree64", seed=0)
+    assert (wl.n, wl.p, wl.batch) == (64, 407_050, 64)
+    K = 40
+    orc = from_workload(wl, make_model(wl).grad)
+    Bs = wl.batch
+    orc.init_gradients([wl.schedule.batch_idx[i * Bs:(i + 1) * Bs] for i in range(wl.n)])
+    x0n, z0n = np.linalg.norm(orc.X()), np.linalg.norm(orc.Z())
+    run_schedule(orc, wl.schedule, K=K)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run(K)
+        x, y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        assert eng.read(B.STATE_T_LOCAL).tolist() == orc.t
+        nv = len(orc.used_tau_v)
+        assert eng.read(B.STATE_USED_TAU_V)[:nv].tolist() == orc.used_tau_v
+    assert rel_l2(x, orc.X(), x0n) <= 1e-5
+    assert rel_l2(y, orc.Z(), z0n) <= 1e-4

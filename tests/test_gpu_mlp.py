@@ -1,0 +1,88 @@
+"""Parity of the tensor-core MLP gradient path (config 3) with the oracle.
+
+The MLP rounds its GEMM operands to bf16.  Rounding the *state* W1 turns a 1e-7 relative
+difference between the fp32 iterate and the fp64 oracle iterate into a different bf16 weight
+for a few weights in 1e5, and each such flip moves a hidden unit by ~1e-4: along a trajectory
+the two sides therefore agree to about 1e-5 in the gradients and trackers, not to fp32
+rounding.  The tests separate the two effects: from identical state the gradient must agree
+to fp32 accuracy; along a trajectory x must meet 1e-5 and y a derived 1e-4."""
+
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from oracle import from_workload, make_model, rel_l2, run_schedule
+from workloads import build_config
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    dict(n=6, F=64, H=128, C=10, rows=128, K=20, batch=64),
+    dict(n=5, F=48, H=256, C=3, rows=96, K=12, batch=64),
+    dict(n=8, F=784, H=512, C=10, rows=256, K=15, batch=64),
+]
+
+
+def _blocks(wl):
+    H, F, C = wl.dims["n_hidden"], wl.dims["n_features"], wl.dims["n_classes"]
+    o1, o2, o3 = H * F, H * F + H, H * F + H + C * H
+    return {"W1": (0, o1), "b1": (o1, o2), "W2": (o2, o3), "b2": (o3, wl.p)}
+
+
+@pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
+def test_mlp_gradient_from_identical_state(rfast_lib, ov):
+    """Initial gradients (same x0 on both sides): every block to fp32 accuracy."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("mlp_tree64", seed=1, **ov)
+    m = make_model(wl)
+    Bs = wl.batch
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        g = eng.read(B.STATE_G_LAST)
+    ref = np.stack([m.grad(i, wl.x0[i].astype(np.float64), wl.schedule.batch_idx[i * Bs:(i + 1) * Bs])
+                    for i in range(wl.n)])
+    for nm, (a, b) in _blocks(wl).items():
+        assert rel_l2(g[:, a:b], ref[:, a:b]) <= 1e-5, nm
+    assert rel_l2(g, ref) <= 2e-6
+
+
+@pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
+def test_mlp_trajectory_and_gradient_at_device_iterate(rfast_lib, ov):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("mlp_tree64", seed=1, **ov)
+    m = make_model(wl)
+    orc = from_workload(wl, m.grad)
+    Bs, s = wl.batch, wl.schedule
+    orc.init_gradients([s.batch_idx[i * Bs:(i + 1) * Bs] for i in range(wl.n)])
+    x0n, z0n = np.linalg.norm(orc.X()), np.linalg.norm(orc.Z())
+    run_schedule(orc, s)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(s)
+        eng.run()
+        x, y, g = eng.read(B.STATE_X), eng.read(B.STATE_Y), eng.read(B.STATE_G_LAST)
+        assert eng.read(B.STATE_USED_TAU_V).tolist() == orc.used_tau_v
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
+        assert eng.read(B.STATE_T_LOCAL).tolist() == orc.t
+    assert np.isfinite(x).all() and np.isfinite(y).all()
+    assert rel_l2(x, orc.X(), x0n) <= 1e-5
+    assert rel_l2(y, orc.Z(), z0n) <= 1e-4
+    # teacher-forced: the oracle's gradient at the device's own fp32 iterate, same last sample;
+    # the bf16 decisions on the state are then identical on both sides
+    last = {}
+    for ev, i in enumerate(s.act_node):
+        last[int(i)] = wl.n + ev
+    ref = np.stack([m.grad(i, x[i].astype(np.float64),
+                           s.batch_idx[last.get(i, i) * Bs:(last.get(i, i) + 1) * Bs]) for i in range(wl.n)])
+    assert rel_l2(g, ref) <= 1e-5
+
+
+def test_mlp_unsupported_shape_is_refused(rfast_lib):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import EINVAL, RFastError
+    wl = build_config("mlp_tree64", seed=1, n=4, F=20, H=96, C=3, rows=32, K=3, batch=8)
+    with pytest.raises(RFastError) as ei:
+        pkg.Engine(wl)
+    assert ei.value.code == EINVAL and "tensor-core path" in str(ei.value)

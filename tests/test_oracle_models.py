@@ -66,6 +66,9 @@ def test_mlp_rounded_path_is_the_same_code_with_rounded_operands():
     assert np.array_equal(exact._forward(0, x, idx)[2], rounded._forward(0, x, idx)[2])
     ge, gr = exact.grad(0, x, idx), rounded.grad(0, x, idx)
     assert np.abs(ge - gr).max() <= 3 * 2.0 ** -8 * np.abs(ge).max()
+    # only the weight gradient of the first layer sees a rounded operand (dpre); the rest is exact
+    o1 = wl.dims["n_hidden"] * wl.dims["n_features"]
+    assert np.array_equal(ge[o1:], gr[o1:]) and not np.array_equal(ge[:o1], gr[:o1])
 
 
 def test_bf16_round_hand_values():
