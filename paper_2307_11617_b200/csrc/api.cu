@@ -55,6 +55,9 @@ struct rfast_ctx {
     int max_round_events = 0;
     int round = 0;
     int64_t launches = 0;
+    cudaGraphExec_t graph_exec = nullptr;   // recorded span of rounds [graph_r0, graph_r1)
+    int graph_r0 = -1, graph_r1 = -1;
+    int64_t graph_launches = 0;
     size_t dev_bytes = 0, sched_bytes = 0;
     std::string err;
 };
@@ -103,6 +106,8 @@ int upload_rows(rfast_ctx* ctx, float* dst, const float* src, int64_t rows) {
 }
 
 void free_schedule(rfast_ctx* c) {
+    if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+    c->graph_r0 = c->graph_r1 = -1;
     for (void* q : c->sched_allocs) cudaFree(q);
     c->sched_allocs.clear();
     c->dev_bytes -= c->sched_bytes;
@@ -188,8 +193,7 @@ int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
         case RFAST_MODEL_LOGISTIC_SPARSE: {
             g.B = ctx->batch;
             k_logit_coef<<<dim3((g.B + 7) / 8, nev), 256, 0, st>>>(g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->label, ctx->scratch);
-            k_logit_grad<<<dim3((unsigned)((g.p + kLogitTile - 1) / kLogitTile), nev), 256, 0, st>>>(
-                g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->scratch);
+            k_logit_scatter<<<nev, 256, 0, st>>>(g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->scratch);
             ctx->launches += 2;
             break;
         }
@@ -231,6 +235,11 @@ int reset_state(rfast_ctx* ctx) {
         if (ctx->model == RFAST_MODEL_MLP) {      // bf16 copy of x0 for the matrix products
             k_rows_to_bf16<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
                 ctx->x, ctx->xb, ctx->stride, n4);
+            CK(cudaGetLastError());
+        }
+        if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {   // dense term of the gradient; the sampled rows are added on top
+            k_scale_rows<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
+                ctx->x, ctx->gbuf, ctx->stride, n4, ctx->l2);
             CK(cudaGetLastError());
         }
         // z_i^0 = g_i^0 = grad f_i(x_i^0; zeta_i^0)  (initialisation line of Algorithm 1)
@@ -416,11 +425,8 @@ int rfast_reset(rfast_ctx* ctx) {
     return reset_state(ctx);
 }
 
-int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
-    if (!ctx) return RFAST_EINVAL;
-    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
-    if (rounds < 0 || ctx->round + (int64_t)rounds > ctx->comp.K)
-        return set_err(ctx, RFAST_ESTATE, "run would pass the end of the schedule");
+// Enqueues the kernels of rounds [r0, r1) on the handle's stream.
+static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
     const Compiled& c = ctx->comp;
     RoundArgs a{};
     a.mix_slot = ctx->d_mix_slot; a.mix_w = ctx->d_mix_w;
@@ -429,7 +435,7 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
     a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
     a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
     const bool big = a.n4 >= kThreads * 4;
-    for (int r = ctx->round; r < ctx->round + rounds; ++r) {
+    for (int r = r0; r < r1; ++r) {
         const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
         if (nev == 0) continue;
         a.ev = ctx->d_ev + c.act_ptr[r];
@@ -439,18 +445,58 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
             else k_fused_quad<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             ctx->launches += 1;
         } else {
-            if (ctx->model == RFAST_MODEL_MLP) k_mix<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb);
-            else k_mix<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr);
+            const int64_t gplane = (int64_t)ctx->n * ctx->stride;
+            if (ctx->model == RFAST_MODEL_MLP)
+                k_mix<1, true, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb, nullptr, 0, 0.f);
+            else if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE)
+                k_mix<1, false, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr, ctx->gbuf, gplane, ctx->l2);
+            else
+                k_mix<1, false, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr, nullptr, 0, 0.f);
             ctx->launches += 1;
             int rc = launch_gradients(ctx, a.ev, nev);
             if (rc != RFAST_OK) return rc;
-            if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
-            else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, (int64_t)ctx->n * ctx->stride);
+            if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+            else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
             ctx->launches += 1;
         }
     }
     CK(cudaGetLastError());
-    ctx->round += rounds;
+    return RFAST_OK;
+}
+
+int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (rounds < 0 || ctx->round + (int64_t)rounds > ctx->comp.K)
+        return set_err(ctx, RFAST_ESTATE, "run would pass the end of the schedule");
+    const int r0 = ctx->round, r1 = ctx->round + rounds;
+    // Many short kernels per round make the launch path the bottleneck of the small problems:
+    // the rounds of one call are recorded once into a CUDA graph and replayed when the same
+    // span is run again (after a reset).  The legacy default stream cannot be captured; there
+    // the kernels are launched directly.
+    const bool graph_ok = ctx->stream != nullptr && rounds >= 2;
+    if (graph_ok && ctx->graph_exec && ctx->graph_r0 == r0 && ctx->graph_r1 == r1) {
+        CK(cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+        ctx->launches += ctx->graph_launches;
+    } else if (graph_ok) {
+        if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
+        const int64_t l0 = ctx->launches;
+        CK(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+        int rc = issue_rounds(ctx, r0, r1);
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+        if (rc != RFAST_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+        if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("cudaStreamEndCapture: ") + cudaGetErrorString(e));
+        e = cudaGraphInstantiate(&ctx->graph_exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) { ctx->graph_exec = nullptr; return set_err(ctx, RFAST_ECUDA, std::string("cudaGraphInstantiate: ") + cudaGetErrorString(e)); }
+        ctx->graph_r0 = r0; ctx->graph_r1 = r1; ctx->graph_launches = ctx->launches - l0;
+        CK(cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+    } else {
+        int rc = issue_rounds(ctx, r0, r1);
+        if (rc != RFAST_OK) return rc;
+    }
+    ctx->round = r1;
     if (sync) {
         CK(cudaStreamSynchronize(ctx->stream));
         return check_device_status(ctx);

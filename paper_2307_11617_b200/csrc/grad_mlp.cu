@@ -162,22 +162,30 @@ __global__ void k_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restri
 // Sampled rows of one activation, as the two GEMMs want them:
 //   Ab  [ev][B][Fp]  row k = features of sample k, zero beyond F (K-major operand of pre)
 //   AbT [ev][F][B]   the transpose                      (K-major operand of gW1, K = batch)
+// One CTA moves a 64 x 64 tile and transposes it through shared memory.  grid = (Fp / 64, events)
 __global__ void __launch_bounds__(256)
 k_mlp_gather(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx,
              const __nv_bfloat16* __restrict__ featb, __nv_bfloat16* __restrict__ Ab,
              __nv_bfloat16* __restrict__ AbT, int rows, int F, int Fp) {
-    const EvDesc e = evs[blockIdx.x];
-    const int* idx = batch_idx + (int64_t)e.sample * kBatch;
+    __shared__ __nv_bfloat16 tile[kBatch][kKBlock + 2];
+    __shared__ int idx[kBatch];
+    const int ev = blockIdx.y, f0 = blockIdx.x * kKBlock;
+    const EvDesc e = evs[ev];
+    if (threadIdx.x < kBatch) idx[threadIdx.x] = batch_idx[(int64_t)e.sample * kBatch + threadIdx.x];
+    __syncthreads();
     const __nv_bfloat16* shard = featb + (int64_t)e.node * rows * F;
-    __nv_bfloat16* ab = Ab + (int64_t)blockIdx.x * kBatch * Fp;
-    __nv_bfloat16* abt = AbT + (int64_t)blockIdx.x * F * kBatch;
-    for (int q = threadIdx.x; q < kBatch * Fp; q += 256) {
-        const int k = q / Fp, f = q % Fp;
-        ab[q] = f < F ? shard[(int64_t)idx[k] * F + f] : __float2bfloat16_rn(0.f);
+    __nv_bfloat16* ab = Ab + (int64_t)ev * kBatch * Fp;
+    __nv_bfloat16* abt = AbT + (int64_t)ev * F * kBatch;
+    for (int q = threadIdx.x; q < kBatch * kKBlock; q += 256) {
+        const int k = q / kKBlock, f = q % kKBlock;
+        const __nv_bfloat16 v = (f0 + f < F) ? shard[(int64_t)idx[k] * F + f0 + f] : __float2bfloat16_rn(0.f);
+        ab[(int64_t)k * Fp + f0 + f] = v;
+        tile[k][f] = v;
     }
-    for (int q = threadIdx.x; q < F * kBatch; q += 256) {
+    __syncthreads();
+    for (int q = threadIdx.x; q < kBatch * kKBlock; q += 256) {
         const int f = q / kBatch, k = q % kBatch;
-        abt[q] = shard[(int64_t)idx[k] * F + f];
+        if (f0 + f < F) abt[(int64_t)(f0 + f) * kBatch + k] = tile[k][f];
     }
 }
 
@@ -286,14 +294,37 @@ k_mlp_mid(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, con
     const float* W2 = x + row + oW2;
     float* g = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
-    for (int k = warp; k < kBatch; k += nwarp)
-        for (int c = 0; c < C; ++c) {
-            float s = 0.f;
-            for (int j = lane; j < H; j += 32)
-                s = fmaf(h[(int64_t)k * H + j], W2[(int64_t)c * H + j], s);
-            s = warp_sum(s);
-            if (lane == 0) logit[k * C + c] = s + x[row + ob2 + c];
+    // logits: a warp owns the rows k = warp, warp + nwarp, ... (4 with 16 warps); every lane
+    // walks the hidden units j = lane, lane + 32, ... once and feeds all of its rows and classes
+    for (int kbase = warp; kbase < kBatch; kbase += 4 * nwarp) {
+        float acc[4][16];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 16; ++c) acc[r][c] = 0.f;
+        for (int j = lane; j < H; j += 32) {
+            float w2[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int k = kbase + r * nwarp;
+                const float hv = k < kBatch ? h[(int64_t)k * H + j] : 0.f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) if (c < C) acc[r][c] = fmaf(hv, w2[c], acc[r][c]);
+            }
         }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int k = kbase + r * nwarp;
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                if (c < C) {
+                    const float s = warp_sum(acc[r][c]);
+                    if (lane == 0 && k < kBatch) logit[k * C + c] = s + x[row + ob2 + c];
+                }
+        }
+    }
     __syncthreads();
     if (threadIdx.x < kBatch) {
         const int k = threadIdx.x;
@@ -343,100 +374,80 @@ k_mlp_mid(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, con
     }
 }
 
-// gW1 slab [h0 .. h0+128) x F = q(dpre)^T (K = batch) x A, N tiles of NT features, accumulators
-// double-buffered in tensor memory.  grid = (H / 128, events)
-constexpr int kStagesB = 3;
+// One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A).
+// grid = (H / 128, F / NT, events)
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmAT,
           const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
           float* __restrict__ gbuf, int64_t gplane, int F, int H, int NT, float l2, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr int kABytes = kMTile * kKBlock * 2;          // q(dpre)^T slab, loaded once
-    constexpr int kBMax = 128 * kKBlock * 2;               // room for one N tile of A^T
+    constexpr int kABytes = kMTile * kKBlock * 2;          // q(dpre)^T slab
     uint8_t* sA = smem;
-    uint8_t* sB = smem + kABytes;                          // [stages][NT][64] bf16, stage pitch kBMax
-    __shared__ uint64_t a_full, b_full[kStagesB], b_empty[kStagesB], acc_full[2], acc_empty[2];
+    uint8_t* sB = smem + kABytes;                          // [NT][64] bf16 tile of A^T
+    __shared__ uint64_t ab_full, acc_full;
     __shared__ uint32_t tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ev = blockIdx.y, h0 = blockIdx.x * kMTile;
+    const int ev = blockIdx.z, h0 = blockIdx.x * kMTile, f0 = blockIdx.y * NT;
     const EvDesc e = evs[ev];
-    const int ntiles = F / NT;
     if (threadIdx.x == 0) {
-        mbar_init(&a_full, 1);
-        for (int s = 0; s < kStagesB; ++s) { mbar_init(&b_full[s], 1); mbar_init(&b_empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+        mbar_init(&ab_full, 1);
+        mbar_init(&acc_full, 1);
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(&tmem_base, 256);
+    if (warp == 1) tmem_alloc(&tmem_base, 128);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tacc = tmem_base;
 
     if (warp == 0 && lane == 0) {                          // ---- TMA producer
-        bool ok = true;
-        mbar_expect_tx(&a_full, kABytes);
-        tma_load_2d(sA, &tmD, &a_full, 0, ev * H + h0);
-        for (int t = 0; t < ntiles; ++t) {
-            const int s = t % kStagesB;
-            if (t >= kStagesB) ok = mbar_wait(&b_empty[s], ((t / kStagesB) - 1) & 1);
-            if (!ok) break;
-            mbar_expect_tx(&b_full[s], NT * kKBlock * 2);
-            tma_load_2d(sB + s * kBMax, &tmAT, &b_full[s], 0, ev * F + t * NT);
-        }
-        if (!ok) atomicExch(status, kErrProducer);
+        mbar_expect_tx(&ab_full, kABytes + NT * kKBlock * 2);
+        tma_load_2d(sA, &tmD, &ab_full, 0, ev * H + h0);
+        tma_load_2d(sB, &tmAT, &ab_full, 0, ev * F + f0);
     } else if (warp == 1 && lane == 0) {                   // ---- MMA issuer
         const uint32_t idesc = umma_idesc_bf16(kMTile, NT);
-        bool ok = mbar_wait(&a_full, 0);
-        const uint64_t ad = umma_desc_sw128(smem_u32(sA));
-        for (int t = 0; t < ntiles && ok; ++t) {
-            const int s = t % kStagesB, a = t & 1;
-            if (t >= 2) ok = mbar_wait(&acc_empty[a], ((t >> 1) - 1) & 1);
-            if (ok) ok = mbar_wait(&b_full[s], (t / kStagesB) & 1);
-            if (!ok) break;
+        const bool ok = mbar_wait(&ab_full, 0);
+        if (ok) {
             tc_fence_after();
-            const uint64_t bd = umma_desc_sw128(smem_u32(sB + s * kBMax));
+            const uint64_t ad = umma_desc_sw128(smem_u32(sA));
+            const uint64_t bd = umma_desc_sw128(smem_u32(sB));
 #pragma unroll
             for (int k = 0; k < kKBlock / 16; ++k)
-                umma_bf16(tacc + a * 128, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, k ? 1u : 0u);
-            umma_commit(&b_empty[s]);
-            umma_commit(&acc_full[a]);
+                umma_bf16(tacc, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), idesc, k ? 1u : 0u);
+            umma_commit(&acc_full);
+        } else {
+            atomicExch(status, kErrMma);
+            mbar_arrive(&acc_full);
         }
-        if (!ok) { atomicExch(status, kErrMma); mbar_arrive(&acc_full[0]); mbar_arrive(&acc_full[1]); }
     } else if (warp >= 2) {                                // ---- epilogue: TMEM -> global
         const int q = warp & 3;
         const int j = h0 + q * 32 + lane;
         const int64_t row = (int64_t)e.node * stride;
-        float* grow = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row + (int64_t)j * F;
-        const float* xrow = x + row + (int64_t)j * F;
-        for (int t = 0; t < ntiles; ++t) {
-            const int a = t & 1;
-            const bool ok = mbar_wait(&acc_full[a], (t >> 1) & 1);
-            tc_fence_after();
-            if (!ok || atomicAdd(status, 0) != kErrNone) { if (!ok && lane == 0) atomicExch(status, kErrEpilogue); break; }
+        float* grow = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row + (int64_t)j * F + f0;
+        const float* xrow = x + row + (int64_t)j * F + f0;
+        const bool ok = mbar_wait(&acc_full, 0);
+        tc_fence_after();
+        if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
+        else if (atomicAdd(status, 0) == kErrNone) {
             for (int c0 = 0; c0 < NT; c0 += 16) {
                 float v[16];
-                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + a * 128 + c0, v);
-                const int f0 = t * NT + c0;
+                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
 #pragma unroll
                 for (int i = 0; i < 16; i += 4) {
                     float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
                     if (l2 != 0.f) {
-                        const float4 xv = *reinterpret_cast<const float4*>(xrow + f0 + i);
+                        const float4 xv = *reinterpret_cast<const float4*>(xrow + c0 + i);
                         o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
                     }
-                    *reinterpret_cast<float4*>(grow + f0 + i) = o;
+                    *reinterpret_cast<float4*>(grow + c0 + i) = o;
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[a]);
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 256); }
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 128); }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -475,7 +486,7 @@ bool make_map(CUtensorMap* m, void* base, int rank, const uint64_t* dims, const 
 }
 
 constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 1024;
-constexpr size_t kDw1Smem = kMTile * kKBlock * 2 + kStagesB * (128 * kKBlock * 2) + 1024;
+constexpr size_t kDw1Smem = kMTile * kKBlock * 2 + 128 * kKBlock * 2 + 1024;
 
 }  // namespace
 
@@ -548,12 +559,12 @@ void mlp_plan_destroy(MlpPlan* p) {
 int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
                     int n_events, cudaStream_t st, int64_t* launches, std::string& err) {
     if (!p || n_events > p->maxev) { err = "MLP: too many events for the plan"; return RFAST_EINVAL; }
-    k_mlp_gather<<<n_events, 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
+    k_mlp_gather<<<dim3(p->Fp / kKBlock, n_events), 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
     k_mlp_fwd<<<dim3(p->H / kMTile, n_events), kGemmThreads, kFwdSmem, st>>>(
         p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
     k_mlp_mid<<<n_events, 512, 2 * kBatch * p->C * sizeof(float), st>>>(
         g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dpqT, g.gbuf, g.gplane, p->rows, p->F, p->H, p->C, g.l2);
-    k_mlp_dw1<<<dim3(p->H / kMTile, n_events), kGemmThreads, kDw1Smem, st>>>(
+    k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
         p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);
     *launches += 4;
     return RFAST_OK;

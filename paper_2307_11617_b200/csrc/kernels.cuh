@@ -285,11 +285,12 @@ k_quad_grad(const float* __restrict__ x, const float* __restrict__ qd, const flo
 
 // ---------------------------------------------------------------------------------------------
 // S1 + S2a for objectives whose gradient needs the whole new x first.  Optionally leaves a
-// bf16 copy of the new x (operand of the MLP's matrix products).  grid = (tiles, events)
+// bf16 copy of the new x (operand of the MLP's matrix products), or starts the new gradient
+// row with the dense term l2 * x (sparse objective).  grid = (tiles, events)
 // ---------------------------------------------------------------------------------------------
-template <int U, bool BF16>
+template <int U, bool BF16, bool GINIT>
 __global__ void __launch_bounds__(kThreads)
-k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
+k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int64_t gplane, float l2) {
     const EvDesc e = a.ev[blockIdx.y];
     const int64_t row = (int64_t)e.node * a.stride;
     float* xr = a.x + row;
@@ -327,6 +328,8 @@ k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
         if (i4 < a.n4) {
             // the gradient kernels re-read x soon: keep it cacheable
             reinterpret_cast<float4*>(xr)[i4] = acc[u];
+            if (GINIT)      // dense part of a sparse objective's gradient: g_new = l2 * x_new
+                reinterpret_cast<float4*>(gbuf + (int64_t)(e.g_par ^ 1) * gplane + row)[i4] = f4_scale(l2, acc[u]);
             if (BF16) {
                 __nv_bfloat162 lo = __floats2bfloat162_rn(acc[u].x, acc[u].y);
                 __nv_bfloat162 hi = __floats2bfloat162_rn(acc[u].z, acc[u].w);
@@ -482,41 +485,35 @@ k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restri
     }
 }
 
-// Sparse logistic regression, phase 2: g = l2 x + sum_k coef_k a_k on a tile of kTile
-// coordinates held in shared memory; rows are added one after the other (fixed order), the
-// entries of one row land on distinct coordinates.  grid = (ceil(p / kTile), events)
-constexpr int kLogitTile = 2048;
+// Sparse logistic regression, phase 2: g += sum_k coef_k a_k on top of the dense term l2 * x
+// that is already in the gradient row.  One CTA per activation; the sampled rows are added one
+// after the other (a barrier in between keeps the order fixed, so repeated columns add up in
+// batch order on every run), the entries of one row land on distinct coordinates.
+// grid = events
 __global__ void __launch_bounds__(256)
-k_logit_grad(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col,
-             const float* __restrict__ sp_val, const float* __restrict__ coef) {
-    __shared__ float tile[kLogitTile];
-    __shared__ int64_t lo_s, hi_s;
-    const EvDesc e = g.ev[blockIdx.y];
-    const int64_t c0 = (int64_t)blockIdx.x * kLogitTile;
-    const int64_t c1 = min(c0 + (int64_t)kLogitTile, g.p);
-    const int64_t row = (int64_t)e.node * g.stride;
-    for (int c = threadIdx.x; c < kLogitTile; c += 256)
-        tile[c] = (c0 + c < c1) ? g.l2 * g.x[row + c0 + c] : 0.f;
-    __syncthreads();
+k_logit_scatter(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col,
+                const float* __restrict__ sp_val, const float* __restrict__ coef) {
+    const EvDesc e = g.ev[blockIdx.x];
+    float* out = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + (int64_t)e.node * g.stride;
     for (int k = 0; k < g.B; ++k) {
         const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
         const int64_t r = (int64_t)e.node * g.rows + rrow;
-        if (threadIdx.x == 0) {                      // entries of row r with c0 <= col < c1
-            int64_t lo = sp_ptr[r], hi = sp_ptr[r + 1], end = hi;
-            while (lo < hi) { int64_t m = (lo + hi) >> 1; if (sp_col[m] < c0) lo = m + 1; else hi = m; }
-            lo_s = lo;
-            hi = end;
-            while (lo < hi) { int64_t m = (lo + hi) >> 1; if (sp_col[m] < c1) lo = m + 1; else hi = m; }
-            hi_s = lo;
+        const float ck = coef[(int64_t)blockIdx.x * g.B + k];
+        for (int64_t q = sp_ptr[r] + threadIdx.x; q < sp_ptr[r + 1]; q += 256) {
+            const int c = sp_col[q];
+            out[c] = fmaf(ck, sp_val[q], out[c]);
         }
         __syncthreads();
-        const float ck = coef[(int64_t)blockIdx.y * g.B + k];
-        for (int64_t q = lo_s + threadIdx.x; q < hi_s; q += 256)
-            tile[sp_col[q] - c0] = fmaf(ck, sp_val[q], tile[sp_col[q] - c0]);
-        __syncthreads();
     }
-    float* out = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row;
-    for (int c = threadIdx.x; c0 + c < c1; c += 256) out[c0 + c] = tile[c];
+}
+
+// g = l2 * x for every node (start of the initial gradients of the sparse objective).  grid = (tiles, n)
+__global__ void __launch_bounds__(kThreads)
+k_scale_rows(const float* __restrict__ x, float* __restrict__ out, int64_t stride, int n4, float l2) {
+    const int i4 = blockIdx.x * kThreads + threadIdx.x;
+    if (i4 >= n4) return;
+    const int64_t row = (int64_t)blockIdx.y * stride;
+    reinterpret_cast<float4*>(out + row)[i4] = f4_scale(l2, reinterpret_cast<const float4*>(x + row)[i4]);
 }
 
 // row copy helpers ----------------------------------------------------------------------------

@@ -169,3 +169,40 @@ def test_empty_rounds_and_x0(rfast_lib):
         eng.load_schedule(wl.schedule)
         eng.run()
         _compare(eng, orc, ref0)
+
+
+@pytest.mark.parametrize("name,ov", [
+    ("quad_tree64", dict(n=16, p=5000, K=25)),
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=60, batch=8)),
+    ("logistic_tree1024", dict(n=64, p=3000, rows=8, K=30, batch=4, nnz=40)),
+], ids=["quad", "softmax", "logistic"])
+def test_graph_replay_on_a_user_stream_equals_direct_launches(rfast_lib, name, ov):
+    """On a non-default stream a span of rounds is recorded into a CUDA graph and replayed
+    after a reset; both must be bit-identical to direct launches on the default stream."""
+    import torch
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config(name, seed=5, **ov)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:                      # default stream: direct launches
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        xd, yd = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        direct_launches = eng.query(B.Q_LAUNCHES)
+    stream = torch.cuda.Stream()
+    with pkg.Engine(wl, stream.cuda_stream) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()                                    # records and launches the graph
+        _compare(eng, orc, ref0)
+        x1, y1 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        assert eng.query(B.Q_LAUNCHES) == direct_launches
+        eng.reset()
+        eng.run()                                    # replays it
+        x2, y2 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        assert eng.query(B.Q_LAUNCHES) == 2 * direct_launches
+        eng.reset()
+        eng.run(3)                                   # another span: re-recorded
+        eng.run(wl.schedule.K - 3)
+        x3 = eng.read(B.STATE_X)
+    assert np.array_equal(xd, x1) and np.array_equal(yd, y1)
+    assert np.array_equal(x1, x2) and np.array_equal(y1, y2) and np.array_equal(x1, x3)
