@@ -39,6 +39,8 @@ struct rfast_ctx {
     float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
     int* label = nullptr;
     int64_t* sp_ptr = nullptr;
+    int64_t* sp_tile_ptr = nullptr;   // [n*rows][tiles+1] first entry of each shard row in each coordinate tile
+    int sp_tiles = 0;
     int* sp_col = nullptr;
     float* sp_val = nullptr;
     __nv_bfloat16* xb = nullptr;
@@ -121,6 +123,10 @@ ModelTraffic traffic_of(int model, bool compensated) {
     ModelTraffic mt;
     mt.elementwise = (model == RFAST_MODEL_QUAD_DIAG);
     mt.data_streams = (mt.elementwise ? 2 : 0) + (compensated ? 2 : 0);
+    // sparse logistic: the fused gradient+tracking pass reads x, z, g_old and writes g (4);
+    // the others: gradient reads x (the MLP: a bf16 copy written by the mix pass), writes g,
+    // tracking reads z, g_old, g_new (5).  z's write and the packets are counted elsewhere.
+    mt.grad_track_streams = (model == RFAST_MODEL_LOGISTIC_SPARSE ? 4 : 5) + (mt.elementwise ? 0 : (compensated ? 2 : 0));
     return mt;
 }
 
@@ -165,13 +171,31 @@ int validate_problem(const rfast_problem* p, std::string& err) {
 
 dim3 tile_grid(int n4, int U, int events) { return dim3((n4 + kThreads * U - 1) / (kThreads * U), events); }
 
-// sample gradients of `nev` events (descriptors on the device) into gbuf[par^1]
-int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
+GradArgs grad_args(rfast_ctx* ctx, const EvDesc* d_ev) {
     GradArgs g{};
     g.ev = d_ev; g.x = ctx->x; g.gbuf = ctx->gbuf; g.stride = ctx->stride;
     g.gplane = (int64_t)ctx->n * ctx->stride;
     g.batch_idx = ctx->d_batch_idx; g.rows = ctx->rows; g.F = ctx->F; g.C = ctx->C; g.H = ctx->H;
-    g.p = ctx->p; g.l2 = ctx->l2;
+    g.p = ctx->p; g.l2 = ctx->l2; g.B = ctx->batch;
+    return g;
+}
+
+// sparse logistic: gradient tile + tracking in one pass (or the gradient alone for the initial trackers)
+int launch_logit_track(rfast_ctx* ctx, const RoundArgs& a, const EvDesc* d_ev, int nev, int init_only) {
+    GradArgs g = grad_args(ctx, d_ev);
+    const dim3 grid(ctx->sp_tiles, nev);
+    if (ctx->compensated)
+        k_logit_track<true><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_tiles, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
+    else
+        k_logit_track<false><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_tiles, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
+    ctx->launches += 1;
+    CK(cudaGetLastError());
+    return RFAST_OK;
+}
+
+// sample gradients of `nev` events (descriptors on the device) into gbuf[par^1]
+int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
+    GradArgs g = grad_args(ctx, d_ev);
     cudaStream_t st = ctx->stream;
     switch (ctx->model) {
         case RFAST_MODEL_LEAST_SQUARES: {
@@ -191,10 +215,8 @@ int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
             break;
         }
         case RFAST_MODEL_LOGISTIC_SPARSE: {
-            g.B = ctx->batch;
             k_logit_coef<<<dim3((g.B + 7) / 8, nev), 256, 0, st>>>(g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->label, ctx->scratch);
-            k_logit_scatter<<<nev, 256, 0, st>>>(g, ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->scratch);
-            ctx->launches += 2;
+            ctx->launches += 1;       // the second phase is fused with the tracking pass (k_logit_track)
             break;
         }
         case RFAST_MODEL_MLP: {
@@ -237,14 +259,14 @@ int reset_state(rfast_ctx* ctx) {
                 ctx->x, ctx->xb, ctx->stride, n4);
             CK(cudaGetLastError());
         }
-        if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {   // dense term of the gradient; the sampled rows are added on top
-            k_scale_rows<<<dim3((n4 + kThreads - 1) / kThreads, ctx->n), kThreads, 0, ctx->stream>>>(
-                ctx->x, ctx->gbuf, ctx->stride, n4, ctx->l2);
-            CK(cudaGetLastError());
-        }
         // z_i^0 = g_i^0 = grad f_i(x_i^0; zeta_i^0)  (initialisation line of Algorithm 1)
         int rc = launch_gradients(ctx, ctx->d_init_ev, ctx->n);
         if (rc != RFAST_OK) return rc;
+        if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {
+            RoundArgs a{};
+            a.stride = ctx->stride; a.n4 = n4;
+            if ((rc = launch_logit_track(ctx, a, ctx->d_init_ev, ctx->n, 1)) != RFAST_OK) return rc;
+        }
         CK(cudaMemcpyAsync(ctx->z, ctx->gbuf, plane, cudaMemcpyDeviceToDevice, ctx->stream));
     }
     ctx->round = 0;
@@ -265,7 +287,7 @@ void rfast_destroy(rfast_ctx* c) {
     free_schedule(c);
     if (c->mlp) mlp_plan_destroy(c->mlp);
     void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
-                    c->sp_ptr, c->sp_col, c->sp_val, c->xb};
+                    c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete c;
 }
@@ -336,6 +358,23 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
                         return set_err(ctx, RFAST_EINVAL, "sp_col must be strictly ascending inside a row and below p");
                 }
                 if (prob->label[r] != 1 && prob->label[r] != -1) return set_err(ctx, RFAST_EINVAL, "labels must be -1 or +1");
+            }
+            {   // per shard row, where each tile of kLogitTile coordinates starts (one walk over the entries)
+                ctx->sp_tiles = (int)((ctx->p + kLogitTile - 1) / kLogitTile);
+                std::vector<int64_t> tp((size_t)nrows * (ctx->sp_tiles + 1));
+                for (size_t r = 0; r < nrows; ++r) {
+                    int64_t q = prob->sp_rowptr[r];
+                    const int64_t qe = prob->sp_rowptr[r + 1];
+                    int64_t* dst = tp.data() + r * (ctx->sp_tiles + 1);
+                    for (int t = 0; t <= ctx->sp_tiles; ++t) {
+                        const int64_t bound = (int64_t)t * kLogitTile;
+                        while (q < qe && prob->sp_col[q] < bound) ++q;
+                        dst[t] = q;
+                    }
+                }
+                CK(dev_alloc(ctx, &ctx->sp_tile_ptr, tp.size()));
+                CK(cudaMemcpyAsync(ctx->sp_tile_ptr, tp.data(), tp.size() * sizeof(int64_t), cudaMemcpyHostToDevice, ctx->stream));
+                CK(cudaStreamSynchronize(ctx->stream));       // tp goes out of scope
             }
             CK(dev_alloc(ctx, &ctx->sp_ptr, nrows + 1));
             CK(dev_alloc(ctx, &ctx->sp_col, (size_t)nnz));
@@ -448,16 +487,18 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
             const int64_t gplane = (int64_t)ctx->n * ctx->stride;
             if (ctx->model == RFAST_MODEL_MLP)
                 k_mix<1, true, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb, nullptr, 0, 0.f);
-            else if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE)
-                k_mix<1, false, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr, ctx->gbuf, gplane, ctx->l2);
             else
                 k_mix<1, false, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr, nullptr, 0, 0.f);
             ctx->launches += 1;
             int rc = launch_gradients(ctx, a.ev, nev);
             if (rc != RFAST_OK) return rc;
-            if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
-            else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
-            ctx->launches += 1;
+            if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {
+                if ((rc = launch_logit_track(ctx, a, a.ev, nev, 0)) != RFAST_OK) return rc;
+            } else {
+                if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                ctx->launches += 1;
+            }
         }
     }
     CK(cudaGetLastError());

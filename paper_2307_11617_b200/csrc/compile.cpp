@@ -360,7 +360,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             // packet leaves) and x; S2b/S2c read the news, write z and the running sums
             int64_t st = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
             if (mt.elementwise) st += mt.data_streams;
-            else st += 1 /*gradient reads x*/ + 1 /*writes g*/ + 3 /*track re-reads z, g_old, g_new*/;
+            else st += mt.grad_track_streams;
             streams += st;
         }
         c.round_streams[r + 1] = c.round_streams[r] + streams;

@@ -145,6 +145,7 @@ struct MlpPlan {
     int64_t stride = 0;
     __nv_bfloat16 *featb = nullptr, *Ab = nullptr, *AbT = nullptr, *dpqT = nullptr;
     float* hf = nullptr;               // [ev][B][H] hidden activations
+    float* dlog = nullptr;             // [ev][B][C] gradient w.r.t. the logits
     int* status = nullptr;
     CUtensorMap tmW1, tmA, tmD, tmAT;
 };
@@ -202,12 +203,14 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
     uint8_t* sB = smem + kStagesFwd * kABytes;            // [stages][64][64] bf16
     __shared__ uint64_t full[kStagesFwd], empty[kStagesFwd], acc_full;
     __shared__ uint32_t tmem_base;
+    __shared__ volatile int aborted;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ev = blockIdx.y, h0 = blockIdx.x * kMTile;
     const EvDesc e = evs[ev];
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesFwd; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         mbar_init(&acc_full, 1);
+        aborted = 0;
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&tmem_base, 64);
@@ -250,12 +253,12 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
             umma_commit(&empty[s]);
         }
         if (ok) umma_commit(&acc_full);
-        else { atomicExch(status, kErrMma); mbar_arrive(&acc_full); }
+        else { atomicExch(status, kErrMma); aborted = 1; __threadfence_block(); mbar_arrive(&acc_full); }
     } else if (warp >= 2) {                                // ---- epilogue: TMEM -> relu -> hf
         const bool ok = mbar_wait(&acc_full, 0);
         tc_fence_after();
         if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
-        else if (atomicAdd(status, 0) == kErrNone) {
+        else if (!aborted) {
             const int q = warp & 3;                         // this warp owns tensor-memory lanes 32q .. 32q+31
             const int j = h0 + q * 32 + lane;               // hidden unit
             const float b1 = x[(int64_t)e.node * stride + (int64_t)H * F + j];
@@ -275,103 +278,97 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 64); }
 }
 
-// Everything between the two big products, one CTA per activation (CUDA cores):
-// logits, softmax, dlog; gW2, gb2, dh, dpre, gb1; q(dpre)^T for the second product.
-// grid = events, 512 threads; dynamic shared memory: 2 * B * C floats
-__global__ void __launch_bounds__(512)
-k_mlp_mid(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
-          const float* __restrict__ x, int64_t stride,
-          const float* __restrict__ hf, __nv_bfloat16* __restrict__ dpqT,
-          float* __restrict__ gbuf, int64_t gplane, int rows, int F, int H, int C, float l2) {
-    extern __shared__ float sm[];
-    float* logit = sm;                     // [B][C]
-    float* dl = sm + kBatch * C;           // [B][C] dlog
-    const int ev = blockIdx.x;
+// Output layer forward, softmax and dlog = (softmax - onehot) / B: one warp per sampled row.
+// grid = (B / 8, events), 256 threads.  dlog: [events][B][C]; CTA 0's first warps also leave gb2.
+__global__ void __launch_bounds__(256)
+k_mlp_logits(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
+             const float* __restrict__ x, int64_t stride, const float* __restrict__ hf,
+             float* __restrict__ dlog, int rows, int F, int H, int C) {
+    const int ev = blockIdx.y;
+    const EvDesc e = evs[ev];
+    const int64_t row = (int64_t)e.node * stride;
+    const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k = blockIdx.x * 8 + warp;
+    const float* h = hf + ((int64_t)ev * kBatch + k) * H;
+    const float* W2 = x + row + oW2;
+    float acc[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+    for (int j = lane; j < H; j += 32) {
+        // all loads of the iteration first, then the arithmetic: the loads then overlap
+        float w[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) w[c] = c < C ? W2[(int64_t)c * H + j] : 0.f;
+        const float hv = h[j];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) acc[c] = fmaf(hv, w[c], acc[c]);
+    }
+    float lg[16], m = -3.0e38f;
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        if (c < C) { lg[c] = warp_sum(acc[c]) + x[row + ob2 + c]; m = fmaxf(m, lg[c]); }
+    float den = 0.f;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) if (c < C) den += expf(lg[c] - m);
+    const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        if (c < C && lane == c)
+            dlog[((int64_t)ev * kBatch + k) * C + c] = (expf(lg[c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)kBatch;
+}
+
+// Backward through the output layer for a slab of 128 hidden units: gW2, gb1, dpre and its
+// bf16 transpose for the second big product; the first slab also sums gb2.
+// grid = (H / 128, events), 128 threads; dynamic shared memory: B * C floats
+__global__ void __launch_bounds__(128)
+k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
+           const float* __restrict__ hf, const float* __restrict__ dlog, __nv_bfloat16* __restrict__ dpqT,
+           float* __restrict__ gbuf, int64_t gplane, int F, int H, int C, float l2) {
+    extern __shared__ float dl[];            // [B][C]
+    const int ev = blockIdx.y;
     const EvDesc e = evs[ev];
     const int64_t row = (int64_t)e.node * stride;
     const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
     const float* h = hf + (int64_t)ev * kBatch * H;
     const float* W2 = x + row + oW2;
     float* g = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
-    // logits: a warp owns the rows k = warp, warp + nwarp, ... (4 with 16 warps); every lane
-    // walks the hidden units j = lane, lane + 32, ... once and feeds all of its rows and classes
-    for (int kbase = warp; kbase < kBatch; kbase += 4 * nwarp) {
-        float acc[4][16];
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-#pragma unroll
-            for (int c = 0; c < 16; ++c) acc[r][c] = 0.f;
-        for (int j = lane; j < H; j += 32) {
-            float w2[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f;
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const int k = kbase + r * nwarp;
-                const float hv = k < kBatch ? h[(int64_t)k * H + j] : 0.f;
-#pragma unroll
-                for (int c = 0; c < 16; ++c) if (c < C) acc[r][c] = fmaf(hv, w2[c], acc[r][c]);
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int k = kbase + r * nwarp;
-#pragma unroll
-            for (int c = 0; c < 16; ++c)
-                if (c < C) {
-                    const float s = warp_sum(acc[r][c]);
-                    if (lane == 0 && k < kBatch) logit[k * C + c] = s + x[row + ob2 + c];
-                }
-        }
-    }
+    for (int q = threadIdx.x; q < kBatch * C; q += 128) dl[q] = dlog[(int64_t)ev * kBatch * C + q];
     __syncthreads();
-    if (threadIdx.x < kBatch) {
-        const int k = threadIdx.x;
-        const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
-        float m = logit[k * C];
-        for (int c = 1; c < C; ++c) m = fmaxf(m, logit[k * C + c]);
-        float den = 0.f;
-        for (int c = 0; c < C; ++c) den += expf(logit[k * C + c] - m);
-        for (int c = 0; c < C; ++c) {
-            const float d = (expf(logit[k * C + c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)kBatch;
-            dl[k * C + c] = d;
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < C) {
+    if (blockIdx.x == 0 && threadIdx.x < C) {
         float s = 0.f;
         for (int k = 0; k < kBatch; ++k) s += dl[k * C + threadIdx.x];
         g[ob2 + threadIdx.x] = s + l2 * x[row + ob2 + threadIdx.x];
     }
-    for (int j = threadIdx.x; j < H; j += blockDim.x) {
-        float w2[16], gw2[16];
+    const int j = blockIdx.x * 128 + threadIdx.x;
+    float w2[16], gw2[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
-        float gb1 = 0.f;
-        __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch;
-        for (int k0 = 0; k0 < kBatch; k0 += 8) {
-            __align__(16) __nv_bfloat16 pack[8];
+    for (int c = 0; c < 16; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
+    float gb1 = 0.f;
+    __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch;
+    for (int k0 = 0; k0 < kBatch; k0 += 8) {
+        __align__(16) __nv_bfloat16 pack[8];
+        float hv[8];
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const int k = k0 + kk;
-                const float hv = h[(int64_t)k * H + j];
-                float dh = 0.f;
+        for (int kk = 0; kk < 8; ++kk) hv[kk] = h[(int64_t)(k0 + kk) * H + j];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) if (c < C) dh = fmaf(dl[k * C + c], w2[c], dh);
-                const float dp = hv > 0.f ? dh : 0.f;
-                gb1 += dp;
-                pack[kk] = __float2bfloat16_rn(dp);
+        for (int kk = 0; kk < 8; ++kk) {
+            const int k = k0 + kk;
+            float dh = 0.f;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) if (c < C) gw2[c] = fmaf(dl[k * C + c], hv, gw2[c]);
-            }
-            *reinterpret_cast<uint4*>(drow + k0) = *reinterpret_cast<const uint4*>(pack);
+            for (int c = 0; c < 16; ++c) if (c < C) dh = fmaf(dl[k * C + c], w2[c], dh);
+            const float dp = hv[kk] > 0.f ? dh : 0.f;
+            gb1 += dp;
+            pack[kk] = __float2bfloat16_rn(dp);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) if (c < C) gw2[c] = fmaf(dl[k * C + c], hv[kk], gw2[c]);
         }
-        g[(int64_t)H * F + j] = gb1 + l2 * x[row + (int64_t)H * F + j];
-#pragma unroll
-        for (int c = 0; c < 16; ++c)
-            if (c < C) g[oW2 + (int64_t)c * H + j] = gw2[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
+        *reinterpret_cast<uint4*>(drow + k0) = *reinterpret_cast<const uint4*>(pack);
     }
+    g[(int64_t)H * F + j] = gb1 + l2 * x[row + (int64_t)H * F + j];
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        if (c < C) g[oW2 + (int64_t)c * H + j] = gw2[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
 }
 
 // One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A).
@@ -387,12 +384,14 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
     uint8_t* sB = smem + kABytes;                          // [NT][64] bf16 tile of A^T
     __shared__ uint64_t ab_full, acc_full;
     __shared__ uint32_t tmem_base;
+    __shared__ volatile int aborted;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ev = blockIdx.z, h0 = blockIdx.x * kMTile, f0 = blockIdx.y * NT;
     const EvDesc e = evs[ev];
     if (threadIdx.x == 0) {
         mbar_init(&ab_full, 1);
         mbar_init(&acc_full, 1);
+        aborted = 0;
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&tmem_base, 128);
@@ -418,6 +417,8 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
             umma_commit(&acc_full);
         } else {
             atomicExch(status, kErrMma);
+            aborted = 1;
+            __threadfence_block();
             mbar_arrive(&acc_full);
         }
     } else if (warp >= 2) {                                // ---- epilogue: TMEM -> global
@@ -429,7 +430,7 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
         const bool ok = mbar_wait(&acc_full, 0);
         tc_fence_after();
         if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
-        else if (atomicAdd(status, 0) == kErrNone) {
+        else if (!aborted) {
             for (int c0 = 0; c0 < NT; c0 += 16) {
                 float v[16];
                 tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
@@ -515,6 +516,7 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
               alloc(&p->AbT, (size_t)max_events * F * kBatch) &&
               alloc(&p->dpqT, (size_t)max_events * H * kBatch) &&
               cudaMalloc((void**)&p->hf, (size_t)max_events * kBatch * H * sizeof(float)) == cudaSuccess &&
+              cudaMalloc((void**)&p->dlog, (size_t)max_events * kBatch * 16 * sizeof(float)) == cudaSuccess &&
               cudaMalloc((void**)&p->status, sizeof(int)) == cudaSuccess;
     if (!ok) { mlp_plan_destroy(p); err = "MLP: device allocation failed"; return RFAST_ENOMEM; }
     cudaMemsetAsync(p->status, 0, sizeof(int), st);
@@ -551,7 +553,7 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
 
 void mlp_plan_destroy(MlpPlan* p) {
     if (!p) return;
-    void* ptrs[] = {p->featb, p->Ab, p->AbT, p->hf, p->dpqT, p->status};
+    void* ptrs[] = {p->featb, p->Ab, p->AbT, p->hf, p->dlog, p->dpqT, p->status};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete p;
 }
@@ -562,11 +564,13 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
     k_mlp_gather<<<dim3(p->Fp / kKBlock, n_events), 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
     k_mlp_fwd<<<dim3(p->H / kMTile, n_events), kGemmThreads, kFwdSmem, st>>>(
         p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
-    k_mlp_mid<<<n_events, 512, 2 * kBatch * p->C * sizeof(float), st>>>(
-        g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dpqT, g.gbuf, g.gplane, p->rows, p->F, p->H, p->C, g.l2);
+    k_mlp_logits<<<dim3(kBatch / 8, n_events), 256, 0, st>>>(
+        g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dlog, p->rows, p->F, p->H, p->C);
+    k_mlp_back<<<dim3(p->H / 128, n_events), 128, kBatch * p->C * sizeof(float), st>>>(
+        g.ev, g.x, g.stride, p->hf, p->dlog, p->dpqT, g.gbuf, g.gplane, p->F, p->H, p->C, g.l2);
     k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
         p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);
-    *launches += 4;
+    *launches += 5;
     return RFAST_OK;
 }
 

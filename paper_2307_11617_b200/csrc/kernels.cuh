@@ -485,35 +485,100 @@ k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restri
     }
 }
 
-// Sparse logistic regression, phase 2: g += sum_k coef_k a_k on top of the dense term l2 * x
-// that is already in the gradient row.  One CTA per activation; the sampled rows are added one
-// after the other (a barrier in between keeps the order fixed, so repeated columns add up in
-// batch order on every run), the entries of one row land on distinct coordinates.
-// grid = events
-__global__ void __launch_bounds__(256)
-k_logit_scatter(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col,
-                const float* __restrict__ sp_val, const float* __restrict__ coef) {
-    const EvDesc e = g.ev[blockIdx.x];
-    float* out = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + (int64_t)e.node * g.stride;
-    for (int k = 0; k < g.B; ++k) {
-        const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
-        const int64_t r = (int64_t)e.node * g.rows + rrow;
-        const float ck = coef[(int64_t)blockIdx.x * g.B + k];
-        for (int64_t q = sp_ptr[r] + threadIdx.x; q < sp_ptr[r + 1]; q += 256) {
-            const int c = sp_col[q];
-            out[c] = fmaf(ck, sp_val[q], out[c]);
+// Sparse logistic regression, phase 2, fused with S2b/S2c.  A CTA owns a tile of kLogitTile
+// coordinates of one activation: it forms g = l2 x + sum_k coef_k a_k for the tile in shared
+// memory (the sampled rows are added one after the other, so repeated columns add up in batch
+// order on every run; the entries of one row land on distinct coordinates), stores it as the
+// new remembered gradient and, unless init_only, runs the tracking update on the tile, 1024
+// coordinates at a time.
+// tile_ptr[r][t] = index of the first entry of shard row r with column >= t * kLogitTile
+// (computed once per problem on the host), so no search is needed here.
+// grid = (tiles, events), 256 threads
+constexpr int kLogitSub = 4;                               // passes of kThreads float4 per tile
+constexpr int kLogitTile = kLogitSub * 4 * kThreads;
+template <bool COMP>
+__global__ void __launch_bounds__(kThreads)
+k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int ntiles,
+              const int* __restrict__ sp_col, const float* __restrict__ sp_val,
+              const float* __restrict__ coef, int init_only) {
+    constexpr int kStage = 2048;           // staged entries per pass (about 40 per row and tile are typical)
+    __shared__ float tile[kLogitTile];
+    __shared__ int64_t lo_s[64];
+    __shared__ int cnt_s[64], pref_s[65];
+    __shared__ float ck_s[64];
+    __shared__ int st_col[kStage];
+    __shared__ float st_val[kStage];
+    const EvDesc e = g.ev[blockIdx.y];
+    const int64_t row = (int64_t)e.node * g.stride;
+    const int64_t c0 = (int64_t)blockIdx.x * kLogitTile;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int sub = 0; sub < kLogitSub; ++sub) {
+        const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
+        float4 xv = make_float4(0, 0, 0, 0);
+        if (i4 < a.n4) xv = reinterpret_cast<const float4*>(g.x + row)[i4];
+        reinterpret_cast<float4*>(tile)[sub * kThreads + threadIdx.x] = f4_scale(g.l2, xv);
+    }
+    for (int k0 = 0; k0 < g.B; k0 += 64) {                       // up to 64 sampled rows per pass
+        const int nb = min(64, g.B - k0);
+        __syncthreads();
+        if (threadIdx.x < nb) {
+            const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k0 + threadIdx.x];
+            const int64_t r = (int64_t)e.node * g.rows + rrow;
+            const int64_t lo = tile_ptr[r * (ntiles + 1) + blockIdx.x];
+            lo_s[threadIdx.x] = lo;
+            cnt_s[threadIdx.x] = (int)(tile_ptr[r * (ntiles + 1) + blockIdx.x + 1] - lo);
+            ck_s[threadIdx.x] = coef[(int64_t)blockIdx.y * g.B + k0 + threadIdx.x];
         }
         __syncthreads();
+        if (threadIdx.x <= nb) {
+            int s = 0;
+            for (int u = 0; u < threadIdx.x; ++u) s += cnt_s[u];
+            pref_s[threadIdx.x] = s;
+        }
+        __syncthreads();
+        const int total = pref_s[nb];
+        if (total <= kStage) {
+            // all entries of this tile are fetched at once (one memory latency), then one warp
+            // adds them row after row so that the order of additions is the same on every run
+            for (int t = threadIdx.x; t < total; t += kThreads) {
+                int k = 0;
+                while (pref_s[k + 1] <= t) ++k;
+                const int64_t q = lo_s[k] + (t - pref_s[k]);
+                st_col[t] = sp_col[q] - (int)c0;
+                st_val[t] = ck_s[k] * sp_val[q];
+            }
+            __syncthreads();
+            if (warp == 0)
+                for (int k = 0; k < nb; ++k) {
+                    for (int t = pref_s[k] + lane; t < pref_s[k + 1]; t += 32) tile[st_col[t]] += st_val[t];
+                    __syncwarp();
+                }
+        } else {
+            for (int k = 0; k < nb; ++k) {
+                for (int64_t q = lo_s[k] + threadIdx.x; q < lo_s[k] + cnt_s[k]; q += kThreads) {
+                    const int c = sp_col[q] - (int)c0;
+                    tile[c] += ck_s[k] * sp_val[q];
+                }
+                __syncthreads();
+            }
+        }
     }
-}
-
-// g = l2 * x for every node (start of the initial gradients of the sparse objective).  grid = (tiles, n)
-__global__ void __launch_bounds__(kThreads)
-k_scale_rows(const float* __restrict__ x, float* __restrict__ out, int64_t stride, int n4, float l2) {
-    const int i4 = blockIdx.x * kThreads + threadIdx.x;
-    if (i4 >= n4) return;
-    const int64_t row = (int64_t)blockIdx.y * stride;
-    reinterpret_cast<float4*>(out + row)[i4] = f4_scale(l2, reinterpret_cast<const float4*>(x + row)[i4]);
+    __syncthreads();
+    float* zr = a.z + row;
+    const float* gold = g.gbuf + (int64_t)e.g_par * g.gplane + row;
+    float* gnew = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row;
+    for (int sub = 0; sub < kLogitSub; ++sub) {
+        const int base = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
+        if (base >= a.n4) break;
+        float4 zh[1], gnv[1], gov[1];
+        gnv[0] = reinterpret_cast<const float4*>(tile)[sub * kThreads + threadIdx.x];
+        reinterpret_cast<float4*>(gnew)[base] = gnv[0];
+        if (init_only) continue;
+        zh[0] = ld_stream(zr, base);
+        gov[0] = ld_stream(gold, base);
+        track_and_push<1, COMP>(a, e, base, zr, zh, gnv, gov);
+    }
 }
 
 // row copy helpers ----------------------------------------------------------------------------

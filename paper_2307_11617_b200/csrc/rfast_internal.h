@@ -74,7 +74,7 @@ struct GradArgs {
 struct ModelTraffic {
     bool elementwise = false;   // one fused pass, gradient recomputed instead of stored
     int  data_streams = 0;      // model data streams per coordinate in the fused pass
-    bool bf16_copy = false;     // the mix pass also writes a bf16 copy of x (counts as half a stream: rounded up per event pair)
+    int  grad_track_streams = 5; // split path: gradient reads x, writes g; tracking reads z, g_old, g_new
 };
 
 int build_host_graph(const rfast_graph& g, int n, bool row_stochastic, HostGraph& out, std::string& err);
