@@ -121,6 +121,9 @@ typedef struct rfast_schedule {
     const int8_t*  send_c;      /* [n_send_c] */
     int64_t        n_batch_idx;
     const int32_t* batch_idx;   /* [(n + events) * B] */
+    const float*   alpha_round; /* [K] step size gamma^r of every activation of round r (the paper    */
+                                /* allows a time-varying gamma^t, Algorithm 1 S1 / Algorithm 2 S.1),  */
+                                /* or NULL: the problem's constant alpha                              */
 } rfast_schedule;
 
 /* Views for rfast_read_state.  Float views are fp32 row-major, unpadded. */

@@ -205,7 +205,10 @@ def run_schedule(orc: RFastOracle, sch, K=None, after_round=None):
     for ev in range(ev0):
         pr += outdeg_r[int(sch.act_node[ev])]
         pc += outdeg_c[int(sch.act_node[ev])]
+    alpha_round = getattr(sch, "alpha_round", None)
     for r in range(orc.round, K):
+        if alpha_round is not None:          # time-varying step size gamma^r (Algorithm 2, S.1)
+            orc.alpha = float(alpha_round[r])
         for ev in range(int(sch.act_ptr[r]), int(sch.act_ptr[r + 1])):
             i = int(sch.act_node[ev])
             cr = sch.send_r[pr:pr + outdeg_r[i]]

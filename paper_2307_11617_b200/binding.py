@@ -52,7 +52,8 @@ class _Problem(C.Structure):
 class _Schedule(C.Structure):
     _fields_ = [("K", C.c_int32), ("act_ptr", C.c_void_p), ("act_node", C.c_void_p),
                 ("n_send_r", C.c_int64), ("send_r", C.c_void_p), ("n_send_c", C.c_int64),
-                ("send_c", C.c_void_p), ("n_batch_idx", C.c_int64), ("batch_idx", C.c_void_p)]
+                ("send_c", C.c_void_p), ("n_batch_idx", C.c_int64), ("batch_idx", C.c_void_p),
+                ("alpha_round", C.c_void_p)]
 
 
 _lib = None
@@ -142,6 +143,12 @@ def _schedule(s, keep):
     S.n_send_r, S.send_r = len(send_r), _ptr(send_r)
     S.n_send_c, S.send_c = len(send_c), _ptr(send_c)
     S.n_batch_idx, S.batch_idx = len(bidx), _ptr(bidx)
+    if getattr(s, "alpha_round", None) is not None:
+        ar = _arr(s.alpha_round, np.float32)
+        if len(ar) != int(s.K):
+            raise ValueError("alpha_round must hold one step size per round")
+        keep.append(ar)
+        S.alpha_round = _ptr(ar)
     return S
 
 

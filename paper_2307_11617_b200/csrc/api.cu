@@ -54,6 +54,7 @@ struct rfast_ctx {
         *d_out_new = nullptr, *d_batch_idx = nullptr;
     float *d_mix_w = nullptr, *d_out_a = nullptr;
     std::vector<void*> sched_allocs;
+    std::vector<float> alpha_round;         // per-round step size, empty: constant alpha
     int max_round_events = 0;
     int round = 0;
     int64_t launches = 0;
@@ -415,6 +416,12 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated), comp, err);
     if (rc != RFAST_OK) return set_err(ctx, rc, err);
     free_schedule(ctx);
+    ctx->alpha_round.clear();
+    if (s->alpha_round) {
+        for (int r = 0; r < s->K; ++r)
+            if (!(s->alpha_round[r] == s->alpha_round[r])) return set_err(ctx, RFAST_ESCHED, "schedule: alpha_round holds a NaN");
+        ctx->alpha_round.assign(s->alpha_round, s->alpha_round + s->K);
+    }
     ctx->comp = std::move(comp);
     Compiled& c = ctx->comp;
     ctx->max_round_events = 0;
@@ -478,6 +485,7 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
         const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
         if (nev == 0) continue;
         a.ev = ctx->d_ev + c.act_ptr[r];
+        if (!ctx->alpha_round.empty()) a.alpha = ctx->alpha_round[r];
         if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
             if (ctx->compensated) k_fused_quad<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             else if (big) k_fused_quad<2, false><<<tile_grid(a.n4, 2, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);

@@ -137,6 +137,25 @@ def test_conservation_on_the_device_state(rfast_lib):
     assert np.abs(res).max() <= 1e-5 * scale
 
 
+@pytest.mark.parametrize("name,ov", [("quad_tree64", dict(n=16, p=3000, K=40)),
+                                     ("softmax_exp16", dict(F=40, C=5, rows=32, K=60, batch=8))],
+                         ids=["quad", "softmax"])
+def test_time_varying_step_size(rfast_lib, name, ov):
+    """A per-round step size (step decay, as in the paper's ResNet schedule) on both sides."""
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=6, **ov)
+    K = wl.schedule.K
+    wl.schedule.alpha_round = (0.02 * 0.1 ** (np.arange(K) // (K // 3 + 1))).astype(np.float32)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+    wl.schedule.alpha_round = None                 # and it really was used
+    orc2, _ = _oracle(wl)
+    assert rel_l2(orc2.X(), orc.X()) > 1e-3
+
+
 def test_run_past_the_schedule_is_refused(rfast_lib):
     import paper_2307_11617_b200 as pkg
     from paper_2307_11617_b200.binding import ESTATE, RFastError

@@ -325,3 +325,20 @@ def test_augmented_systems_dense(seed):
         assert np.abs(mass - M).max() < 1e-12
         assert np.abs(zhat.sum(axis=0) - np.stack(
             [grad(q, h[q]) for q in range(n)]).sum(axis=0)).max() < 1e-12   # Lemma 3 on the dense system
+
+
+def test_time_varying_step_size_single_node():
+    """gamma^t of Algorithm 1 S1 varying per round: n = 1 is gradient descent with that step sequence."""
+    rng = _rng(21)
+    p, rows, K = 5, 12, 30
+    G_R = graph_from_edges(1, [], "row"); G_C = graph_from_edges(1, [], "col")
+    feat = rng.standard_normal((1, rows, p)); target = rng.standard_normal((1, rows))
+    x0 = rng.standard_normal((1, p))
+    sch = make_schedule(G_R, G_C, activation_all(1, K), 0.0, 0, rng)
+    sch.alpha_round = (0.1 * 0.5 ** (np.arange(K) // 10)).astype(np.float32)     # step decay
+    orc = RFastOracle(1, p, 123.0, G_R, G_C, LeastSquares(feat, target).grad, x0=x0)
+    run_schedule(orc, sch)
+    x = x0[0].copy()
+    for t in range(K):
+        x = x - float(sch.alpha_round[t]) * (feat[0].T @ (feat[0] @ x - target[0]) / rows)
+    assert np.abs(orc.X()[0] - x).max() < 1e-13

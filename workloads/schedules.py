@@ -29,6 +29,7 @@ class Schedule:
     send_c: np.ndarray       # int8, same for G_C
     batch: int               # B, 0 when the model takes no minibatch
     batch_idx: np.ndarray    # int32 [(n + E_ev) * B]; first n*B entries: the initial samples
+    alpha_round: np.ndarray | None = None   # float32 [K] step size per round, or None (constant)
 
     @property
     def n_events(self) -> int:
