@@ -194,6 +194,28 @@ int64_t rfast_query(rfast_ctx* ctx, int what);
 /* Waits for the handle's stream; reports a pending asynchronous error. */
 int rfast_sync(rfast_ctx* ctx);
 
+/* Checkpoint / resume.  The blob holds the complete device state of the handle -- x, the
+ * trackers, the remembered gradients, every live packet version (published v and running sums
+ * rho, i.e. also the packets still in flight) and the round counter -- so that
+ *     create + load_schedule(same schedule) + checkpoint_load + run(K - r)
+ * continues bit for bit where  run(r) + checkpoint_save  stopped.  The blob is opaque and tied
+ * to the problem's shape and to the loaded schedule (a hash of its arrays is checked);
+ * RFAST_ESTATE if no schedule is loaded, RFAST_EINVAL on a size or identity mismatch.
+ * dst / src are caller-owned HOST buffers of rfast_checkpoint_size() bytes. */
+int64_t rfast_checkpoint_size(rfast_ctx* ctx);
+int     rfast_checkpoint_save(rfast_ctx* ctx, void* dst, size_t bytes);
+int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
+
+/* On-device diagnostics of the current state (off the hot path; reads every state row once):
+ *   out[0] consensus error  || x - 1 xbar^T ||_F        (xbar = mean of the x_i)
+ *   out[1] || xbar ||_2
+ *   out[2] conservation residual of Lemma 3:
+ *          max_c | sum_i z_i + sum_e (rho_e - rho~_e) - sum_i g_i |   (0 up to rounding)
+ *   out[3] max_c | sum_i g_i |   (the scale of out[2])
+ *   out[4] || z ||_F
+ * n_out must be 5 (RFAST_EINVAL otherwise); out is a caller-owned HOST array of doubles. */
+int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out);
+
 /* Host-only companion of rfast_load_schedule (needs no CUDA device): compiles the schedule
  * for the two graphs of `prob` (only n, root, batch, rows, model, G_R, G_C are read) and
  * writes the integer artefacts into caller-owned HOST arrays, any of which may be NULL:

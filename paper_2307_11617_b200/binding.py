@@ -82,6 +82,11 @@ def lib():
         L.rfast_version.restype = C.c_char_p
         L.rfast_compile_host.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule)] + [C.c_void_p] * 5 + \
             [C.c_char_p, C.c_size_t]
+        L.rfast_checkpoint_size.argtypes = [C.c_void_p]
+        L.rfast_checkpoint_size.restype = C.c_int64
+        L.rfast_checkpoint_save.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+        L.rfast_checkpoint_load.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+        L.rfast_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.rfast_ls_gradient_static.argtypes = [C.c_void_p] * 4 + [C.c_int32, C.c_int32, C.c_float,
                                                C.c_void_p, C.c_char_p, C.c_size_t]
         _lib = L
@@ -232,6 +237,30 @@ def rfast_compile_host(wl, s):
             "streams": int(counts[3])}
 
 
+def rfast_checkpoint_save(handle) -> np.ndarray:
+    """The handle's complete state as an opaque byte array (see rfast_checkpoint_save in rfast.h)."""
+    size = lib().rfast_checkpoint_size(handle)
+    if size < 0:
+        _check(int(size), handle)
+    blob = np.empty(size, dtype=np.uint8)
+    _check(lib().rfast_checkpoint_save(handle, _ptr(blob), blob.nbytes), handle)
+    return blob
+
+
+def rfast_checkpoint_load(handle, blob: np.ndarray) -> None:
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    _check(lib().rfast_checkpoint_load(handle, _ptr(blob), blob.nbytes), handle)
+
+
+def rfast_diagnostics(handle) -> dict:
+    """Consensus error, norm of the mean iterate, conservation residual (Lemma 3) and its scale,
+    tracker norm, all computed on the device."""
+    out = np.zeros(5, dtype=np.float64)
+    _check(lib().rfast_diagnostics(handle, _ptr(out), 5), handle)
+    return {"consensus_error": out[0], "xbar_norm": out[1], "conservation_residual": out[2],
+            "gradient_sum_max": out[3], "tracker_norm": out[4]}
+
+
 STATIC_MAX_ROWS = 65536
 
 
@@ -288,6 +317,15 @@ class Engine:
         if which == STATE_USED_TAU_RHO:
             shape = (self.query(Q_N_USED_TAU_RHO),)
         return rfast_read_state(self.h, which, shape, out)
+
+    def checkpoint(self):
+        return rfast_checkpoint_save(self.h)
+
+    def restore(self, blob):
+        rfast_checkpoint_load(self.h, blob)
+
+    def diagnostics(self):
+        return rfast_diagnostics(self.h)
 
     def close(self):
         if self.h:

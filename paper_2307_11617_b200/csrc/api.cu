@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -55,6 +56,7 @@ struct rfast_ctx {
     float *d_mix_w = nullptr, *d_out_a = nullptr;
     std::vector<void*> sched_allocs;
     std::vector<float> alpha_round;         // per-round step size, empty: constant alpha
+    uint64_t sched_hash = 0;                // identity of the loaded schedule (checkpoints)
     int max_round_events = 0;
     int round = 0;
     int64_t launches = 0;
@@ -422,6 +424,21 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
             if (!(s->alpha_round[r] == s->alpha_round[r])) return set_err(ctx, RFAST_ESCHED, "schedule: alpha_round holds a NaN");
         ctx->alpha_round.assign(s->alpha_round, s->alpha_round + s->K);
     }
+    {   // FNV-1a over the raw arrays: a checkpoint is only valid for this very schedule
+        uint64_t hsh = 1469598103934665603ull;
+        auto mix = [&](const void* ptr, size_t bytes) {
+            const unsigned char* q = (const unsigned char*)ptr;
+            for (size_t k = 0; k < bytes; ++k) { hsh ^= q[k]; hsh *= 1099511628211ull; }
+        };
+        mix(&s->K, sizeof s->K);
+        mix(s->act_ptr, (size_t)(s->K + 1) * sizeof(int32_t));
+        if (s->act_ptr[s->K] > 0) mix(s->act_node, (size_t)s->act_ptr[s->K] * sizeof(int32_t));
+        if (s->n_send_r > 0) mix(s->send_r, (size_t)s->n_send_r);
+        if (s->n_send_c > 0) mix(s->send_c, (size_t)s->n_send_c);
+        if (ctx->batch > 0) mix(s->batch_idx, (size_t)s->n_batch_idx * sizeof(int32_t));
+        if (s->alpha_round) mix(s->alpha_round, (size_t)s->K * sizeof(float));
+        ctx->sched_hash = hsh;
+    }
     ctx->comp = std::move(comp);
     Compiled& c = ctx->comp;
     ctx->max_round_events = 0;
@@ -701,6 +718,140 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32
 } catch (...) {
     if (errbuf && err_len) std::snprintf(errbuf, err_len, "host allocation failed");
     return RFAST_ENOMEM;
+}
+
+}  // extern "C"
+
+namespace {
+
+struct CkptHeader {
+    uint64_t magic, sched_hash;
+    int64_t  p, stride, n_events;
+    int32_t  n, model, compensated, K, n_v_slots, n_rho_slots, round, pad;
+};
+constexpr uint64_t kCkptMagic = 0x5246415354434B31ull;   // "RFASTCK1"
+
+// the device buffers that make up the state, in blob order
+std::vector<std::pair<void*, size_t>> state_buffers(rfast_ctx* c) {
+    const size_t plane = (size_t)c->n * c->stride * sizeof(float);
+    std::vector<std::pair<void*, size_t>> v;
+    v.push_back({c->x, plane});
+    v.push_back({c->z, plane});
+    if (c->zc) v.push_back({c->zc, plane});
+    if (c->gbuf) v.push_back({c->gbuf, 2 * plane});
+    if (c->xb) v.push_back({c->xb, plane / 2});
+    v.push_back({c->vbuf, (size_t)c->comp.n_v_slots * c->stride * sizeof(float)});
+    v.push_back({c->rbuf, (size_t)c->comp.n_rho_slots * c->stride * sizeof(float)});
+    return v;
+}
+
+CkptHeader make_header(rfast_ctx* c) {
+    CkptHeader h{};
+    h.magic = kCkptMagic; h.sched_hash = c->sched_hash;
+    h.p = c->p; h.stride = c->stride; h.n_events = c->comp.n_events;
+    h.n = c->n; h.model = c->model; h.compensated = c->compensated; h.K = c->comp.K;
+    h.n_v_slots = c->comp.n_v_slots; h.n_rho_slots = c->comp.n_rho_slots; h.round = c->round;
+    return h;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t rfast_checkpoint_size(rfast_ctx* ctx) {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    size_t total = sizeof(CkptHeader);
+    for (auto& b : state_buffers(ctx)) total += b.second;
+    return (int64_t)total;
+}
+
+int rfast_checkpoint_save(rfast_ctx* ctx, void* dst, size_t bytes) {
+    if (!ctx || !dst) return RFAST_EINVAL;
+    const int64_t need = rfast_checkpoint_size(ctx);
+    if (need < 0) return (int)need;
+    if ((size_t)need != bytes) return set_err(ctx, RFAST_EINVAL, "checkpoint_save: size mismatch");
+    int rc = check_device_status(ctx);
+    if (rc != RFAST_OK) return rc;
+    CkptHeader h = make_header(ctx);
+    std::memcpy(dst, &h, sizeof h);
+    char* q = (char*)dst + sizeof h;
+    for (auto& b : state_buffers(ctx)) {
+        if (b.second) CK(cudaMemcpyAsync(q, b.first, b.second, cudaMemcpyDeviceToHost, ctx->stream));
+        q += b.second;
+    }
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
+int rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes) {
+    if (!ctx || !src) return RFAST_EINVAL;
+    const int64_t need = rfast_checkpoint_size(ctx);
+    if (need < 0) return (int)need;
+    if ((size_t)need != bytes) return set_err(ctx, RFAST_EINVAL, "checkpoint_load: size mismatch");
+    CkptHeader h;
+    std::memcpy(&h, src, sizeof h);
+    CkptHeader mine = make_header(ctx);
+    mine.round = h.round;
+    if (std::memcmp(&h, &mine, sizeof h) != 0 || h.round < 0 || h.round > ctx->comp.K)
+        return set_err(ctx, RFAST_EINVAL, "checkpoint_load: blob belongs to another problem or schedule");
+    const char* q = (const char*)src + sizeof h;
+    for (auto& b : state_buffers(ctx)) {
+        if (b.second) CK(cudaMemcpyAsync(b.first, q, b.second, cudaMemcpyHostToDevice, ctx->stream));
+        q += b.second;
+    }
+    CK(cudaStreamSynchronize(ctx->stream));
+    ctx->round = h.round;
+    return RFAST_OK;
+}
+
+int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
+    if (!ctx || !out || n_out != 5) return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5") : RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    const Compiled& c = ctx->comp;
+    const int n = ctx->n, E = ctx->Cg.E;
+    // which rows hold the current g, the latest rho and the buffered rho of every edge
+    std::vector<int> gsel(n), latest(std::max(E, 1), -1), buf(std::max(E, 1), -1), t(n, 0);
+    const int ev_end = c.act_ptr[ctx->round];
+    for (int ev = 0; ev < ev_end; ++ev) {
+        const EvDesc& d = c.ev[ev];
+        t[d.node]++;
+        for (int k = 0; k < d.out_cnt; ++k) latest[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
+        for (int k = 0; k < d.news_cnt; ++k) buf[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
+    }
+    for (int i = 0; i < n; ++i) gsel[i] = (t[i] & 1) * n + i;
+    const int blocks = (int)((ctx->p + kThreads - 1) / kThreads);
+    int *d_gsel = nullptr, *d_latest = nullptr, *d_buf = nullptr;
+    double* d_part = nullptr;
+    auto cleanup = [&]() { cudaFree(d_gsel); cudaFree(d_latest); cudaFree(d_buf); cudaFree(d_part); };
+    if (cudaMalloc((void**)&d_gsel, n * sizeof(int)) != cudaSuccess ||
+        cudaMalloc((void**)&d_latest, latest.size() * sizeof(int)) != cudaSuccess ||
+        cudaMalloc((void**)&d_buf, buf.size() * sizeof(int)) != cudaSuccess ||
+        cudaMalloc((void**)&d_part, (size_t)blocks * 5 * sizeof(double)) != cudaSuccess) {
+        cleanup();
+        return set_err(ctx, RFAST_ENOMEM, "diagnostics: temporary allocation failed");
+    }
+    cudaMemcpyAsync(d_gsel, gsel.data(), n * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
+    cudaMemcpyAsync(d_latest, latest.data(), latest.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
+    cudaMemcpyAsync(d_buf, buf.data(), buf.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
+    k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
+                                                          ctx->quad_b, ctx->rbuf, d_latest, d_buf, n, E,
+                                                          ctx->stride, ctx->p, d_part);
+    std::vector<double> part((size_t)blocks * 5);
+    cudaError_t e = cudaMemcpyAsync(part.data(), d_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    cleanup();
+    if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("diagnostics: ") + cudaGetErrorString(e));
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0;
+    for (int b = 0; b < blocks; ++b) {          // fixed order: the same bits on every run
+        cons += part[(size_t)b * 5]; xb2 += part[(size_t)b * 5 + 1];
+        res = std::max(res, part[(size_t)b * 5 + 2]); gs = std::max(gs, part[(size_t)b * 5 + 3]);
+        z2 += part[(size_t)b * 5 + 4];
+    }
+    out[0] = std::sqrt(std::max(cons, 0.0)); out[1] = std::sqrt(xb2); out[2] = res; out[3] = gs; out[4] = std::sqrt(z2);
+    return RFAST_OK;
+} catch (...) {
+    return set_err(ctx, RFAST_ENOMEM, "diagnostics: host allocation failed");
 }
 
 }  // extern "C"

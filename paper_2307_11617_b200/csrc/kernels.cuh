@@ -594,6 +594,62 @@ k_gather_rows(const float* __restrict__ src, const int* __restrict__ idx, float*
     reinterpret_cast<float4*>(dst + (int64_t)blockIdx.y * dst_stride)[i4] = v;
 }
 
+// Diagnostics: per coordinate, sums over nodes and edges; per block, partial results.
+//   part[block][0] = sum_c (sum_i x_ic^2 - n xbar_c^2)    (consensus error squared)
+//   part[block][1] = sum_c xbar_c^2
+//   part[block][2] = max_c | sum_i z_ic + sum_e (rho_ec - rho~_ec) - sum_i g_ic |
+//   part[block][3] = max_c | sum_i g_ic |
+//   part[block][4] = sum_c sum_i z_ic^2
+// g_i is row gsel[i] of gpool (or recomputed for the element-wise objective when gpool is null).
+// grid = tiles of kThreads coordinates (scalar: diagnostics favour clarity over speed)
+__global__ void __launch_bounds__(kThreads)
+k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const float* __restrict__ zc,
+              const float* __restrict__ gpool, const int* __restrict__ gsel,
+              const float* __restrict__ qd, const float* __restrict__ qb,
+              const float* __restrict__ rbuf, const int* __restrict__ rho_latest,
+              const int* __restrict__ rho_buf, int n, int n_edges, int64_t stride, int64_t p,
+              double* __restrict__ part) {
+    __shared__ double red[5][kThreads];
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0;
+    if (c < p) {
+        double sx = 0, sx2 = 0, sz = 0, sg = 0;
+        for (int i = 0; i < n; ++i) {
+            const double xv = x[(int64_t)i * stride + c];
+            double zv = z[(int64_t)i * stride + c];
+            if (zc) zv += (double)zc[(int64_t)i * stride + c];
+            double gv;
+            if (gpool) gv = gpool[(int64_t)gsel[i] * stride + c];
+            else { const float d = qd[(int64_t)i * stride + c]; gv = d * d * ((float)xv - qb[(int64_t)i * stride + c]); }
+            sx += xv; sx2 += xv * xv; sz += zv; sg += gv; z2 += zv * zv;
+        }
+        double mass = 0;
+        for (int e = 0; e < n_edges; ++e) {
+            if (rho_latest[e] >= 0) mass += (double)rbuf[(int64_t)rho_latest[e] * stride + c];
+            if (rho_buf[e] >= 0) mass -= (double)rbuf[(int64_t)rho_buf[e] * stride + c];
+        }
+        const double xbar = sx / n;
+        cons = sx2 - n * xbar * xbar;
+        xb2 = xbar * xbar;
+        res = fabs(sz + mass - sg);
+        gs = fabs(sg);
+    }
+    red[0][threadIdx.x] = cons; red[1][threadIdx.x] = xb2; red[2][threadIdx.x] = res;
+    red[3][threadIdx.x] = gs; red[4][threadIdx.x] = z2;
+    __syncthreads();
+    for (int s = kThreads / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) {
+            red[0][threadIdx.x] += red[0][threadIdx.x + s];
+            red[1][threadIdx.x] += red[1][threadIdx.x + s];
+            red[2][threadIdx.x] = fmax(red[2][threadIdx.x], red[2][threadIdx.x + s]);
+            red[3][threadIdx.x] = fmax(red[3][threadIdx.x], red[3][threadIdx.x + s]);
+            red[4][threadIdx.x] += red[4][threadIdx.x + s];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x < 5) part[(int64_t)blockIdx.x * 5 + threadIdx.x] = red[threadIdx.x][0];
+}
+
 // bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)
 __global__ void __launch_bounds__(kThreads)
 k_rows_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int n4) {

@@ -1,0 +1,85 @@
+"""Checkpoint / resume and the on-device diagnostics (auxiliary entry points)."""
+
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from oracle import from_workload, make_model, run_schedule
+from workloads import build_config
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    ("quad_tree64", dict(n=16, p=3000, K=30)),
+    ("softmax_exp16", dict(F=40, C=5, rows=32, K=40, batch=8)),          # compensated tracker
+    ("logistic_tree1024", dict(n=48, p=2500, rows=8, K=30, batch=4, nnz=30)),
+    ("mlp_tree64", dict(n=5, F=64, H=128, C=4, rows=96, K=12, batch=64)),
+]
+
+
+@pytest.mark.parametrize("name,ov", CASES, ids=[c[0] for c in CASES])
+def test_resume_from_checkpoint_is_bit_identical(rfast_lib, name, ov):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config(name, seed=8, **ov)
+    K, r = wl.schedule.K, wl.schedule.K // 3
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run(r)
+        blob = eng.checkpoint()
+        eng.run(K - r)
+        x1, y1, g1 = eng.read(B.STATE_X), eng.read(B.STATE_Y), eng.read(B.STATE_G_LAST)
+        rl1 = eng.read(B.STATE_RHO_LATEST)
+    with pkg.Engine(wl) as eng:                      # a fresh handle, as after a restart
+        eng.load_schedule(wl.schedule)
+        eng.restore(blob)
+        assert eng.query(B.Q_ROUND) == r
+        eng.run(K - r)
+        assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
+        assert np.array_equal(g1, eng.read(B.STATE_G_LAST))
+        assert np.array_equal(rl1, eng.read(B.STATE_RHO_LATEST))
+
+
+def test_checkpoint_of_another_schedule_is_refused(rfast_lib):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import EINVAL, ESTATE, RFastError
+    wl = build_config("quad_tree64", seed=8, n=8, p=100, K=10)
+    other = build_config("quad_tree64", seed=9, n=8, p=100, K=10)
+    with pkg.Engine(wl) as eng:
+        with pytest.raises(RFastError) as ei:
+            eng.checkpoint()                         # nothing loaded yet
+        assert ei.value.code == ESTATE
+        eng.load_schedule(wl.schedule)
+        eng.run(4)
+        blob = eng.checkpoint()
+        eng.load_schedule(other.schedule)
+        try:
+            eng.restore(blob)
+            raised = None
+        except RFastError as e:
+            raised = e
+        assert raised is not None and raised.code == EINVAL
+
+
+@pytest.mark.parametrize("name,ov", CASES[:3], ids=[c[0] for c in CASES[:3]])
+def test_diagnostics_match_the_oracle_state(rfast_lib, name, ov):
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=8, **ov)
+    orc = from_workload(wl, make_model(wl).grad)
+    run_schedule(orc, wl.schedule)
+    X, Z, G = orc.X(), orc.Z(), orc.G()
+    xbar = X.mean(axis=0)
+    want = {"consensus_error": np.linalg.norm(X - xbar), "xbar_norm": np.linalg.norm(xbar),
+            "gradient_sum_max": np.abs(G.sum(axis=0)).max(), "tracker_norm": np.linalg.norm(Z)}
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        d0 = eng.diagnostics()
+        assert d0["conservation_residual"] <= 1e-6 * max(d0["gradient_sum_max"], 1e-30)   # z^0 = g^0
+        eng.run()
+        d = eng.diagnostics()
+    for key, w in want.items():
+        assert abs(d[key] - w) <= 1e-4 * max(w, 1e-6), (key, d[key], w)
+    # Lemma 3 on the device state, relative to the gradients that are summed
+    scale = np.abs(G).sum(axis=0).max()
+    assert d["conservation_residual"] <= 1e-5 * scale
