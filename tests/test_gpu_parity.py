@@ -156,6 +156,22 @@ def test_time_varying_step_size(rfast_lib, name, ov):
     assert rel_l2(orc2.X(), orc.X()) > 1e-3
 
 
+def test_parity_under_acknowledgement_gated_loss(rfast_lib):
+    """The paper's own packet-loss emulation (send only after the last packet was acknowledged)."""
+    import paper_2307_11617_b200 as pkg
+    from workloads import activation_bernoulli, make_schedule_ack_gated
+    wl = build_config("quad_tree64", seed=4, n=32, p=2000, K=10)
+    rng = np.random.default_rng(4)
+    wl.schedule = make_schedule_ack_gated(wl.G_R, wl.G_C, activation_bernoulli(wl.n, 80, 0.5, rng), 4, rng)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        from paper_2307_11617_b200 import binding as B
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
+
+
 def test_run_past_the_schedule_is_refused(rfast_lib):
     import paper_2307_11617_b200 as pkg
     from paper_2307_11617_b200.binding import ESTATE, RFastError

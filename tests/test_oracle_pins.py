@@ -342,3 +342,20 @@ def test_time_varying_step_size_single_node():
     for t in range(K):
         x = x - float(sch.alpha_round[t]) * (feat[0].T @ (feat[0] @ x - target[0]) / rows)
     assert np.abs(orc.X()[0] - x).max() < 1e-13
+
+
+def test_convergence_under_acknowledgement_gated_loss():
+    """Theorem 1 (sigma = 0) with the paper's own loss emulation instead of i.i.d. drops."""
+    from workloads import make_schedule_ack_gated
+    n, p, K = 4, 3, 20000
+    feat, target, xstar, L = _ls_problem(7)
+    rng = _rng(9)
+    G_R, G_C = ring_graphs(n)
+    sch = make_schedule_ack_gated(G_R, G_C, activation_bernoulli(n, K, 0.6, rng), 3, rng)
+    assert (sch.send_c == -1).mean() > 0.2
+    # three packets in four are discarded here, which lengthens the effective delays: smaller step
+    orc = RFastOracle(n, p, 0.8 / L, G_R, G_C, LeastSquares(feat, target).grad)
+    run_schedule(orc, sch)
+    assert np.linalg.norm(orc.X() - xstar) <= 1e-8 * np.linalg.norm(xstar)
+    # the identity of Lemma 3 holds to rounding of the running sums it is made of
+    assert np.abs(orc.conservation_residual()).max() <= 1e-13 * max(1.0, np.abs(orc.RHO()).max()) * 100

@@ -82,3 +82,28 @@ def test_full_size_shapes_of_the_small_configs():
     assert (wl.n, wl.p, wl.batch) == (64, 407050, 64)
     wl = build_config("logistic_tree1024", p=1000, rows=2, K=2)
     assert wl.n == 1024 and np.bincount(wl.G_C.rowptr[1:] - wl.G_C.rowptr[:-1]).size <= 9
+
+
+def test_ack_gated_schedule_never_has_two_unacknowledged_packets():
+    """Section VI's packet-loss emulation: at most one packet per edge awaits its receiver."""
+    from workloads import activation_bernoulli, make_schedule_ack_gated, ring_graphs
+    from helpers import out_edges
+    rng = np.random.default_rng(3)
+    n, K = 6, 80
+    G_R, G_C = ring_graphs(n)
+    acts = activation_bernoulli(n, K, 0.5, rng)
+    s = make_schedule_ack_gated(G_R, G_C, acts, 3, rng)
+    assert (s.send_r == -1).any() and (s.send_r >= 0).any()
+    out = out_edges(G_R)
+    act_rounds = [[r for r in range(K) if i in acts[r]] for i in range(n)]
+    pending = {}                                    # edge -> round at which its packet gets processed
+    pos = 0
+    for r in range(K):
+        for i in acts[r]:
+            for e in out[int(i)]:
+                code = int(s.send_r[pos]); pos += 1
+                if code >= 0:
+                    assert e not in pending or pending[e] < r, "sent while the last packet was unprocessed"
+                    recv = int(np.searchsorted(G_R.rowptr, e, side="right") - 1)
+                    later = [q for q in act_rounds[recv] if q >= r + 1 + code]
+                    pending[e] = later[0] if later else K + 1

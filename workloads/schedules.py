@@ -104,6 +104,54 @@ def make_schedule(G_R: Graph, G_C: Graph, active_sets, drop: float, max_delay: i
     return Schedule(K, act_ptr, act_node, send_r, send_c, batch, batch_idx)
 
 
+def make_schedule_ack_gated(G_R: Graph, G_C: Graph, active_sets, max_delay: int,
+                            rng: np.random.Generator, batch: int = 0, rows_per_node: int = 0) -> Schedule:
+    """Packet loss as the paper emulates it (Section VI, first paragraph): a node sends a new
+    packet to an out-neighbour only once that neighbour has acknowledged the previous one, and
+    otherwise discards the packet of this activation.  Here: a packet sent in round r with
+    delay d is usable from round r+1+d; the receiver acknowledges it at its first activation
+    from then on, and the acknowledgement travels back with its own delay (same distribution).
+    Until it has arrived the sender's packets on that edge are dropped (code -1)."""
+    n = G_R.n
+    K = len(active_sets)
+    act_ptr = np.zeros(K + 1, dtype=np.int32)
+    act_ptr[1:] = np.cumsum([len(a) for a in active_sets])
+    act_node = (np.concatenate(active_sets).astype(np.int32) if K and act_ptr[-1] else np.zeros(0, np.int32))
+    act_rounds = [[] for _ in range(n)]
+    for r, a in enumerate(active_sets):
+        for i in a:
+            act_rounds[int(i)].append(r)
+    act_rounds = [np.asarray(a, dtype=np.int64) for a in act_rounds]
+
+    def codes(G):
+        optr, orecv, oeid = sender_csr(G)
+        ack_ready = np.zeros(G.n_edges, dtype=np.int64)        # round from which the edge may send again
+        out = []
+        for r, a in enumerate(active_sets):
+            for i in a:
+                for k in range(optr[i], optr[i + 1]):
+                    e, j = int(oeid[k]), int(orecv[k])
+                    if r < ack_ready[e]:
+                        out.append(-1)
+                        continue
+                    d = int(rng.integers(0, max_delay + 1))
+                    out.append(d)
+                    pos = np.searchsorted(act_rounds[j], r + 1 + d)
+                    if pos == len(act_rounds[j]):
+                        ack_ready[e] = K + 1                     # never processed within the horizon
+                    else:
+                        ack_ready[e] = int(act_rounds[j][pos]) + 1 + int(rng.integers(0, max_delay + 1))
+        return np.asarray(out, dtype=np.int8)
+
+    send_r = codes(G_R)
+    send_c = codes(G_C)
+    if batch > 0:
+        batch_idx = rng.integers(0, rows_per_node, size=(n + len(act_node)) * batch).astype(np.int32)
+    else:
+        batch_idx = np.zeros(0, np.int32)
+    return Schedule(K, act_ptr, act_node, send_r, send_c, batch, batch_idx)
+
+
 def realised_T_D(G_R: Graph, G_C: Graph, s: Schedule):
     """Realised constants of Assumption 3 in units of rounds: T = longest stretch
     of rounds in which some node stays inactive plus one; D = largest delay code."""
