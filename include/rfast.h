@@ -191,6 +191,16 @@ int rfast_reset(rfast_ctx* ctx);
 /* A counter (>= 0), or a negative status for an unknown id / NULL handle. */
 int64_t rfast_query(rfast_ctx* ctx, int what);
 
+/* Execution options (they never change results: every path produces the same bits).
+ *   RFAST_OPT_PERSISTENT  1 (default): problems whose state fits L2 (least squares, softmax
+ *                         regression) run a span of rounds as ONE cooperative persistent
+ *                         kernel with bounded grid barriers between the phases of a round;
+ *                         0: one kernel per phase.
+ *   RFAST_OPT_GRAPHS      1 (default): spans of rounds are recorded into a CUDA graph and
+ *                         replayed (non-default streams only); 0: direct launches. */
+enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1 };
+int rfast_set_option(rfast_ctx* ctx, int option, int64_t value);
+
 /* Waits for the handle's stream; reports a pending asynchronous error. */
 int rfast_sync(rfast_ctx* ctx);
 

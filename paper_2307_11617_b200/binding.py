@@ -82,6 +82,7 @@ def lib():
         L.rfast_version.restype = C.c_char_p
         L.rfast_compile_host.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule)] + [C.c_void_p] * 5 + \
             [C.c_char_p, C.c_size_t]
+        L.rfast_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int64]
         L.rfast_checkpoint_size.argtypes = [C.c_void_p]
         L.rfast_checkpoint_size.restype = C.c_int64
         L.rfast_checkpoint_save.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
@@ -237,6 +238,13 @@ def rfast_compile_host(wl, s):
             "streams": int(counts[3])}
 
 
+OPT_PERSISTENT, OPT_GRAPHS = 0, 1
+
+
+def rfast_set_option(handle, option: int, value: int) -> None:
+    _check(lib().rfast_set_option(handle, int(option), int(value)), handle)
+
+
 def rfast_checkpoint_save(handle) -> np.ndarray:
     """The handle's complete state as an opaque byte array (see rfast_checkpoint_save in rfast.h)."""
     size = lib().rfast_checkpoint_size(handle)
@@ -317,6 +325,9 @@ class Engine:
         if which == STATE_USED_TAU_RHO:
             shape = (self.query(Q_N_USED_TAU_RHO),)
         return rfast_read_state(self.h, which, shape, out)
+
+    def set_option(self, option, value):
+        rfast_set_option(self.h, option, value)
 
     def checkpoint(self):
         return rfast_checkpoint_save(self.h)

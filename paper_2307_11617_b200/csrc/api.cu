@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "persist.cuh"
 #include "rfast_internal.h"
 
 using namespace rfast;
@@ -57,6 +58,13 @@ struct rfast_ctx {
     std::vector<void*> sched_allocs;
     std::vector<float> alpha_round;         // per-round step size, empty: constant alpha
     uint64_t sched_hash = 0;                // identity of the loaded schedule (checkpoints)
+    // persistent multi-round kernel (L2-resident problems)
+    bool opt_persistent = true, opt_graphs = true, persist_ok = false;
+    int persist_grid = 0;
+    int* d_act_ptr = nullptr;
+    float* d_alpha_round = nullptr;
+    unsigned int* d_bar = nullptr;
+    int* d_pstatus = nullptr;
     int max_round_events = 0;
     int round = 0;
     int64_t launches = 0;
@@ -119,6 +127,8 @@ void free_schedule(rfast_ctx* c) {
     c->sched_bytes = 0;
     c->d_ev = c->d_init_ev = nullptr;
     c->vbuf = c->rbuf = c->scratch = nullptr;
+    c->d_act_ptr = nullptr; c->d_alpha_round = nullptr; c->d_bar = nullptr; c->d_pstatus = nullptr;
+    c->persist_ok = false;
     c->has_sched = false;
 }
 
@@ -235,8 +245,28 @@ int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
     return RFAST_OK;
 }
 
+size_t persist_smem(rfast_ctx* ctx) {
+    if (ctx->model != RFAST_MODEL_SOFTMAX) return 0;
+    return (size_t)ctx->batch * ctx->C * sizeof(float) + (size_t)ctx->batch * sizeof(int);
+}
+const void* persist_kernel(rfast_ctx* ctx) {
+    if (ctx->model == RFAST_MODEL_LEAST_SQUARES)
+        return ctx->compensated ? (const void*)k_persist_rounds<RFAST_MODEL_LEAST_SQUARES, true>
+                                : (const void*)k_persist_rounds<RFAST_MODEL_LEAST_SQUARES, false>;
+    if (ctx->model == RFAST_MODEL_SOFTMAX)
+        return ctx->compensated ? (const void*)k_persist_rounds<RFAST_MODEL_SOFTMAX, true>
+                                : (const void*)k_persist_rounds<RFAST_MODEL_SOFTMAX, false>;
+    return nullptr;
+}
+
 // after a synchronisation: did a bounded device-side wait run out?
 int check_device_status(rfast_ctx* ctx) {
+    if (ctx->d_pstatus) {
+        int st = 0;
+        CK(cudaMemcpyAsync(&st, ctx->d_pstatus, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+        CK(cudaStreamSynchronize(ctx->stream));
+        if (st != 0) return set_err(ctx, RFAST_ETIMEOUT, "a grid barrier of the persistent kernel ran out of time");
+    }
     if (ctx->mlp) {
         const int st = mlp_plan_status(ctx->mlp, ctx->stream);
         if (st < 0) return set_err(ctx, RFAST_ECUDA, "reading the device status word failed");
@@ -471,6 +501,30 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     if (ctx->model == RFAST_MODEL_SOFTMAX) per_ev = (size_t)ctx->batch * ctx->C;
     if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) per_ev = ctx->batch;
     CK(dev_alloc(ctx, &ctx->scratch, per_ev * std::max(ctx->n, ctx->max_round_events), true));
+    // persistent path: act_ptr / step sizes on the device, barrier counter, status word
+    if ((rc = upload(ctx, &ctx->d_act_ptr, c.act_ptr))) return rc;
+    if (!ctx->alpha_round.empty() && (rc = upload(ctx, &ctx->d_alpha_round, ctx->alpha_round))) return rc;
+    CK(dev_alloc(ctx, &ctx->d_bar, 1, true));
+    CK(dev_alloc(ctx, &ctx->d_pstatus, 1, true));
+    CK(cudaMemsetAsync(ctx->d_pstatus, 0, sizeof(int), ctx->stream));
+    ctx->persist_ok = false;
+    if ((ctx->model == RFAST_MODEL_LEAST_SQUARES || ctx->model == RFAST_MODEL_SOFTMAX) &&
+        (size_t)ctx->n * ctx->stride * sizeof(float) <= ((size_t)8 << 20)) {
+        int dev = 0, coop = 0, sms = 0, occ = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const size_t smem = persist_smem(ctx);
+        const void* fn = persist_kernel(ctx);
+        if (coop && fn && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, kThreads, smem) == cudaSuccess && occ > 0) {
+            const int tiles = (int)((ctx->stride / 4 + kThreads - 1) / kThreads);
+            const int B = ctx->batch ? ctx->batch : ctx->rows;
+            const int per_ev = std::max(tiles, ctx->model == RFAST_MODEL_SOFTMAX ? B : (B + 7) / 8);
+            const int want = std::max(1, ctx->max_round_events * per_ev);
+            ctx->persist_grid = std::min(want, sms * std::min(occ, 2));
+            ctx->persist_ok = true;
+        }
+    }
     ctx->has_sched = true;
     rc = reset_state(ctx);
     if (rc != RFAST_OK) return rc;
@@ -540,8 +594,27 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
     // the rounds of one call are recorded once into a CUDA graph and replayed when the same
     // span is run again (after a reset).  The legacy default stream cannot be captured; there
     // the kernels are launched directly.
-    const bool graph_ok = ctx->stream != nullptr && rounds >= 2;
-    if (graph_ok && ctx->graph_exec && ctx->graph_r0 == r0 && ctx->graph_r1 == r1) {
+    const bool graph_ok = ctx->opt_graphs && ctx->stream != nullptr && rounds >= 2;
+    if (ctx->persist_ok && ctx->opt_persistent && rounds >= 1) {
+        PersistArgs P{};
+        P.a.mix_slot = ctx->d_mix_slot; P.a.mix_w = ctx->d_mix_w;
+        P.a.news_new = ctx->d_news_new; P.a.news_prev = ctx->d_news_prev;
+        P.a.out_cur = ctx->d_out_cur; P.a.out_new = ctx->d_out_new; P.a.out_a = ctx->d_out_a;
+        P.a.x = ctx->x; P.a.z = ctx->z; P.a.zc = ctx->zc; P.a.vbuf = ctx->vbuf; P.a.rbuf = ctx->rbuf;
+        P.a.stride = ctx->stride; P.a.n4 = (int)(ctx->stride / 4); P.a.alpha = ctx->alpha;
+        P.a.ev = ctx->d_ev;
+        P.g = grad_args(ctx, ctx->d_ev);
+        P.use_all = (ctx->model == RFAST_MODEL_LEAST_SQUARES && ctx->batch == 0) ? 1 : 0;
+        if (P.use_all) P.g.B = ctx->rows;
+        P.act_ptr = ctx->d_act_ptr; P.alpha_round = ctx->d_alpha_round; P.r0 = r0; P.r1 = r1;
+        P.feat = ctx->feat; P.target = ctx->target; P.label = ctx->label; P.scratch = ctx->scratch;
+        P.bar = ctx->d_bar; P.status = ctx->d_pstatus;
+        CK(cudaMemsetAsync(ctx->d_bar, 0, sizeof(unsigned int), ctx->stream));
+        void* args[] = {&P};
+        CK(cudaLaunchCooperativeKernel(persist_kernel(ctx), dim3(ctx->persist_grid), dim3(kThreads), args,
+                                       persist_smem(ctx), ctx->stream));
+        ctx->launches += 1;
+    } else if (graph_ok && ctx->graph_exec && ctx->graph_r0 == r0 && ctx->graph_r1 == r1) {
         CK(cudaGraphLaunch(ctx->graph_exec, ctx->stream));
         ctx->launches += ctx->graph_launches;
     } else if (graph_ok) {
@@ -568,6 +641,15 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         return check_device_status(ctx);
     }
     return RFAST_OK;
+}
+
+int rfast_set_option(rfast_ctx* ctx, int option, int64_t value) {
+    if (!ctx) return RFAST_EINVAL;
+    switch (option) {
+        case RFAST_OPT_PERSISTENT: ctx->opt_persistent = value != 0; return RFAST_OK;
+        case RFAST_OPT_GRAPHS: ctx->opt_graphs = value != 0; return RFAST_OK;
+        default: return set_err(ctx, RFAST_EINVAL, "unknown option");
+    }
 }
 
 int rfast_sync(rfast_ctx* ctx) {

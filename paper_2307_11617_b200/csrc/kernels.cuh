@@ -32,6 +32,14 @@ struct RoundArgs {
 __device__ __forceinline__ float4 ld_stream(const float* row, int i4) {
     return __ldcs(reinterpret_cast<const float4*>(row) + i4);
 }
+// CG = true: go to L2 (ld.global.cg).  Used inside the persistent multi-round kernel, where rows
+// written by other CTAs earlier in the same launch must never be served from a stale L1 line.
+template <bool CG>
+__device__ __forceinline__ float4 ld_sel(const float* row, int i4) {
+    return CG ? __ldcg(reinterpret_cast<const float4*>(row) + i4) : __ldcs(reinterpret_cast<const float4*>(row) + i4);
+}
+template <bool CG>
+__device__ __forceinline__ float ld_sel1(const float* p) { return CG ? __ldcg(p) : *p; }
 __device__ __forceinline__ void st_stream(float* row, int i4, float4 v) {
     __stcs(reinterpret_cast<float4*>(row) + i4, v);
 }
@@ -72,7 +80,7 @@ constexpr int kThreads = 256;
 // and kept in the node's own low-order part, so that the tracked mass of Lemma 3 is conserved
 // to second order instead of drifting with every fp32 rounding.  The running sums stay fp32.
 // ---------------------------------------------------------------------------------------------
-template <int U, bool COMP>
+template <int U, bool COMP, bool CG = false>
 __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc& e, int base, float* zr,
                                                const float4 (&zv)[U], const float4 (&gn)[U],
                                                const float4 (&go)[U]) {
@@ -88,8 +96,8 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
             for (int u = 0; u < U; ++u) {
                 const int i4 = base + u * kThreads;
                 if (i4 < a.n4) {
-                    float4 dl = ld_stream(nr, i4);
-                    if (prev >= 0) dl = f4_sub(dl, ld_stream(pr, i4));
+                    float4 dl = ld_sel<CG>(nr, i4);
+                    if (prev >= 0) dl = f4_sub(dl, ld_sel<CG>(pr, i4));
                     zh[u] = f4_add(zh[u], dl);
                 }
             }
@@ -110,7 +118,7 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
                 const int i4 = base + u * kThreads;
                 if (i4 < a.n4) {
                     float4 r = f4_scale(aw, zh[u]);
-                    if (cur >= 0) r = f4_add(ld_stream(cr, i4), r);
+                    if (cur >= 0) r = f4_add(ld_sel<CG>(cr, i4), r);
                     st_stream(wr, i4, r);
                 }
             }
@@ -123,7 +131,7 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
             const int i4 = base + u * kThreads;
             hi[u] = zv[u];
             lo[u] = make_float4(0, 0, 0, 0);
-            if (i4 < a.n4) lo[u] = ld_stream(cr_, i4);
+            if (i4 < a.n4) lo[u] = ld_sel<CG>(cr_, i4);
         }
         for (int m = 0; m < e.news_cnt; ++m) {
             const float* nr = a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride;
@@ -133,8 +141,8 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
             for (int u = 0; u < U; ++u) {
                 const int i4 = base + u * kThreads;
                 if (i4 < a.n4) {
-                    const float4 nv = ld_stream(nr, i4);
-                    const float4 pv = prev >= 0 ? ld_stream(pr, i4) : make_float4(0, 0, 0, 0);
+                    const float4 nv = ld_sel<CG>(nr, i4);
+                    const float4 pv = prev >= 0 ? ld_sel<CG>(pr, i4) : make_float4(0, 0, 0, 0);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         float d, de, s, se;
@@ -173,7 +181,7 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
             for (int u = 0; u < U; ++u) {
                 const int i4 = base + u * kThreads;
                 if (i4 < a.n4) {
-                    const float4 cv = cur >= 0 ? ld_stream(cr, i4) : make_float4(0, 0, 0, 0);
+                    const float4 cv = cur >= 0 ? ld_sel<CG>(cr, i4) : make_float4(0, 0, 0, 0);
                     float4 r;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -288,20 +296,19 @@ k_quad_grad(const float* __restrict__ x, const float* __restrict__ qd, const flo
 // bf16 copy of the new x (operand of the MLP's matrix products), or starts the new gradient
 // row with the dense term l2 * x (sparse objective).  grid = (tiles, events)
 // ---------------------------------------------------------------------------------------------
-template <int U, bool BF16, bool GINIT>
-__global__ void __launch_bounds__(kThreads)
-k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int64_t gplane, float l2) {
-    const EvDesc e = a.ev[blockIdx.y];
+template <int U, bool BF16, bool GINIT, bool CG>
+__device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, int tile, __nv_bfloat16* xb,
+                                         float* gbuf, int64_t gplane, float l2) {
     const int64_t row = (int64_t)e.node * a.stride;
     float* xr = a.x + row;
     const float* zr = a.z + row;
-    const int base = blockIdx.x * (kThreads * U) + threadIdx.x;
+    const int base = tile * (kThreads * U) + threadIdx.x;
     float4 acc[U], v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const int i4 = base + u * kThreads;
         float4 xv = make_float4(0, 0, 0, 0), zv = xv;
-        if (i4 < a.n4) { xv = ld_stream(xr, i4); zv = ld_stream(zr, i4); }
+        if (i4 < a.n4) { xv = ld_sel<CG>(xr, i4); zv = ld_sel<CG>(zr, i4); }
         v[u] = f4_axpy(-a.alpha, zv, xv);
         acc[u] = f4_scale(e.w_self, v[u]);
     }
@@ -319,7 +326,7 @@ k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int i4 = base + u * kThreads;
-            if (i4 < a.n4) acc[u] = f4_axpy(w, ld_stream(nr, i4), acc[u]);
+            if (i4 < a.n4) acc[u] = f4_axpy(w, ld_sel<CG>(nr, i4), acc[u]);
         }
     }
 #pragma unroll
@@ -340,6 +347,12 @@ k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int
             }
         }
     }
+}
+
+template <int U, bool BF16, bool GINIT>
+__global__ void __launch_bounds__(kThreads)
+k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int64_t gplane, float l2) {
+    mix_tile<U, BF16, GINIT, false>(a, a.ev[blockIdx.y], blockIdx.x, xb, gbuf, gplane, l2);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -376,83 +389,99 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// The per-row and per-coordinate pieces below are shared by the one-kernel-per-phase path and
+// by the persistent multi-round kernel, so that both produce the same bits.  ev_local is the
+// event's index inside its round (the scratch arrays are laid out per round).
+
 // Least squares, phase 1: residual r_k = a_k . x - y_k, one warp per sampled row.
-// grid = (ceil(B / 8), events), 256 threads.  res: [events][B]
-__global__ void __launch_bounds__(256)
-k_ls_residual(GradArgs g, const float* __restrict__ feat, const float* __restrict__ target,
-              float* __restrict__ res, int use_all) {
-    const EvDesc e = g.ev[blockIdx.y];
-    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (k >= g.B) return;
+template <bool CG>
+__device__ __forceinline__ void ls_residual_row(const GradArgs& g, const EvDesc& e, int ev_local, int k, int lane,
+                                                const float* feat, const float* target, float* res, int use_all) {
     const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
     const float* a = feat + ((int64_t)e.node * g.rows + rrow) * g.F;
     const float* x = g.x + (int64_t)e.node * g.stride;
     float s = 0.f;
-    for (int c = lane; c < g.F; c += 32) s = fmaf(a[c], x[c], s);
+    for (int c = lane; c < g.F; c += 32) s = fmaf(a[c], ld_sel1<CG>(x + c), s);
     s = warp_sum(s);
-    if (lane == 0) res[(int64_t)blockIdx.y * g.B + k] = s - target[(int64_t)e.node * g.rows + rrow];
+    if (lane == 0) res[(int64_t)ev_local * g.B + k] = s - target[(int64_t)e.node * g.rows + rrow];
+}
+// grid = (ceil(B / 8), events), 256 threads.  res: [events][B]
+__global__ void __launch_bounds__(256)
+k_ls_residual(GradArgs g, const float* __restrict__ feat, const float* __restrict__ target,
+              float* __restrict__ res, int use_all) {
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (k >= g.B) return;
+    ls_residual_row<false>(g, g.ev[blockIdx.y], blockIdx.y, k, threadIdx.x & 31, feat, target, res, use_all);
 }
 
-// Least squares, phase 2: g_c = (1/B) sum_k a_k[c] r_k + l2 x_c.  grid = (ceil(p/256), events)
+// Least squares, phase 2: g_c = (1/B) sum_k a_k[c] r_k + l2 x_c.
+template <bool CG>
+__device__ __forceinline__ float ls_grad_coord(const GradArgs& g, const EvDesc& e, int ev_local, int c,
+                                               const float* feat, const float* res, int use_all) {
+    const float* abase = feat + (int64_t)e.node * g.rows * g.F;
+    float s = 0.f;
+    for (int k = 0; k < g.B; ++k) {
+        const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+        s = fmaf(abase[(int64_t)rrow * g.F + c], ld_sel1<CG>(res + (int64_t)ev_local * g.B + k), s);
+    }
+    return s / (float)g.B + g.l2 * ld_sel1<CG>(g.x + (int64_t)e.node * g.stride + c);
+}
+// grid = (ceil(p/256), events)
 __global__ void __launch_bounds__(256)
 k_ls_grad(GradArgs g, const float* __restrict__ feat, const float* __restrict__ res, int use_all) {
     const EvDesc e = g.ev[blockIdx.y];
     const int c = blockIdx.x * 256 + threadIdx.x;
     if (c >= g.F) return;
-    const float* abase = feat + (int64_t)e.node * g.rows * g.F;
-    float s = 0.f;
-    for (int k = 0; k < g.B; ++k) {
-        const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
-        s = fmaf(abase[(int64_t)rrow * g.F + c], res[(int64_t)blockIdx.y * g.B + k], s);
-    }
-    const int64_t row = (int64_t)e.node * g.stride;
-    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + row + c] = s / (float)g.B + g.l2 * g.x[row + c];
+    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + (int64_t)e.node * g.stride + c] =
+        ls_grad_coord<false>(g, e, blockIdx.y, c, feat, res, use_all);
 }
 
-// Softmax regression, phase 1: logits[k][c] = W_c . a_k + bias_c; one block per sampled row,
-// one warp per class (round-robin).  grid = (B, events).  logit: [events][B][C]
-__global__ void __launch_bounds__(256)
-k_softmax_logits(GradArgs g, const float* __restrict__ feat, float* __restrict__ logit) {
-    const EvDesc e = g.ev[blockIdx.y];
-    const int k = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// Softmax regression, phase 1: logits[k][c] = W_c . a_k + bias_c for one sampled row k by one
+// block, one warp per class (round-robin).  logit: [events][B][C]
+template <bool CG>
+__device__ __forceinline__ void softmax_logits_row(const GradArgs& g, const EvDesc& e, int ev_local, int k,
+                                                   const float* feat, float* logit) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
     const float* a = feat + ((int64_t)e.node * g.rows + rrow) * g.F;
     const float* x = g.x + (int64_t)e.node * g.stride;
     for (int c = warp; c < g.C; c += 8) {
         const float* w = x + (int64_t)c * g.F;
         float s = 0.f;
-        for (int f = lane; f < g.F; f += 32) s = fmaf(a[f], w[f], s);
+        for (int f = lane; f < g.F; f += 32) s = fmaf(a[f], ld_sel1<CG>(w + f), s);
         s = warp_sum(s);
-        if (lane == 0) logit[((int64_t)blockIdx.y * g.B + k) * g.C + c] = s + x[(int64_t)g.C * g.F + c];
+        if (lane == 0) logit[((int64_t)ev_local * g.B + k) * g.C + c] = s + ld_sel1<CG>(x + (int64_t)g.C * g.F + c);
     }
 }
-
-// Softmax regression, phase 2: delta = (softmax(logits) - onehot) / B (recomputed per block in
-// shared memory), then g[c][f] = sum_k delta[k][c] a_k[f] + l2 W[c][f] and the bias gradient.
-// grid = (ceil(p / 256), events); dynamic shared memory: B*C floats + B ints
+// grid = (B, events)
 __global__ void __launch_bounds__(256)
-k_softmax_grad(GradArgs g, const float* __restrict__ feat, const int* __restrict__ label,
-               const float* __restrict__ logit) {
-    extern __shared__ float sm[];
-    float* delta = sm;                                   // [B][C]
-    int* rowid = reinterpret_cast<int*>(sm + g.B * g.C); // [B]
-    const EvDesc e = g.ev[blockIdx.y];
+k_softmax_logits(GradArgs g, const float* __restrict__ feat, float* __restrict__ logit) {
+    softmax_logits_row<false>(g, g.ev[blockIdx.y], blockIdx.y, blockIdx.x, feat, logit);
+}
+
+// Softmax regression, phase 2: delta = (softmax(logits) - onehot) / B for all sampled rows of
+// one event into shared memory (block-wide, ends with a barrier) ...
+template <bool CG>
+__device__ __forceinline__ void softmax_delta_block(const GradArgs& g, const EvDesc& e, int ev_local,
+                                                    const int* label, const float* logit, float* delta, int* rowid) {
     for (int k = threadIdx.x; k < g.B; k += 256) {
         const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
         rowid[k] = rrow;
-        const float* lg = logit + ((int64_t)blockIdx.y * g.B + k) * g.C;
-        float m = lg[0];
-        for (int c = 1; c < g.C; ++c) m = fmaxf(m, lg[c]);
+        const float* lg = logit + ((int64_t)ev_local * g.B + k) * g.C;
+        float m = ld_sel1<CG>(lg);
+        for (int c = 1; c < g.C; ++c) m = fmaxf(m, ld_sel1<CG>(lg + c));
         float den = 0.f;
-        for (int c = 0; c < g.C; ++c) den += expf(lg[c] - m);
+        for (int c = 0; c < g.C; ++c) den += expf(ld_sel1<CG>(lg + c) - m);
         const int lab = label[(int64_t)e.node * g.rows + rrow];
         for (int c = 0; c < g.C; ++c)
-            delta[k * g.C + c] = (expf(lg[c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)g.B;
+            delta[k * g.C + c] = (expf(ld_sel1<CG>(lg + c) - m) / den - (c == lab ? 1.f : 0.f)) / (float)g.B;
     }
     __syncthreads();
-    const int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (q >= g.p) return;
-    const int64_t row = (int64_t)e.node * g.stride;
+}
+// ... then g[c][f] = sum_k delta[k][c] a_k[f] + l2 W[c][f], and the bias gradient, per coordinate q.
+template <bool CG>
+__device__ __forceinline__ float softmax_grad_coord(const GradArgs& g, const EvDesc& e, int64_t q,
+                                                    const float* feat, const float* delta, const int* rowid) {
     float s = 0.f;
     if (q < (int64_t)g.C * g.F) {
         const int c = (int)(q / g.F), f = (int)(q % g.F);
@@ -462,7 +491,21 @@ k_softmax_grad(GradArgs g, const float* __restrict__ feat, const int* __restrict
         const int c = (int)(q - (int64_t)g.C * g.F);
         for (int k = 0; k < g.B; ++k) s += delta[k * g.C + c];
     }
-    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + row + q] = s + g.l2 * g.x[row + q];
+    return s + g.l2 * ld_sel1<CG>(g.x + (int64_t)e.node * g.stride + q);
+}
+// grid = (ceil(p / 256), events); dynamic shared memory: B*C floats + B ints
+__global__ void __launch_bounds__(256)
+k_softmax_grad(GradArgs g, const float* __restrict__ feat, const int* __restrict__ label,
+               const float* __restrict__ logit) {
+    extern __shared__ float sm[];
+    float* delta = sm;                                   // [B][C]
+    int* rowid = reinterpret_cast<int*>(sm + g.B * g.C); // [B]
+    const EvDesc e = g.ev[blockIdx.y];
+    softmax_delta_block<false>(g, e, blockIdx.y, label, logit, delta, rowid);
+    const int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (q >= g.p) return;
+    g.gbuf[(int64_t)(e.g_par ^ 1) * g.gplane + (int64_t)e.node * g.stride + q] =
+        softmax_grad_coord<false>(g, e, q, feat, delta, rowid);
 }
 
 // Sparse logistic regression, phase 1: coef_k = -y_k / (1 + exp(y_k a_k.x)) / B, one warp per

@@ -241,3 +241,35 @@ def test_graph_replay_on_a_user_stream_equals_direct_launches(rfast_lib, name, o
         x3 = eng.read(B.STATE_X)
     assert np.array_equal(xd, x1) and np.array_equal(yd, y1)
     assert np.array_equal(x1, x2) and np.array_equal(y1, y2) and np.array_equal(x1, x3)
+
+
+@pytest.mark.parametrize("name,ov", [
+    ("ls_ring4", {}),
+    ("ls_ring4", dict(n=9, p=300, rows=40, K=60)),
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=150, batch=8)),
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=80, batch=8, compensated=False)),
+    ("softmax_exp16", dict(n=8, F=784, C=10, rows=64, K=40, batch=32)),
+], ids=["config 1", "ls wider", "softmax", "softmax plain", "softmax 784x10"])
+def test_persistent_kernel_equals_one_kernel_per_phase(rfast_lib, name, ov):
+    """L2-resident problems run a span of rounds as one cooperative persistent kernel with
+    bounded grid barriers; with the option off, one kernel per phase.  Same bits, and parity
+    with the oracle either way."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config(name, seed=3, **ov)
+    orc, ref0 = _oracle(wl)
+    res = {}
+    for persistent in (1, 0):
+        with pkg.Engine(wl) as eng:
+            eng.set_option(B.OPT_PERSISTENT, persistent)
+            eng.load_schedule(wl.schedule)
+            l0 = eng.query(B.Q_LAUNCHES)             # the initial gradients are launched at load time
+            eng.run(7)                               # spans of several lengths
+            eng.run(1)
+            eng.run()
+            _compare(eng, orc, ref0)
+            res[persistent] = (eng.read(B.STATE_X), eng.read(B.STATE_Y), eng.read(B.STATE_G_LAST),
+                               eng.read(B.STATE_RHO_LATEST), eng.query(B.Q_LAUNCHES) - l0)
+    for u, v in zip(res[1][:4], res[0][:4]):
+        assert np.array_equal(u, v)
+    assert res[1][4] == 3 and res[0][4] > 3 * 7       # one launch per span against several per round
