@@ -191,14 +191,21 @@ int rfast_reset(rfast_ctx* ctx);
 /* A counter (>= 0), or a negative status for an unknown id / NULL handle. */
 int64_t rfast_query(rfast_ctx* ctx, int what);
 
-/* Execution options (they never change results: every path produces the same bits).
- *   RFAST_OPT_PERSISTENT  1 (default): problems whose state fits L2 (least squares, softmax
- *                         regression) run a span of rounds as ONE cooperative persistent
- *                         kernel with bounded grid barriers between the phases of a round;
- *                         0: one kernel per phase.
+/* Execution options.  The first two never change results: every path produces the same bits.
+ *   RFAST_OPT_PERSISTENT  0 (default): one kernel per phase of a round.  1: problems whose state
+ *                         fits L2 (least squares, softmax regression) run a span of rounds as
+ *                         ONE cooperative persistent kernel with grid barriers between the
+ *                         phases of a round.  Every barrier wait is bounded; if one runs out
+ *                         the kernel returns and the next synchronising call reports
+ *                         RFAST_ETIMEOUT (the state is then undefined, the device healthy:
+ *                         rfast_reset starts over).
  *   RFAST_OPT_GRAPHS      1 (default): spans of rounds are recorded into a CUDA graph and
- *                         replayed (non-default streams only); 0: direct launches. */
-enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1 };
+ *                         replayed (non-default streams only); 0: direct launches.
+ *   RFAST_OPT_WAIT_LIMIT_MS     bound of every device-side barrier wait, 1..60000 (default 2000).
+ *   RFAST_OPT_PHANTOM_ARRIVALS  failure injection for tests, made on the host: the grid barrier
+ *                         expects this many arrivals that nobody makes, so its bounded wait runs
+ *                         out and the timeout path is exercised (default 0). */
+enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1, RFAST_OPT_WAIT_LIMIT_MS = 2, RFAST_OPT_PHANTOM_ARRIVALS = 3 };
 int rfast_set_option(rfast_ctx* ctx, int option, int64_t value);
 
 /* Waits for the handle's stream; reports a pending asynchronous error. */

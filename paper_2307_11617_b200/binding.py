@@ -238,7 +238,7 @@ def rfast_compile_host(wl, s):
             "streams": int(counts[3])}
 
 
-OPT_PERSISTENT, OPT_GRAPHS = 0, 1
+OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS = 0, 1, 2, 3
 
 
 def rfast_set_option(handle, option: int, value: int) -> None:

@@ -59,7 +59,8 @@ struct rfast_ctx {
     std::vector<float> alpha_round;         // per-round step size, empty: constant alpha
     uint64_t sched_hash = 0;                // identity of the loaded schedule (checkpoints)
     // persistent multi-round kernel (L2-resident problems)
-    bool opt_persistent = true, opt_graphs = true, persist_ok = false;
+    bool opt_persistent = false, opt_graphs = true, persist_ok = false;
+    int64_t opt_wait_limit_ms = 2000, opt_phantom = 0;
     int persist_grid = 0;
     int* d_act_ptr = nullptr;
     float* d_alpha_round = nullptr;
@@ -245,10 +246,13 @@ int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
     return RFAST_OK;
 }
 
-size_t persist_smem(rfast_ctx* ctx) {
-    if (ctx->model != RFAST_MODEL_SOFTMAX) return 0;
-    return (size_t)ctx->batch * ctx->C * sizeof(float) + (size_t)ctx->batch * sizeof(int);
+// floats in front of the x staging area: delta [B][C] + row ids [B] (softmax), residuals [B] (least squares)
+int persist_xs_off(rfast_ctx* ctx) {
+    const int B = ctx->batch ? ctx->batch : ctx->rows;
+    const int head = ctx->model == RFAST_MODEL_SOFTMAX ? B * ctx->C + B : B;
+    return (head + 3) / 4 * 4;
 }
+size_t persist_smem(rfast_ctx* ctx) { return ((size_t)persist_xs_off(ctx) + ctx->stride) * sizeof(float); }
 const void* persist_kernel(rfast_ctx* ctx) {
     if (ctx->model == RFAST_MODEL_LEAST_SQUARES)
         return ctx->compensated ? (const void*)k_persist_rounds<RFAST_MODEL_LEAST_SQUARES, true>
@@ -509,19 +513,20 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     CK(cudaMemsetAsync(ctx->d_pstatus, 0, sizeof(int), ctx->stream));
     ctx->persist_ok = false;
     if ((ctx->model == RFAST_MODEL_LEAST_SQUARES || ctx->model == RFAST_MODEL_SOFTMAX) &&
-        (size_t)ctx->n * ctx->stride * sizeof(float) <= ((size_t)8 << 20)) {
+        (size_t)ctx->n * ctx->stride * sizeof(float) <= ((size_t)8 << 20) && persist_smem(ctx) <= 200 * 1024) {
         int dev = 0, coop = 0, sms = 0, occ = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const size_t smem = persist_smem(ctx);
         const void* fn = persist_kernel(ctx);
+        if (fn) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (coop && fn && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, kThreads, smem) == cudaSuccess && occ > 0) {
             const int tiles = (int)((ctx->stride / 4 + kThreads - 1) / kThreads);
             const int B = ctx->batch ? ctx->batch : ctx->rows;
-            const int per_ev = std::max(tiles, ctx->model == RFAST_MODEL_SOFTMAX ? B : (B + 7) / 8);
+            const int per_ev = std::max(tiles, ctx->model == RFAST_MODEL_SOFTMAX ? (B + 3) / 4 : (B + 7) / 8);
             const int want = std::max(1, ctx->max_round_events * per_ev);
-            ctx->persist_grid = std::min(want, sms * std::min(occ, 2));
+            ctx->persist_grid = std::min(want, sms);          // one CTA per SM keeps the barrier short
             ctx->persist_ok = true;
         }
     }
@@ -609,6 +614,9 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         P.act_ptr = ctx->d_act_ptr; P.alpha_round = ctx->d_alpha_round; P.r0 = r0; P.r1 = r1;
         P.feat = ctx->feat; P.target = ctx->target; P.label = ctx->label; P.scratch = ctx->scratch;
         P.bar = ctx->d_bar; P.status = ctx->d_pstatus;
+        P.xs_off = persist_xs_off(ctx); P.rows_per_item = 4;
+        P.phantom = (unsigned int)ctx->opt_phantom; P.limit_ns = (unsigned long long)ctx->opt_wait_limit_ms * 1000000ull;
+        CK(cudaMemsetAsync(ctx->d_pstatus, 0, sizeof(int), ctx->stream));
         CK(cudaMemsetAsync(ctx->d_bar, 0, sizeof(unsigned int), ctx->stream));
         void* args[] = {&P};
         CK(cudaLaunchCooperativeKernel(persist_kernel(ctx), dim3(ctx->persist_grid), dim3(kThreads), args,
@@ -648,6 +656,12 @@ int rfast_set_option(rfast_ctx* ctx, int option, int64_t value) {
     switch (option) {
         case RFAST_OPT_PERSISTENT: ctx->opt_persistent = value != 0; return RFAST_OK;
         case RFAST_OPT_GRAPHS: ctx->opt_graphs = value != 0; return RFAST_OK;
+        case RFAST_OPT_WAIT_LIMIT_MS:
+            if (value < 1 || value > 60000) return set_err(ctx, RFAST_EINVAL, "wait limit must be 1..60000 ms");
+            ctx->opt_wait_limit_ms = value; return RFAST_OK;
+        case RFAST_OPT_PHANTOM_ARRIVALS:
+            if (value < 0 || value > 1024) return set_err(ctx, RFAST_EINVAL, "phantom arrivals must be 0..1024");
+            ctx->opt_phantom = value; return RFAST_OK;
         default: return set_err(ctx, RFAST_EINVAL, "unknown option");
     }
 }

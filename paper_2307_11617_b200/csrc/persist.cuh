@@ -8,7 +8,8 @@
 // one-kernel-per-phase path, so the results are bit-identical.
 //
 // Grid barrier: one monotone counter in global memory; CTA leaders add 1 and spin until it
-// reaches (number of barriers so far) x (number of CTAs).  Every spin is bounded in time: when
+// reaches (number of barriers so far) x (number of CTAs).  Every spin is bounded in time (2 s by
+// default, RFAST_OPT_WAIT_LIMIT_MS): when
 // it runs out (or another CTA has already given up) the CTA records a code in the status word
 // and returns; the host reports RFAST_ETIMEOUT.  The launch is cooperative, so all CTAs are
 // co-resident and the barrier cannot starve.  State written by other CTAs earlier in the same
@@ -28,32 +29,40 @@ struct PersistArgs {
     const float* feat;  const float* target;  const int* label;
     float* scratch;              // residuals [events in round][B] / logits [events in round][B][C]
     int use_all;                 // least squares: the whole shard is the batch
+    int xs_off;                  // offset (floats) of the x staging area in dynamic shared memory
+    int rows_per_item;           // softmax: sampled rows handled per work item of phase 2
+    unsigned int phantom;        // arrivals the barrier expects beyond the launched CTAs (0 in normal
+                                 // use; a host-side failure-injection hook: nobody makes them, so the
+                                 // bounded wait runs out and the kernel returns with the status set)
+    unsigned long long limit_ns; // bound of every barrier wait
     unsigned int* bar;           // barrier counter, zero at launch
     int* status;                 // 0, or kPersistTimeout once a wait ran out
 };
 
 constexpr int kPersistTimeout = 9;
-constexpr unsigned long long kBarrierLimitNs = 2000000000ull;
 
 // false: give up (status is set)
-__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int& target, int* status) {
+__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int& target, int* status,
+                                             unsigned int arrivals, unsigned long long limit_ns) {
     __syncthreads();
     int ok = 1;
     if (threadIdx.x == 0) {
-        target += gridDim.x;
+        target += arrivals;
         __threadfence();                                   // publish this CTA's writes
         atomicAdd(bar, 1u);
-        unsigned long long t0, now;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-        while (true) {
+        unsigned long long t0 = 0, now;
+        for (unsigned int spins = 0;; ++spins) {
             unsigned int seen;
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(bar) : "memory");
             if (seen >= target) break;
-            int st;
-            asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(st) : "l"(status) : "memory");
-            if (st != 0) { ok = 0; break; }
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-            if (now - t0 > kBarrierLimitNs) { atomicExch(status, kPersistTimeout); ok = 0; break; }
+            if ((spins & 255u) == 255u) {                    // the clock and the status word are slow to read
+                int st;
+                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(st) : "l"(status) : "memory");
+                if (st != 0) { ok = 0; break; }
+                asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > limit_ns) { atomicExch(status, kPersistTimeout); ok = 0; break; }
+            }
         }
         __threadfence();                                   // and see everybody else's
     }
@@ -61,7 +70,8 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int& ta
 }
 
 // MODEL: RFAST_MODEL_LEAST_SQUARES or RFAST_MODEL_SOFTMAX.  Launched cooperatively with
-// gridDim.x <= number of co-resident CTAs; dynamic shared memory: B*C floats + B ints (softmax).
+// gridDim.x <= number of co-resident CTAs; dynamic shared memory: B*C floats + B ints (softmax) or
+// B floats (least squares: the residuals of the item's event), then stride floats for x.
 template <int MODEL, bool COMP>
 __global__ void __launch_bounds__(kThreads)
 k_persist_rounds(PersistArgs P) {
@@ -79,22 +89,53 @@ k_persist_rounds(PersistArgs P) {
             const EvDesc e = a.ev[ev0 + item / tiles];
             mix_tile<1, false, false, true>(a, e, item % tiles, nullptr, nullptr, 0, 0.f);
         }
-        if (!grid_barrier(P.bar, target, P.status)) return;
+        if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
         // ---- phase 2: per-row scalars of the sample gradient --------------------------------------
-        if (MODEL == RFAST_MODEL_LEAST_SQUARES) {
-            const int groups = (g.B + 7) / 8;
-            for (int item = blockIdx.x; item < nev * groups; item += gridDim.x) {
-                const int el = item / groups, k = (item % groups) * 8 + (threadIdx.x >> 5);
-                if (k < g.B)
-                    ls_residual_row<true>(g, a.ev[ev0 + el], el, k, threadIdx.x & 31, P.feat, P.target, P.scratch, P.use_all);
-            }
-        } else {
-            for (int item = blockIdx.x; item < nev * g.B; item += gridDim.x) {
-                const int el = item / g.B;
-                softmax_logits_row<true>(g, a.ev[ev0 + el], el, item % g.B, P.feat, P.scratch);
+        // The new x of the item's node is first copied into shared memory with wide L2 loads that
+        // are all in flight together; the dot products then run out of shared memory.  (Reading x
+        // element by element through L2 inside the reduction loops would serialise on L2 latency.)
+        {
+            float* xs = sm + P.xs_off;                       // [stride] floats
+            const int per_ev = MODEL == RFAST_MODEL_LEAST_SQUARES ? (g.B + 7) / 8 : (g.B + P.rows_per_item - 1) / P.rows_per_item;
+            int have = -1;                                   // event whose x is in shared memory
+            for (int item = blockIdx.x; item < nev * per_ev; item += gridDim.x) {
+                const int el = item / per_ev, sub = item % per_ev;
+                const EvDesc e = a.ev[ev0 + el];
+                if (have != el) {
+                    __syncthreads();
+                    const float* xr = g.x + (int64_t)e.node * g.stride;
+                    for (int i4 = threadIdx.x; i4 < a.n4; i4 += kThreads)
+                        reinterpret_cast<float4*>(xs)[i4] = __ldcg(reinterpret_cast<const float4*>(xr) + i4);
+                    __syncthreads();
+                    have = el;
+                }
+                if (MODEL == RFAST_MODEL_LEAST_SQUARES) {
+                    const int k = sub * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+                    if (k < g.B) {
+                        const int rrow = P.use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+                        const float* arow = P.feat + ((int64_t)e.node * g.rows + rrow) * g.F;
+                        float s = 0.f;
+                        for (int c = lane; c < g.F; c += 32) s = fmaf(arow[c], xs[c], s);
+                        s = warp_sum(s);
+                        if (lane == 0) P.scratch[(int64_t)el * g.B + k] = s - P.target[(int64_t)e.node * g.rows + rrow];
+                    }
+                } else {
+                    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+                    for (int k = sub * P.rows_per_item; k < min(g.B, (sub + 1) * P.rows_per_item); ++k) {
+                        const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
+                        const float* arow = P.feat + ((int64_t)e.node * g.rows + rrow) * g.F;
+                        for (int c = warp; c < g.C; c += 8) {
+                            const float* w = xs + (int64_t)c * g.F;
+                            float s = 0.f;
+                            for (int f = lane; f < g.F; f += 32) s = fmaf(arow[f], w[f], s);
+                            s = warp_sum(s);
+                            if (lane == 0) P.scratch[((int64_t)el * g.B + k) * g.C + c] = s + xs[(int64_t)g.C * g.F + c];
+                        }
+                    }
+                }
             }
         }
-        if (!grid_barrier(P.bar, target, P.status)) return;
+        if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
         // ---- phase 3: gradient per coordinate, then S2b + S2c on the same coordinates ---------------
         for (int item = blockIdx.x; item < nev * tiles; item += gridDim.x) {
             const int el = item / tiles, tile = item % tiles;
@@ -104,6 +145,10 @@ k_persist_rounds(PersistArgs P) {
             if (MODEL == RFAST_MODEL_SOFTMAX) {
                 __syncthreads();                             // the previous item's readers are done
                 softmax_delta_block<true>(g, e, el, P.label, P.scratch, delta, rowid);
+            } else {
+                __syncthreads();
+                for (int k = threadIdx.x; k < g.B; k += kThreads) delta[k] = __ldcg(P.scratch + (int64_t)el * g.B + k);
+                __syncthreads();
             }
             const int i4 = tile * kThreads + threadIdx.x;
             const int64_t row = (int64_t)e.node * a.stride;
@@ -114,9 +159,19 @@ k_persist_rounds(PersistArgs P) {
                 for (int j = 0; j < 4; ++j) {
                     const int64_t q = (int64_t)i4 * 4 + j;
                     float v = 0.f;
-                    if (q < g.p)
-                        v = MODEL == RFAST_MODEL_SOFTMAX ? softmax_grad_coord<true>(g, e, q, P.feat, delta, rowid)
-                                                         : ls_grad_coord<true>(g, e, el, (int)q, P.feat, P.scratch, P.use_all);
+                    if (q < g.p) {
+                        if (MODEL == RFAST_MODEL_SOFTMAX) {
+                            v = softmax_grad_coord<true>(g, e, q, P.feat, delta, rowid);
+                        } else {                             // same order of operations as ls_grad_coord
+                            const float* abase = P.feat + (int64_t)e.node * g.rows * g.F;
+                            float s = 0.f;
+                            for (int k = 0; k < g.B; ++k) {
+                                const int rrow = P.use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+                                s = fmaf(abase[(int64_t)rrow * g.F + q], delta[k], s);
+                            }
+                            v = s / (float)g.B + g.l2 * __ldcg(g.x + row + q);
+                        }
+                    }
                     comp(gnv[0], j) = v;
                 }
                 reinterpret_cast<float4*>(g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row)[i4] = gnv[0];
@@ -125,7 +180,7 @@ k_persist_rounds(PersistArgs P) {
             }
             track_and_push<1, COMP, true>(a, e, i4, a.z + row, zh, gnv, gov);
         }
-        if (!grid_barrier(P.bar, target, P.status)) return;
+        if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
     }
 }
 

@@ -83,3 +83,31 @@ def test_diagnostics_match_the_oracle_state(rfast_lib, name, ov):
     # Lemma 3 on the device state, relative to the gradients that are summed
     scale = np.abs(G).sum(axis=0).max()
     assert d["conservation_residual"] <= 1e-5 * scale
+
+
+def test_bounded_barrier_wait_reports_timeout_and_the_handle_recovers(rfast_lib):
+    """Failure detection without faulting the GPU: the persistent kernel's grid barrier is told
+    (on the host) to expect an arrival that nobody makes; its bounded wait runs out, the kernel
+    returns, the next synchronising call reports RFAST_ETIMEOUT, and after a reset the same
+    handle runs the schedule correctly."""
+    import time
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    from paper_2307_11617_b200.binding import ETIMEOUT, RFastError
+    wl = build_config("ls_ring4", seed=2)
+    orc = from_workload(wl, make_model(wl).grad)
+    run_schedule(orc, wl.schedule)
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_PERSISTENT, 1)
+        eng.set_option(B.OPT_WAIT_LIMIT_MS, 200)
+        eng.set_option(B.OPT_PHANTOM_ARRIVALS, 1)
+        eng.load_schedule(wl.schedule)
+        t0 = time.time()
+        with pytest.raises(RFastError) as ei:
+            eng.run()
+        assert ei.value.code == ETIMEOUT and time.time() - t0 < 5.0
+        eng.set_option(B.OPT_PHANTOM_ARRIVALS, 0)
+        eng.reset()
+        eng.run()
+        x = eng.read(B.STATE_X)
+    assert np.linalg.norm(x - orc.X()) <= 1e-5 * np.linalg.norm(orc.X())

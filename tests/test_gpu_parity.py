@@ -251,8 +251,8 @@ def test_graph_replay_on_a_user_stream_equals_direct_launches(rfast_lib, name, o
     ("softmax_exp16", dict(n=8, F=784, C=10, rows=64, K=40, batch=32)),
 ], ids=["config 1", "ls wider", "softmax", "softmax plain", "softmax 784x10"])
 def test_persistent_kernel_equals_one_kernel_per_phase(rfast_lib, name, ov):
-    """L2-resident problems run a span of rounds as one cooperative persistent kernel with
-    bounded grid barriers; with the option off, one kernel per phase.  Same bits, and parity
+    """L2-resident problems can run a span of rounds as one cooperative persistent kernel with
+    bounded grid barriers (an option); by default, one kernel per phase.  Same bits, and parity
     with the oracle either way."""
     import paper_2307_11617_b200 as pkg
     from paper_2307_11617_b200 import binding as B
