@@ -80,6 +80,23 @@ class ClockSampler:
                 "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """The slowest rank's time: every multi-rank number is the max over ranks (replicas run
+    independently; the job is done when the last one is)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: int, world: int, seconds: float) -> float:
+    """Replicas only: every rank processes the same number of units; aggregate = sum / max time."""
+    return world * units_per_rank / seconds
+
+
 def build_workload(name, small=False):
     from workloads import build_config
     if small:
@@ -215,11 +232,8 @@ def main():
     launches = eng.query(B.Q_LAUNCHES) - l0
     ms = [a.elapsed_time(b) for a, b in pairs]
     ms_step = float(sum(ms) / len(ms))
-    if world > 1:
-        t = torch.tensor([ms_step], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    value = world * events / (ms_step * 1e-3)
+    ms_step = max_over_ranks(ms_step, "cuda")
+    value = whole_job_rate(events, world, ms_step * 1e-3)
 
     # end to end through the C ABI with host buffers: schedule arrays in (compiled and uploaded),
     # the run, x and y back into pinned host memory
@@ -240,11 +254,8 @@ def main():
             eng.read(B.STATE_Y, yo)
         barrier()
         dt = (time.perf_counter() - t0) / reps
-        if world > 1:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * events / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        dt = max_over_ranks(dt, "cuda")
+        e2e = {"value": whole_job_rate(events, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3}
 
     peak, peak_kind = measured_peaks()
