@@ -80,6 +80,23 @@ class ClockSampler:
                 "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
 
 
+# DRAM traffic / algorithmic bytes of k_fused_quad from the ncu capture summarised in
+# profiles/k_fused_quad_quad_tree64_small_ncu.md (small case; traffic grows in proportion to the
+# coordinates processed).  Valid only for the kernel source the counters were taken with.
+FUSED_TRAFFIC = {"kernels_sha256": "d5c3967c78d4aa042f23814e98e2f3a6eba604b5df2f2b18e58ca2fd962c6514", "ratio": 0.96}
+
+
+def fused_traffic_ratio():
+    import hashlib
+    path = os.path.join(ROOT, "paper_2307_11617_b200", "csrc", "kernels.cuh")
+    try:
+        if hashlib.sha256(open(path, "rb").read()).hexdigest() == FUSED_TRAFFIC["kernels_sha256"]:
+            return FUSED_TRAFFIC["ratio"]
+    except OSError:
+        pass
+    return None                      # the kernel changed since the counters were taken
+
+
 def max_over_ranks(value: float, device=None) -> float:
     """The slowest rank's time: every multi-rank number is the max over ranks (replicas run
     independently; the job is done when the last one is)."""
@@ -265,7 +282,8 @@ def main():
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
                 "algorithmic_bytes_per_launch": bytes_step / max(1, launches // max(1, args.steps)),
-                "traffic": None,
+                "traffic": (fused_traffic_ratio() and fused_traffic_ratio() * bytes_step / max(1, launches // max(1, args.steps)))
+                if wl.model == "quad_diag" else None,
                 "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
 
     cpu = None
