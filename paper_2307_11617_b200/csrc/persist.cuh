@@ -69,6 +69,54 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int& ta
     return __syncthreads_and(ok) != 0;
 }
 
+// Phase 3 of a round for one tile of kThreads float4: the sample gradient of the tile's
+// coordinates from the per-row scalars of phase 2 (softmax: delta in shared memory; least
+// squares: the residuals, staged in shared memory), stored as the new remembered gradient, then
+// S2b + S2c on the same coordinates.  sm: B*C floats + B ints (softmax) or B floats.
+template <int MODEL, bool COMP, bool CG>
+__device__ __forceinline__ void grad_track_tile(const RoundArgs& a, const GradArgs& g, const EvDesc& e, int el, int tile,
+                                                const float* feat, const int* label, const float* scratch,
+                                                int use_all, float* sm) {
+    float* delta = sm;
+    int* rowid = reinterpret_cast<int*>(sm + g.B * g.C);
+    __syncthreads();                                         // the previous item's readers are done
+    if (MODEL == RFAST_MODEL_SOFTMAX) {
+        softmax_delta_block<CG>(g, e, el, label, scratch, delta, rowid);
+    } else {
+        for (int k = threadIdx.x; k < g.B; k += kThreads) delta[k] = ld_sel1<CG>(scratch + (int64_t)el * g.B + k);
+        __syncthreads();
+    }
+    const int i4 = tile * kThreads + threadIdx.x;
+    const int64_t row = (int64_t)e.node * a.stride;
+    float4 gnv[1], gov[1], zh[1];
+    gnv[0] = gov[0] = zh[0] = make_float4(0, 0, 0, 0);
+    if (i4 < a.n4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t q = (int64_t)i4 * 4 + j;
+            float v = 0.f;
+            if (q < g.p) {
+                if (MODEL == RFAST_MODEL_SOFTMAX) {
+                    v = softmax_grad_coord<CG>(g, e, q, feat, delta, rowid);
+                } else {                                     // same order of operations as ls_grad_coord
+                    const float* abase = feat + (int64_t)e.node * g.rows * g.F;
+                    float s = 0.f;
+                    for (int k = 0; k < g.B; ++k) {
+                        const int rrow = use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
+                        s = fmaf(abase[(int64_t)rrow * g.F + q], delta[k], s);
+                    }
+                    v = s / (float)g.B + g.l2 * ld_sel1<CG>(g.x + row + q);
+                }
+            }
+            comp(gnv[0], j) = v;
+        }
+        reinterpret_cast<float4*>(g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row)[i4] = gnv[0];
+        zh[0] = ld_sel<CG>(a.z + row, i4);
+        gov[0] = ld_sel<CG>(g.gbuf + (int64_t)e.g_par * g.gplane + row, i4);
+    }
+    track_and_push<1, COMP, CG>(a, e, i4, a.z + row, zh, gnv, gov);
+}
+
 // MODEL: RFAST_MODEL_LEAST_SQUARES or RFAST_MODEL_SOFTMAX.  Launched cooperatively with
 // gridDim.x <= number of co-resident CTAs; dynamic shared memory: B*C floats + B ints (softmax) or
 // B floats (least squares: the residuals of the item's event), then stride floats for x.
@@ -138,47 +186,9 @@ k_persist_rounds(PersistArgs P) {
         if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
         // ---- phase 3: gradient per coordinate, then S2b + S2c on the same coordinates ---------------
         for (int item = blockIdx.x; item < nev * tiles; item += gridDim.x) {
-            const int el = item / tiles, tile = item % tiles;
-            const EvDesc e = a.ev[ev0 + el];
-            float* delta = sm;
-            int* rowid = reinterpret_cast<int*>(sm + g.B * g.C);
-            if (MODEL == RFAST_MODEL_SOFTMAX) {
-                __syncthreads();                             // the previous item's readers are done
-                softmax_delta_block<true>(g, e, el, P.label, P.scratch, delta, rowid);
-            } else {
-                __syncthreads();
-                for (int k = threadIdx.x; k < g.B; k += kThreads) delta[k] = __ldcg(P.scratch + (int64_t)el * g.B + k);
-                __syncthreads();
-            }
-            const int i4 = tile * kThreads + threadIdx.x;
-            const int64_t row = (int64_t)e.node * a.stride;
-            float4 gnv[1], gov[1], zh[1];
-            gnv[0] = gov[0] = zh[0] = make_float4(0, 0, 0, 0);
-            if (i4 < a.n4) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int64_t q = (int64_t)i4 * 4 + j;
-                    float v = 0.f;
-                    if (q < g.p) {
-                        if (MODEL == RFAST_MODEL_SOFTMAX) {
-                            v = softmax_grad_coord<true>(g, e, q, P.feat, delta, rowid);
-                        } else {                             // same order of operations as ls_grad_coord
-                            const float* abase = P.feat + (int64_t)e.node * g.rows * g.F;
-                            float s = 0.f;
-                            for (int k = 0; k < g.B; ++k) {
-                                const int rrow = P.use_all ? k : g.batch_idx[(int64_t)e.sample * g.B + k];
-                                s = fmaf(abase[(int64_t)rrow * g.F + q], delta[k], s);
-                            }
-                            v = s / (float)g.B + g.l2 * __ldcg(g.x + row + q);
-                        }
-                    }
-                    comp(gnv[0], j) = v;
-                }
-                reinterpret_cast<float4*>(g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row)[i4] = gnv[0];
-                zh[0] = ld_sel<true>(a.z + row, i4);
-                gov[0] = ld_sel<true>(g.gbuf + (int64_t)e.g_par * g.gplane + row, i4);
-            }
-            track_and_push<1, COMP, true>(a, e, i4, a.z + row, zh, gnv, gov);
+            const int el = item / tiles;
+            grad_track_tile<MODEL, COMP, true>(a, g, a.ev[ev0 + el], el, item % tiles, P.feat, P.label, P.scratch,
+                                               P.use_all, sm);
         }
         if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
     }
