@@ -295,14 +295,16 @@ k_mlp_logits(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, 
     float acc[16];
 #pragma unroll
     for (int c = 0; c < 16; ++c) acc[c] = 0.f;
-    for (int j = lane; j < H; j += 32) {
+    for (int j4 = lane; j4 < H / 4; j4 += 32) {
         // all loads of the iteration first, then the arithmetic: the loads then overlap
-        float w[16];
+        float4 w[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) w[c] = c < C ? W2[(int64_t)c * H + j] : 0.f;
-        const float hv = h[j];
+        for (int c = 0; c < 16; ++c)
+            w[c] = c < C ? reinterpret_cast<const float4*>(W2 + (int64_t)c * H)[j4] : make_float4(0, 0, 0, 0);
+        const float4 hv = reinterpret_cast<const float4*>(h)[j4];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) acc[c] = fmaf(hv, w[c], acc[c]);
+        for (int c = 0; c < 16; ++c)
+            acc[c] = fmaf(hv.w, w[c].w, fmaf(hv.z, w[c].z, fmaf(hv.y, w[c].y, fmaf(hv.x, w[c].x, acc[c]))));
     }
     float lg[16], m = -3.0e38f;
 #pragma unroll
@@ -319,13 +321,16 @@ k_mlp_logits(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, 
 }
 
 // Backward through the output layer for a slab of 128 hidden units: gW2, gb1, dpre and its
-// bf16 transpose for the second big product; the first slab also sums gb2.
-// grid = (H / 128, events), 128 threads; dynamic shared memory: B * C floats
-__global__ void __launch_bounds__(128)
+// bf16 transpose for the second big product; the first slab also sums gb2.  A thread owns one
+// hidden unit and a quarter of the batch; the four partial sums are added in a fixed order.
+// grid = (H / 128, events), 512 threads; dynamic shared memory: B*C + 4*128*17 floats
+__global__ void __launch_bounds__(512)
 k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
            const float* __restrict__ hf, const float* __restrict__ dlog, __nv_bfloat16* __restrict__ dpqT,
            float* __restrict__ gbuf, int64_t gplane, int F, int H, int C, float l2) {
-    extern __shared__ float dl[];            // [B][C]
+    extern __shared__ float smb[];
+    float* dl = smb;                          // [B][C]
+    float* part = smb + kBatch * C;           // [4][128][17]: gw2[0..15], gb1
     const int ev = blockIdx.y;
     const EvDesc e = evs[ev];
     const int64_t row = (int64_t)e.node * stride;
@@ -333,20 +338,22 @@ k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t 
     const float* h = hf + (int64_t)ev * kBatch * H;
     const float* W2 = x + row + oW2;
     float* g = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
-    for (int q = threadIdx.x; q < kBatch * C; q += 128) dl[q] = dlog[(int64_t)ev * kBatch * C + q];
+    for (int q = threadIdx.x; q < kBatch * C; q += 512) dl[q] = dlog[(int64_t)ev * kBatch * C + q];
     __syncthreads();
     if (blockIdx.x == 0 && threadIdx.x < C) {
         float s = 0.f;
         for (int k = 0; k < kBatch; ++k) s += dl[k * C + threadIdx.x];
         g[ob2 + threadIdx.x] = s + l2 * x[row + ob2 + threadIdx.x];
     }
-    const int j = blockIdx.x * 128 + threadIdx.x;
+    const int jl = threadIdx.x & 127, kq = threadIdx.x >> 7;
+    const int j = blockIdx.x * 128 + jl;
     float w2[16], gw2[16];
 #pragma unroll
     for (int c = 0; c < 16; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
     float gb1 = 0.f;
     __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch;
-    for (int k0 = 0; k0 < kBatch; k0 += 8) {
+    constexpr int kQuarter = kBatch / 4;
+    for (int k0 = kq * kQuarter; k0 < (kq + 1) * kQuarter; k0 += 8) {
         __align__(16) __nv_bfloat16 pack[8];
         float hv[8];
 #pragma unroll
@@ -365,10 +372,23 @@ k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t 
         }
         *reinterpret_cast<uint4*>(drow + k0) = *reinterpret_cast<const uint4*>(pack);
     }
-    g[(int64_t)H * F + j] = gb1 + l2 * x[row + (int64_t)H * F + j];
+    float* mine = part + ((int64_t)kq * 128 + jl) * 17;
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-        if (c < C) g[oW2 + (int64_t)c * H + j] = gw2[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
+    for (int c = 0; c < 16; ++c) mine[c] = gw2[c];
+    mine[16] = gb1;
+    __syncthreads();
+    if (kq == 0) {
+        float tot[17];
+#pragma unroll
+        for (int c = 0; c < 17; ++c) tot[c] = part[(int64_t)jl * 17 + c];
+        for (int qd = 1; qd < 4; ++qd)
+#pragma unroll
+            for (int c = 0; c < 17; ++c) tot[c] += part[((int64_t)qd * 128 + jl) * 17 + c];
+        g[(int64_t)H * F + j] = tot[16] + l2 * x[row + (int64_t)H * F + j];
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+            if (c < C) g[oW2 + (int64_t)c * H + j] = tot[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
+    }
 }
 
 // One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A).
@@ -566,7 +586,7 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
         p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
     k_mlp_logits<<<dim3(kBatch / 8, n_events), 256, 0, st>>>(
         g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dlog, p->rows, p->F, p->H, p->C);
-    k_mlp_back<<<dim3(p->H / 128, n_events), 128, kBatch * p->C * sizeof(float), st>>>(
+    k_mlp_back<<<dim3(p->H / 128, n_events), 512, (kBatch * p->C + 4 * 128 * 17) * sizeof(float), st>>>(
         g.ev, g.x, g.stride, p->hf, p->dlog, p->dpqT, g.gbuf, g.gplane, p->F, p->H, p->C, g.l2);
     k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
         p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);

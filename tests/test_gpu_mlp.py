@@ -32,7 +32,11 @@ def _blocks(wl):
 
 @pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
 def test_mlp_gradient_from_identical_state(rfast_lib, ov):
-    """Initial gradients (same x0 on both sides): every block to fp32 accuracy."""
+    """Initial gradients (same x0 on both sides).  b1, W2, b2 see no rounded computed operand
+    and agree to fp32 accuracy.  gW1 = q(dpre)^T q(A) rounds the computed dpre to bf16: where
+    fp32 and fp64 accumulation leave dpre on different sides of a rounding boundary (about one
+    element in 4e4) that element differs by one bf16 ulp, ~3e-5 of the block per flip, so the
+    block is held to 1e-4."""
     import paper_2307_11617_b200 as pkg
     from paper_2307_11617_b200 import binding as B
     wl = build_config("mlp_tree64", seed=1, **ov)
@@ -44,8 +48,8 @@ def test_mlp_gradient_from_identical_state(rfast_lib, ov):
     ref = np.stack([m.grad(i, wl.x0[i].astype(np.float64), wl.schedule.batch_idx[i * Bs:(i + 1) * Bs])
                     for i in range(wl.n)])
     for nm, (a, b) in _blocks(wl).items():
-        assert rel_l2(g[:, a:b], ref[:, a:b]) <= 1e-5, nm
-    assert rel_l2(g, ref) <= 2e-6
+        assert rel_l2(g[:, a:b], ref[:, a:b]) <= (1e-4 if nm == "W1" else 1e-5), nm
+    assert rel_l2(g, ref) <= 1e-4
 
 
 @pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
