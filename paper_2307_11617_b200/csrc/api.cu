@@ -556,7 +556,6 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
     a.out_cur = ctx->d_out_cur; a.out_new = ctx->d_out_new; a.out_a = ctx->d_out_a;
     a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
     a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
-    const bool big = a.n4 >= kThreads * 4;
     for (int r = r0; r < r1; ++r) {
         const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
         if (nev == 0) continue;
@@ -564,7 +563,6 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
         if (!ctx->alpha_round.empty()) a.alpha = ctx->alpha_round[r];
         if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
             if (ctx->compensated) k_fused_quad<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
-            else if (big) k_fused_quad<2, false><<<tile_grid(a.n4, 2, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             else k_fused_quad<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             ctx->launches += 1;
         } else {

@@ -219,8 +219,10 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
 // last consumed, kept alive instead of copied).  One HBM pass per activation.
 // grid = (tiles, events of the round)
 // ---------------------------------------------------------------------------------------------
+// (at most 42 registers per thread: six CTAs per SM keep enough loads in flight; measured +4 %
+// over five, +9 % over the two-float4-per-thread variant at three)
 template <int U, bool COMP>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 6)
 k_fused_quad(RoundArgs a, const float* __restrict__ qd, const float* __restrict__ qb) {
     const EvDesc e = a.ev[blockIdx.y];
     const int64_t row = (int64_t)e.node * a.stride;
