@@ -83,16 +83,25 @@ class ClockSampler:
 # DRAM traffic / algorithmic bytes of k_fused_quad from the ncu capture summarised in
 # profiles/k_fused_quad_quad_tree64_small_ncu.md (small case; traffic grows in proportion to the
 # coordinates processed).  Valid only for the kernel source the counters were taken with.
-FUSED_TRAFFIC = {"kernels_sha256": "65dbd72182ffee31503bbf7923ef7b0febf3f9a9b7e825e5140b4cb75109ae82", "ratio": 0.96}
+FUSED_TRAFFIC = {"kernel_sha256": "abc7c3e12905992d6c1afeccf7191c5ef6c8874386b98f10f73e98e9184fad01", "ratio": 0.96}
+
+
+def _fused_kernel_source():
+    """The part of kernels.cuh that the fused kernel is made of: load/store helpers, the shared
+    tracking tail and k_fused_quad itself."""
+    path = os.path.join(ROOT, "paper_2307_11617_b200", "csrc", "kernels.cuh")
+    text = open(path).read()
+    a = text.index("__device__ __forceinline__ float4 ld_stream")
+    b = text.index("// z_i^0 = grad f_i(x_i^0) for the element-wise objective.")
+    return text[a:b]
 
 
 def fused_traffic_ratio():
     import hashlib
-    path = os.path.join(ROOT, "paper_2307_11617_b200", "csrc", "kernels.cuh")
     try:
-        if hashlib.sha256(open(path, "rb").read()).hexdigest() == FUSED_TRAFFIC["kernels_sha256"]:
+        if hashlib.sha256(_fused_kernel_source().encode()).hexdigest() == FUSED_TRAFFIC["kernel_sha256"]:
             return FUSED_TRAFFIC["ratio"]
-    except OSError:
+    except (OSError, ValueError):
         pass
     return None                      # the kernel changed since the counters were taken
 

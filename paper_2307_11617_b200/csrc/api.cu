@@ -568,9 +568,9 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
         } else {
             const int64_t gplane = (int64_t)ctx->n * ctx->stride;
             if (ctx->model == RFAST_MODEL_MLP)
-                k_mix<1, true, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb, nullptr, 0, 0.f);
+                k_mix<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb);
             else
-                k_mix<1, false, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr, nullptr, 0, 0.f);
+                k_mix<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr);
             ctx->launches += 1;
             int rc = launch_gradients(ctx, a.ev, nev);
             if (rc != RFAST_OK) return rc;

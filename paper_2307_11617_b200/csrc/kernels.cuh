@@ -295,12 +295,10 @@ k_quad_grad(const float* __restrict__ x, const float* __restrict__ qd, const flo
 
 // ---------------------------------------------------------------------------------------------
 // S1 + S2a for objectives whose gradient needs the whole new x first.  Optionally leaves a
-// bf16 copy of the new x (operand of the MLP's matrix products), or starts the new gradient
-// row with the dense term l2 * x (sparse objective).  grid = (tiles, events)
+// bf16 copy of the new x (operand of the MLP's matrix products).  grid = (tiles, events)
 // ---------------------------------------------------------------------------------------------
-template <int U, bool BF16, bool GINIT, bool CG>
-__device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, int tile, __nv_bfloat16* xb,
-                                         float* gbuf, int64_t gplane, float l2) {
+template <int U, bool BF16, bool CG>
+__device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, int tile, __nv_bfloat16* xb) {
     const int64_t row = (int64_t)e.node * a.stride;
     float* xr = a.x + row;
     const float* zr = a.z + row;
@@ -337,8 +335,6 @@ __device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, in
         if (i4 < a.n4) {
             // the gradient kernels re-read x soon: keep it cacheable
             reinterpret_cast<float4*>(xr)[i4] = acc[u];
-            if (GINIT)      // dense part of a sparse objective's gradient: g_new = l2 * x_new
-                reinterpret_cast<float4*>(gbuf + (int64_t)(e.g_par ^ 1) * gplane + row)[i4] = f4_scale(l2, acc[u]);
             if (BF16) {
                 __nv_bfloat162 lo = __floats2bfloat162_rn(acc[u].x, acc[u].y);
                 __nv_bfloat162 hi = __floats2bfloat162_rn(acc[u].z, acc[u].w);
@@ -351,10 +347,10 @@ __device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, in
     }
 }
 
-template <int U, bool BF16, bool GINIT>
+template <int U, bool BF16>
 __global__ void __launch_bounds__(kThreads)
-k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb, float* __restrict__ gbuf, int64_t gplane, float l2) {
-    mix_tile<U, BF16, GINIT, false>(a, a.ev[blockIdx.y], blockIdx.x, xb, gbuf, gplane, l2);
+k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
+    mix_tile<U, BF16, false>(a, a.ev[blockIdx.y], blockIdx.x, xb);
 }
 
 // ---------------------------------------------------------------------------------------------

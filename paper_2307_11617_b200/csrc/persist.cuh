@@ -135,7 +135,7 @@ k_persist_rounds(PersistArgs P) {
         // ---- phase 1: S1 + S2a ----------------------------------------------------------------
         for (int item = blockIdx.x; item < nev * tiles; item += gridDim.x) {
             const EvDesc e = a.ev[ev0 + item / tiles];
-            mix_tile<1, false, false, true>(a, e, item % tiles, nullptr, nullptr, 0, 0.f);
+            mix_tile<1, false, true>(a, e, item % tiles, nullptr);
         }
         if (!grid_barrier(P.bar, target, P.status, gridDim.x + P.phantom, P.limit_ns)) return;
         // ---- phase 2: per-row scalars of the sample gradient --------------------------------------

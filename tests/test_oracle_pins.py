@@ -359,3 +359,19 @@ def test_convergence_under_acknowledgement_gated_loss():
     assert np.linalg.norm(orc.X() - xstar) <= 1e-8 * np.linalg.norm(xstar)
     # the identity of Lemma 3 holds to rounding of the running sums it is made of
     assert np.abs(orc.conservation_residual()).max() <= 1e-13 * max(1.0, np.abs(orc.RHO()).max()) * 100
+
+
+def test_oracle_reproduces_its_frozen_output_on_config_1(repo_root):
+    """Regression guard (not a pin by the paper, which prints no iterates): the stored output of
+    tests/golden/make_golden.py, which calls only the oracle and the seeded generators."""
+    import os
+    gold = os.path.join(repo_root, "tests", "golden")
+    wl = build_config("ls_ring4", seed=0)
+    orc = from_workload(wl, make_model(wl).grad)
+    run_schedule(orc, wl.schedule)
+    x = np.loadtxt(os.path.join(gold, "ls_ring4_x_after_200_rounds.txt"))
+    z = np.loadtxt(os.path.join(gold, "ls_ring4_z_after_200_rounds.txt"))
+    st = np.loadtxt(os.path.join(gold, "ls_ring4_stamps.txt"), dtype=np.int64)
+    assert np.abs(orc.X() - x).max() <= 1e-13 * np.abs(x).max()
+    assert np.abs(orc.Z() - z).max() <= 1e-13 * np.abs(z).max()
+    assert st.tolist() == orc.t + orc.tau_v + orc.tau_rho
