@@ -273,3 +273,48 @@ def test_persistent_kernel_equals_one_kernel_per_phase(rfast_lib, name, ov):
     for u, v in zip(res[1][:4], res[0][:4]):
         assert np.array_equal(u, v)
     assert res[1][4] == 3 and res[0][4] > 3 * 7       # one launch per span against several per round
+
+
+def _general_digraphs(n, rng, extra):
+    """Ring plus random chords: several in- and out-neighbours per node in both graphs, weights
+    1/3, 1/4, ... that are not exact in binary."""
+    from workloads import graph_from_edges
+    def edges():
+        e = {(i, (i + 1) % n) for i in range(n)}
+        while len(e) < n + extra:
+            a, b = rng.integers(0, n, size=2)
+            if a != b:
+                e.add((int(a), int(b)))
+        return e
+    return graph_from_edges(n, edges(), "row"), graph_from_edges(n, edges(), "col")
+
+
+@pytest.mark.parametrize("name,ov,comp", [
+    ("quad_tree64", dict(n=12, p=5003, K=50), False),
+    ("quad_tree64", dict(n=12, p=5003, K=50), True),
+    ("softmax_exp16", dict(n=12, F=40, C=5, rows=32, K=60, batch=8), True),
+    ("logistic_tree1024", dict(n=12, p=3000, rows=8, K=50, batch=4, nnz=30), False),
+], ids=["quad", "quad compensated", "softmax compensated", "logistic"])
+def test_parity_on_general_digraphs(rfast_lib, name, ov, comp):
+    """Not only trees and rings: several in-neighbours in G_R (S2a sums more than one packet),
+    several in- and out-neighbours in G_C (S2b consumes several running sums, S2c feeds several)."""
+    import paper_2307_11617_b200 as pkg
+    from workloads import activation_bernoulli, make_schedule
+    wl = build_config(name, seed=11, **ov)
+    rng = np.random.default_rng(12)
+    wl.G_R, wl.G_C = _general_digraphs(wl.n, rng, 2 * wl.n)
+    assert np.diff(wl.G_R.rowptr).max() >= 3 and np.bincount(wl.G_C.col).max() >= 3
+    wl.schedule = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(wl.n, wl.schedule.K, 0.6, rng), 0.25, 3,
+                                rng, batch=wl.batch, rows_per_node=wl.rows)
+    wl.compensated = comp
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        from paper_2307_11617_b200 import binding as B
+        assert eng.read(B.STATE_USED_TAU_V).tolist() == orc.used_tau_v
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
+        d = eng.diagnostics()
+    scale = np.abs(orc.G()).sum(axis=0).max()
+    assert d["conservation_residual"] <= 2e-5 * scale
