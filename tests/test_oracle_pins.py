@@ -241,21 +241,31 @@ def test_consumed_stamps_match_brute_force(seed):
 # ---------------------------------------------------------------------------------------------
 # P5  Appendices E-F: the augmented systems as dense matrices, one active node per iteration
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("seed", [0, 1, 2])
-def test_augmented_systems_dense(seed):
+@pytest.mark.parametrize("seed,multi", [(0, False), (1, False), (2, False), (3, True), (4, True)])
+def test_augmented_systems_dense(seed, multi):
+    """multi = False: one active node per round, Algorithm 2 as printed.  multi = True: rounds
+    with several active nodes, checked against Algorithm 2 run once per member in ascending id
+    (global iteration = event index): members of a round must not see each other's output, which
+    in the global view is simply a larger delay."""
     rng = _rng(100 + seed)
-    n, p, K = 4, 3, 16
+    n, p, K = 4, 3, (10 if multi else 16)
     G_R, G_C = (f64_weights(g) for g in _general_graphs(n, rng))
     W, A = G_R.dense(), G_C.dense()
-    act = [np.array([int(rng.integers(0, n))], dtype=np.int32) for _ in range(K)]
+    if multi:
+        act = activation_uniform_subset(n, K, 1, n, rng)
+    else:
+        act = [np.array([int(rng.integers(0, n))], dtype=np.int32) for _ in range(K)]
     sch = make_schedule(G_R, G_C, act, 0.3, 2, rng)
     d = rng.uniform(0.5, 2, (n, p)); b = rng.standard_normal((n, p)); x0 = rng.standard_normal((n, p))
     gamma = 0.03
     orc = RFastOracle(n, p, gamma, G_R, G_C, QuadDiag(d, b).grad, x0=x0)
 
-    sv, rounds_R = brute_force_stamps(G_R, sch, sch.send_r)
-    sr, rounds_C = brute_force_stamps(G_C, sch, sch.send_c)
-    D = K + 1
+    sv, _ = brute_force_stamps(G_R, sch, sch.send_r)
+    sr, _ = brute_force_stamps(G_C, sch, sch.send_c)
+    events = [(r, int(i)) for r in range(K) for i in act[r]]        # global iteration k = event index
+    ev_idx = [[k for k, (_, i) in enumerate(events) if i == j] for j in range(n)]
+    rounds_R = rounds_C = ev_idx
+    D = len(events) + 1
     E = G_C.n_edges
     grad = lambda i, x: d[i] * d[i] * (x - b[i])
 
@@ -268,8 +278,7 @@ def test_augmented_systems_dense(seed):
     snaps = []
     run_schedule(orc, sch, after_round=lambda o, r: snaps.append(
         (o.X().copy(), o.Z().copy(), o.RHO() - o.RHO_TILDE())))
-    for k in range(K):
-        i = int(act[k][0])
+    for k, (rnd, i) in enumerate(events):
         # delays in the global view: d = k - g(j, tau - 1) - 1; "nothing received yet" reads a
         # slot that still holds the zero initial value
         What = np.zeros(((D + 2) * n,) * 2)
@@ -318,7 +327,9 @@ def test_augmented_systems_dense(seed):
         assert np.allclose(Pk.sum(axis=0), 1) and np.allclose(Sk.sum(axis=0), 1)
         zhalf = Sk @ zhat; zhalf[i] += eps
         zhat = Pk @ zhalf
-        X, Z, M = snaps[k]
+        if k + 1 < len(events) and events[k + 1][0] == rnd:
+            continue                                     # compare at the end of each round
+        X, Z, M = snaps[rnd]
         assert np.abs(h[:n] - X).max() < 1e-12
         assert np.abs(zhat[:n] - Z).max() < 1e-12
         mass = zhat[n:].reshape(D + 1, E, p).sum(axis=0)
