@@ -446,7 +446,16 @@ __device__ __forceinline__ void softmax_logits_row(const GradArgs& g, const EvDe
     for (int c = warp; c < g.C; c += 8) {
         const float* w = x + (int64_t)c * g.F;
         float s = 0.f;
-        for (int f = lane; f < g.F; f += 32) s = fmaf(a[f], ld_sel1<CG>(w + f), s);
+        if ((g.F & 3) == 0) {                                // rows are 16-byte aligned: 128-bit loads
+            for (int f4 = lane; f4 < g.F / 4; f4 += 32) {
+                const float4 av = reinterpret_cast<const float4*>(a)[f4];
+                const float4 wv = CG ? __ldcg(reinterpret_cast<const float4*>(w) + f4)
+                                     : reinterpret_cast<const float4*>(w)[f4];
+                s = fmaf(av.w, wv.w, fmaf(av.z, wv.z, fmaf(av.y, wv.y, fmaf(av.x, wv.x, s))));
+            }
+        } else {
+            for (int f = lane; f < g.F; f += 32) s = fmaf(a[f], ld_sel1<CG>(w + f), s);
+        }
         s = warp_sum(s);
         if (lane == 0) logit[((int64_t)ev_local * g.B + k) * g.C + c] = s + ld_sel1<CG>(x + (int64_t)g.C * g.F + c);
     }
@@ -484,6 +493,7 @@ __device__ __forceinline__ float softmax_grad_coord(const GradArgs& g, const EvD
     if (q < (int64_t)g.C * g.F) {
         const int c = (int)(q / g.F), f = (int)(q % g.F);
         const float* abase = feat + (int64_t)e.node * g.rows * g.F;
+#pragma unroll 8
         for (int k = 0; k < g.B; ++k) s = fmaf(delta[k * g.C + c], abase[(int64_t)rowid[k] * g.F + f], s);
     } else {
         const int c = (int)(q - (int64_t)g.C * g.F);

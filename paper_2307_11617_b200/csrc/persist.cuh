@@ -175,7 +175,15 @@ k_persist_rounds(PersistArgs P) {
                         for (int c = warp; c < g.C; c += 8) {
                             const float* w = xs + (int64_t)c * g.F;
                             float s = 0.f;
-                            for (int f = lane; f < g.F; f += 32) s = fmaf(arow[f], w[f], s);
+                            if ((g.F & 3) == 0) {            // same order of operations as softmax_logits_row
+                                for (int f4 = lane; f4 < g.F / 4; f4 += 32) {
+                                    const float4 av = reinterpret_cast<const float4*>(arow)[f4];
+                                    const float4 wv = reinterpret_cast<const float4*>(w)[f4];
+                                    s = fmaf(av.w, wv.w, fmaf(av.z, wv.z, fmaf(av.y, wv.y, fmaf(av.x, wv.x, s))));
+                                }
+                            } else {
+                                for (int f = lane; f < g.F; f += 32) s = fmaf(arow[f], w[f], s);
+                            }
                             s = warp_sum(s);
                             if (lane == 0) P.scratch[((int64_t)el * g.B + k) * g.C + c] = s + xs[(int64_t)g.C * g.F + c];
                         }
