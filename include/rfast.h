@@ -97,7 +97,10 @@ typedef struct rfast_problem {
     int32_t     compensated;  /* tracker arithmetic of S2b/S2c: 0 = plain fp32; 1 = the tracker is  */
                               /* carried as a sum of two floats and the rounding errors of the      */
                               /* mass-moving operations are fed back (keeps the conservation of      */
-                              /* Lemma 3 over long horizons; one more fp32 stream read and written) */
+                              /* Lemma 3 over long horizons; one more fp32 stream read and written); */
+                              /* 2 = the running sums rho are two floats as well (their fp32         */
+                              /* resolution otherwise limits what a receiver sees once they have     */
+                              /* grown; doubles the rho traffic)                                     */
 } rfast_problem;
 
 /* Raw schedule (value independent).  Round r activates the nodes

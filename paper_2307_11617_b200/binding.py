@@ -116,7 +116,7 @@ def _problem(wl, keep):
     P.G_R, P.G_C = _graph(wl.G_R, keep), _graph(wl.G_C, keep)
     P.model = MODEL_IDS[wl.model] if isinstance(wl.model, str) else int(wl.model)
     P.batch, P.rows = int(wl.batch), int(wl.rows)
-    P.compensated = 1 if getattr(wl, "compensated", False) else 0
+    P.compensated = int(getattr(wl, "compensated", 0) or 0)     # False/True/2 -> 0/1/2
     dims = getattr(wl, "dims", {}) or {}
     P.n_features = int(dims.get("n_features", 0))
     P.n_classes = int(dims.get("n_classes", 0))

@@ -38,6 +38,8 @@ struct rfast_ctx {
     // device state
     float *x = nullptr, *z = nullptr, *zc = nullptr, *gbuf = nullptr, *x0 = nullptr;
     bool compensated = false;
+    bool rho2 = false;                // compensation level 2: two-float running sums
+    int64_t rlo_off() const { return rho2 ? (int64_t)comp.n_rho_slots * stride : 0; }
     float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
     int* label = nullptr;
     int64_t* sp_ptr = nullptr;
@@ -347,6 +349,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
     ctx->model = prob->model; ctx->batch = prob->batch; ctx->rows = prob->rows;
     ctx->F = prob->n_features; ctx->C = prob->n_classes; ctx->H = prob->n_hidden;
     ctx->compensated = prob->compensated != 0;
+    ctx->rho2 = prob->compensated >= 2;
     ctx->stride = (prob->p + 31) / 32 * 32;
     if (ctx->stride / 4 > 0x7fffffff) return set_err(ctx, RFAST_EINVAL, "p too large");
     if ((rc = build_host_graph(prob->G_R, ctx->n, true, ctx->R, err)) != RFAST_OK) return set_err(ctx, rc, "G_R: " + err);
@@ -496,9 +499,9 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     }
     if ((rc = upload(ctx, &ctx->d_init_ev, init))) return rc;
     CK(dev_alloc(ctx, &ctx->vbuf, (size_t)c.n_v_slots * ctx->stride, true));
-    CK(dev_alloc(ctx, &ctx->rbuf, (size_t)c.n_rho_slots * ctx->stride, true));
+    CK(dev_alloc(ctx, &ctx->rbuf, (size_t)c.n_rho_slots * ctx->stride * (ctx->rho2 ? 2 : 1), true));
     CK(cudaMemsetAsync(ctx->vbuf, 0, std::max<size_t>(1, (size_t)c.n_v_slots * ctx->stride) * sizeof(float), ctx->stream));
-    CK(cudaMemsetAsync(ctx->rbuf, 0, std::max<size_t>(1, (size_t)c.n_rho_slots * ctx->stride) * sizeof(float), ctx->stream));
+    CK(cudaMemsetAsync(ctx->rbuf, 0, std::max<size_t>(1, (size_t)c.n_rho_slots * ctx->stride * (ctx->rho2 ? 2 : 1)) * sizeof(float), ctx->stream));
     // scratch of the two-phase gradients: residuals / logits / coefficients per (event, row[, class])
     size_t per_ev = 0;
     if (ctx->model == RFAST_MODEL_LEAST_SQUARES) per_ev = ctx->batch ? ctx->batch : ctx->rows;
@@ -554,7 +557,7 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
     a.mix_slot = ctx->d_mix_slot; a.mix_w = ctx->d_mix_w;
     a.news_new = ctx->d_news_new; a.news_prev = ctx->d_news_prev;
     a.out_cur = ctx->d_out_cur; a.out_new = ctx->d_out_new; a.out_a = ctx->d_out_a;
-    a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf;
+    a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf; a.rlo_off = ctx->rlo_off();
     a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
     for (int r = r0; r < r1; ++r) {
         const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
@@ -603,7 +606,7 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         P.a.mix_slot = ctx->d_mix_slot; P.a.mix_w = ctx->d_mix_w;
         P.a.news_new = ctx->d_news_new; P.a.news_prev = ctx->d_news_prev;
         P.a.out_cur = ctx->d_out_cur; P.a.out_new = ctx->d_out_new; P.a.out_a = ctx->d_out_a;
-        P.a.x = ctx->x; P.a.z = ctx->z; P.a.zc = ctx->zc; P.a.vbuf = ctx->vbuf; P.a.rbuf = ctx->rbuf;
+        P.a.x = ctx->x; P.a.z = ctx->z; P.a.zc = ctx->zc; P.a.vbuf = ctx->vbuf; P.a.rbuf = ctx->rbuf; P.a.rlo_off = ctx->rlo_off();
         P.a.stride = ctx->stride; P.a.n4 = (int)(ctx->stride / 4); P.a.alpha = ctx->alpha;
         P.a.ev = ctx->d_ev;
         P.g = grad_args(ctx, ctx->d_ev);
@@ -835,7 +838,7 @@ std::vector<std::pair<void*, size_t>> state_buffers(rfast_ctx* c) {
     if (c->gbuf) v.push_back({c->gbuf, 2 * plane});
     if (c->xb) v.push_back({c->xb, plane / 2});
     v.push_back({c->vbuf, (size_t)c->comp.n_v_slots * c->stride * sizeof(float)});
-    v.push_back({c->rbuf, (size_t)c->comp.n_rho_slots * c->stride * sizeof(float)});
+    v.push_back({c->rbuf, (size_t)c->comp.n_rho_slots * c->stride * sizeof(float) * (c->rho2 ? 2 : 1)});
     return v;
 }
 
@@ -843,7 +846,7 @@ CkptHeader make_header(rfast_ctx* c) {
     CkptHeader h{};
     h.magic = kCkptMagic; h.sched_hash = c->sched_hash;
     h.p = c->p; h.stride = c->stride; h.n_events = c->comp.n_events;
-    h.n = c->n; h.model = c->model; h.compensated = c->compensated; h.K = c->comp.K;
+    h.n = c->n; h.model = c->model; h.compensated = c->compensated + (c->rho2 ? 1 : 0); h.K = c->comp.K;
     h.n_v_slots = c->comp.n_v_slots; h.n_rho_slots = c->comp.n_rho_slots; h.round = c->round;
     return h;
 }
@@ -929,7 +932,7 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     cudaMemcpyAsync(d_latest, latest.data(), latest.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
     cudaMemcpyAsync(d_buf, buf.data(), buf.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
     k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
-                                                          ctx->quad_b, ctx->rbuf, d_latest, d_buf, n, E,
+                                                          ctx->quad_b, ctx->rbuf, ctx->rlo_off(), d_latest, d_buf, n, E,
                                                           ctx->stride, ctx->p, d_part);
     std::vector<double> part((size_t)blocks * 5);
     cudaError_t e = cudaMemcpyAsync(part.data(), d_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream);

@@ -24,6 +24,8 @@ struct RoundArgs {
     float* zc;                   // [n][stride] low-order part of the tracker (compensated mode), else null
     float* vbuf;                 // [v rows][stride]   published v versions
     float* rbuf;                 // [rho rows][stride] running-sum versions
+    int64_t rlo_off;             // > 0: the running sums are two floats; low parts live this many
+                                 // floats after the high parts (compensation level 2)
     int64_t stride;              // floats per row
     int     n4;                  // float4 per row (stride / 4)
     float   alpha;
@@ -78,7 +80,10 @@ constexpr int kThreads = 256;
 // rounding error of the mass-moving operations (the additions into z^, the products with the
 // weights, the additions into the running sums) is captured with error-free transformations
 // and kept in the node's own low-order part, so that the tracked mass of Lemma 3 is conserved
-// to second order instead of drifting with every fp32 rounding.  The running sums stay fp32.
+// to second order instead of drifting with every fp32 rounding.  The running sums stay fp32,
+// unless a.rlo_off > 0: then they are two floats as well, which removes the last fp32-sized
+// quantity from the tracking path (a receiver otherwise sees its in-neighbours' mass at the
+// resolution of an fp32 sum that keeps growing).
 // ---------------------------------------------------------------------------------------------
 template <int U, bool COMP, bool CG = false>
 __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc& e, int base, float* zr,
@@ -143,13 +148,18 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
                 if (i4 < a.n4) {
                     const float4 nv = ld_sel<CG>(nr, i4);
                     const float4 pv = prev >= 0 ? ld_sel<CG>(pr, i4) : make_float4(0, 0, 0, 0);
+                    float4 nl = make_float4(0, 0, 0, 0), pl = nl;
+                    if (a.rlo_off > 0) {
+                        nl = ld_sel<CG>(nr + a.rlo_off, i4);
+                        if (prev >= 0) pl = ld_sel<CG>(pr + a.rlo_off, i4);
+                    }
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         float d, de, s, se;
                         two_sum(comp(nv, c), -comp(pv, c), d, de);
                         two_sum(comp(hi[u], c), d, s, se);
                         comp(hi[u], c) = s;
-                        comp(lo[u], c) += se + de;
+                        comp(lo[u], c) += se + de + (comp(nl, c) - comp(pl, c));
                     }
                 }
             }
@@ -183,14 +193,28 @@ __device__ __forceinline__ void track_and_push(const RoundArgs& a, const EvDesc&
                 if (i4 < a.n4) {
                     const float4 cv = cur >= 0 ? ld_sel<CG>(cr, i4) : make_float4(0, 0, 0, 0);
                     float4 r;
+                    if (a.rlo_off > 0) {                     // two-float running sum: nothing is left over
+                        const float4 cl = cur >= 0 ? ld_sel<CG>(cr + a.rlo_off, i4) : make_float4(0, 0, 0, 0);
+                        float4 rl;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const float inc = __fmul_rn(aw, comp(zh_hi[u], c));
-                        const float ierr = __fmaf_rn(aw, comp(zh_hi[u], c), -inc) + aw * comp(zh_lo[u], c);
-                        float s, se;
-                        two_sum(comp(cv, c), inc, s, se);
-                        comp(r, c) = s;
-                        comp(k_lo[u], c) += se + ierr;       // what did not fit stays with the sender
+                        for (int c = 0; c < 4; ++c) {
+                            const float inc = __fmul_rn(aw, comp(zh_hi[u], c));
+                            const float ierr = __fmaf_rn(aw, comp(zh_hi[u], c), -inc) + aw * comp(zh_lo[u], c);
+                            float s, se;
+                            two_sum(comp(cv, c), inc, s, se);
+                            two_sum(s, comp(cl, c) + se + ierr, comp(r, c), comp(rl, c));
+                        }
+                        st_stream(wr + a.rlo_off, i4, rl);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const float inc = __fmul_rn(aw, comp(zh_hi[u], c));
+                            const float ierr = __fmaf_rn(aw, comp(zh_hi[u], c), -inc) + aw * comp(zh_lo[u], c);
+                            float s, se;
+                            two_sum(comp(cv, c), inc, s, se);
+                            comp(r, c) = s;
+                            comp(k_lo[u], c) += se + ierr;   // what did not fit stays with the sender
+                        }
                     }
                     st_stream(wr, i4, r);
                 }
@@ -657,7 +681,7 @@ __global__ void __launch_bounds__(kThreads)
 k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const float* __restrict__ zc,
               const float* __restrict__ gpool, const int* __restrict__ gsel,
               const float* __restrict__ qd, const float* __restrict__ qb,
-              const float* __restrict__ rbuf, const int* __restrict__ rho_latest,
+              const float* __restrict__ rbuf, int64_t rlo_off, const int* __restrict__ rho_latest,
               const int* __restrict__ rho_buf, int n, int n_edges, int64_t stride, int64_t p,
               double* __restrict__ part) {
     __shared__ double red[5][kThreads];
@@ -676,8 +700,14 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
         }
         double mass = 0;
         for (int e = 0; e < n_edges; ++e) {
-            if (rho_latest[e] >= 0) mass += (double)rbuf[(int64_t)rho_latest[e] * stride + c];
-            if (rho_buf[e] >= 0) mass -= (double)rbuf[(int64_t)rho_buf[e] * stride + c];
+            if (rho_latest[e] >= 0) {
+                mass += (double)rbuf[(int64_t)rho_latest[e] * stride + c];
+                if (rlo_off > 0) mass += (double)rbuf[(int64_t)rho_latest[e] * stride + rlo_off + c];
+            }
+            if (rho_buf[e] >= 0) {
+                mass -= (double)rbuf[(int64_t)rho_buf[e] * stride + c];
+                if (rlo_off > 0) mass -= (double)rbuf[(int64_t)rho_buf[e] * stride + rlo_off + c];
+            }
         }
         const double xbar = sx / n;
         cons = sx2 - n * xbar * xbar;

@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 CASES = [
     ("quad_tree64", dict(n=16, p=3000, K=30)),
-    ("softmax_exp16", dict(F=40, C=5, rows=32, K=40, batch=8)),          # compensated tracker
+    ("softmax_exp16", dict(F=40, C=5, rows=32, K=40, batch=8)),          # two-float tracker
+    ("ls_ring4", dict(K=60)),                                            # two-float tracker and running sums
     ("logistic_tree1024", dict(n=48, p=2500, rows=8, K=30, batch=4, nnz=30)),
     ("mlp_tree64", dict(n=5, F=64, H=128, C=4, rows=96, K=12, batch=64)),
 ]

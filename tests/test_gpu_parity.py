@@ -100,25 +100,28 @@ def test_parity_round_by_round_and_reset(rfast_lib):
         assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
 
 
+@pytest.mark.parametrize("level", [0, 1, 2], ids=["plain", "two-float tracker", "two-float tracker and sums"])
 @pytest.mark.parametrize("name,ov", [
     ("quad_tree64", dict(n=32, p=4099, K=80, drop=0.4)),
     ("quad_tree64", dict(n=16, p=70_001, K=30)),
     ("ls_ring4", {}),
     ("logistic_tree1024", dict(n=96, p=5000, rows=8, K=60, batch=4, nnz=50)),
-    ("softmax_exp16", dict(F=96, C=7, rows=64, K=150, batch=8, compensated=False)),
-], ids=["quad", "quad tiles", "ls", "logistic", "softmax plain"])
-def test_parity_in_the_other_tracker_arithmetic(rfast_lib, name, ov):
-    """Every objective in the tracker arithmetic its configuration does not use by default
-    (compensated two-float tracker <-> plain fp32)."""
+    ("softmax_exp16", dict(F=96, C=7, rows=64, K=150, batch=8)),
+], ids=["quad", "quad tiles", "ls", "logistic", "softmax"])
+def test_parity_in_every_tracker_arithmetic(rfast_lib, name, ov, level):
+    """Every objective in each of the three tracker arithmetics (plain fp32; tracker as two
+    floats with error feedback; running sums as two floats as well)."""
     import paper_2307_11617_b200 as pkg
     wl = build_config(name, seed=2, **ov)
-    if name != "softmax_exp16":
-        wl.compensated = True
+    wl.compensated = level
     orc, ref0 = _oracle(wl)
     with pkg.Engine(wl) as eng:
         eng.load_schedule(wl.schedule)
         eng.run()
         _compare(eng, orc, ref0)
+        d = eng.diagnostics()
+    if level == 2:                                   # Lemma 3 then holds to double-float accuracy
+        assert d["conservation_residual"] <= 1e-9 * max(d["gradient_sum_max"], d["tracker_norm"])
 
 
 def test_conservation_on_the_device_state(rfast_lib):

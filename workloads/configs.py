@@ -48,7 +48,8 @@ class Workload:
     x0: np.ndarray | None = None    # float32 [n, p] or None (zeros)
     schedule: Schedule | None = None
     meta: dict = field(default_factory=dict)
-    compensated: bool = False       # ask the engine for compensated tracker arithmetic (long horizons)
+    compensated: int = 0            # tracker arithmetic asked of the engine: 0 plain fp32, 1 two-float
+                                    # tracker, 2 two-float tracker and running sums
 
     def __post_init__(self):
         # scalars are handed to every consumer as the fp32-representable value
@@ -114,7 +115,8 @@ def _ls_ring(seed, ov):
     sch = make_schedule(G_R, G_C, act, drop, max_delay, rs, batch=0)
     return Workload("ls_ring4", n, p, 0, alpha, G_R, G_C, MODEL_LEAST_SQUARES, 0, 0.0, rows,
                     dims={"n_features": p}, data={"feat": feat, "target": target}, schedule=sch,
-                    meta={"K": K, "drop": drop, "max_delay": max_delay})
+                    meta={"K": K, "drop": drop, "max_delay": max_delay},
+                    compensated=ov.get("compensated", 2))
 
 
 # -- config 2: n=16 exponential-graph trees, softmax regression, one 4x straggler --------------
@@ -134,7 +136,7 @@ def _softmax_exp(seed, ov):
                     dims={"n_features": F, "n_classes": C}, data={"feat": feat, "label": label},
                     schedule=sch, meta={"K": K, "drop": drop, "max_delay": max_delay,
                                         "straggler": straggler},
-                    compensated=ov.get("compensated", True))
+                    compensated=ov.get("compensated", 1))
 
 
 # -- config 3: n=64 random trees, MLP F-H-C ReLU, lognormal compute times -----------------------
