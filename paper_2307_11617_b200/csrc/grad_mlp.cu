@@ -145,7 +145,7 @@ struct MlpPlan {
     int64_t stride = 0;
     __nv_bfloat16 *featb = nullptr, *Ab = nullptr, *AbT = nullptr, *dpqT = nullptr;
     float* hf = nullptr;               // [ev][B][H] hidden activations
-    float* dlog = nullptr;             // [ev][B][C] gradient w.r.t. the logits
+    float* dlog = nullptr;             // [ev][B][16] gradient w.r.t. the logits, zero beyond C
     int* status = nullptr;
     CUtensorMap tmW1, tmA, tmD, tmAT;
 };
@@ -279,115 +279,146 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
 }
 
 // Output layer forward, softmax and dlog = (softmax - onehot) / B: one warp per sampled row.
-// grid = (B / 8, events), 256 threads.  dlog: [events][B][C]; CTA 0's first warps also leave gb2.
+// W2 is staged once per CTA in shared memory (the per-class loads of the dot products would
+// otherwise each wait on L2), the row of h is fetched with all its loads in flight together.
+// grid = (B / 8, events), 256 threads, dynamic shared memory C*H floats.  dlog: [events][B][16],
+// classes beyond C are zero.
 __global__ void __launch_bounds__(256)
 k_mlp_logits(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
              const float* __restrict__ x, int64_t stride, const float* __restrict__ hf,
              float* __restrict__ dlog, int rows, int F, int H, int C) {
+    extern __shared__ float4 w2s[];                        // [C][H / 4]
     const int ev = blockIdx.y;
     const EvDesc e = evs[ev];
     const int64_t row = (int64_t)e.node * stride;
     const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k = blockIdx.x * 8 + warp;
-    const float* h = hf + ((int64_t)ev * kBatch + k) * H;
-    const float* W2 = x + row + oW2;
+    const float4* h4 = reinterpret_cast<const float4*>(hf + ((int64_t)ev * kBatch + k) * H);
+    const float4* W2 = reinterpret_cast<const float4*>(x + row + oW2);
+    const int H4 = H / 4;
+    for (int q = threadIdx.x; q < C * H4; q += 256) w2s[q] = W2[q];
+    const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
+    const float bias = lane < C ? x[row + ob2 + lane] : 0.f;
     float acc[16];
 #pragma unroll
     for (int c = 0; c < 16; ++c) acc[c] = 0.f;
-    for (int j4 = lane; j4 < H / 4; j4 += 32) {
-        // all loads of the iteration first, then the arithmetic: the loads then overlap
-        float4 w[16];
+    for (int t0 = 0; t0 < H4; t0 += 128) {                 // H is a multiple of 128: lane-strided quads
+        float4 hv[4];
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-            w[c] = c < C ? reinterpret_cast<const float4*>(W2 + (int64_t)c * H)[j4] : make_float4(0, 0, 0, 0);
-        const float4 hv = reinterpret_cast<const float4*>(h)[j4];
+        for (int u = 0; u < 4; ++u)
+            hv[u] = t0 + u * 32 < H4 ? h4[t0 + u * 32 + lane] : make_float4(0, 0, 0, 0);
+        if (t0 == 0) __syncthreads();                      // W2 is in shared memory
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-            acc[c] = fmaf(hv.w, w[c].w, fmaf(hv.z, w[c].z, fmaf(hv.y, w[c].y, fmaf(hv.x, w[c].x, acc[c]))));
+        for (int u = 0; u < 4; ++u) {
+            if (t0 + u * 32 < H4) {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    if (c < C) {
+                        const float4 w = w2s[c * H4 + t0 + u * 32 + lane];
+                        acc[c] = fmaf(hv[u].w, w.w, fmaf(hv[u].z, w.z, fmaf(hv[u].y, w.y, fmaf(hv[u].x, w.x, acc[c]))));
+                    }
+                }
+            }
+        }
     }
-    float lg[16], m = -3.0e38f;
+    float mine = 0.f, m = -3.0e38f;                        // lane c keeps the logit of class c
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-        if (c < C) { lg[c] = warp_sum(acc[c]) + x[row + ob2 + c]; m = fmaxf(m, lg[c]); }
+    for (int c = 0; c < 16; ++c) {
+        if (c < C) {
+            const float s = warp_sum(acc[c]);
+            if (lane == c) mine = s + bias;
+        }
+    }
+    const float lg = lane < C ? mine : -3.0e38f;
+    m = lg;
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));   // lanes 0..15 hold the classes
+    const float ex = lane < C ? expf(lg - m) : 0.f;
     float den = 0.f;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) if (c < C) den += expf(lg[c] - m);
-    const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-        if (c < C && lane == c)
-            dlog[((int64_t)ev * kBatch + k) * C + c] = (expf(lg[c] - m) / den - (c == lab ? 1.f : 0.f)) / (float)kBatch;
+    for (int c = 0; c < 16; ++c) den += __shfl_sync(0xffffffffu, ex, c);   // class order, the same in every lane
+    if (lane < 16)
+        dlog[((int64_t)ev * kBatch + k) * 16 + lane] = lane < C ? (ex / den - (lane == lab ? 1.f : 0.f)) / (float)kBatch : 0.f;
 }
 
-// Backward through the output layer for a slab of 128 hidden units: gW2, gb1, dpre and its
+// Backward through the output layer for a slab of 64 hidden units: gW2, gb1, dpre and its
 // bf16 transpose for the second big product; the first slab also sums gb2.  A thread owns one
 // hidden unit and a quarter of the batch; the four partial sums are added in a fixed order.
-// grid = (H / 128, events), 512 threads; dynamic shared memory: B*C + 4*128*17 floats
-__global__ void __launch_bounds__(512)
+// CQ = ceil(C / 4): the class dimension is processed in quads, dlog being zero beyond C.
+// grid = (H / 64, events), 256 threads
+template <int CQ>
+__global__ void __launch_bounds__(256)
 k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
            const float* __restrict__ hf, const float* __restrict__ dlog, __nv_bfloat16* __restrict__ dpqT,
            float* __restrict__ gbuf, int64_t gplane, int F, int H, int C, float l2) {
-    extern __shared__ float smb[];
-    float* dl = smb;                          // [B][C]
-    float* part = smb + kBatch * C;           // [4][128][17]: gw2[0..15], gb1
+    constexpr int CP = CQ * 4, kSlab = 64, kQuarter = kBatch / 4;
+    __shared__ float4 dl[kBatch][4];                       // [B][16]
+    __shared__ float part[4][kSlab][CP + 1];               // gw2[0..CP), gb1
     const int ev = blockIdx.y;
     const EvDesc e = evs[ev];
     const int64_t row = (int64_t)e.node * stride;
     const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
-    const float* h = hf + (int64_t)ev * kBatch * H;
     const float* W2 = x + row + oW2;
     float* g = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row;
-    for (int q = threadIdx.x; q < kBatch * C; q += 512) dl[q] = dlog[(int64_t)ev * kBatch * C + q];
+    const int jl = threadIdx.x & (kSlab - 1), kq = threadIdx.x >> 6;
+    const int j = blockIdx.x * kSlab + jl;
+    // everything this thread needs from global memory, all in flight together
+    const float4 dmine = reinterpret_cast<const float4*>(dlog + (int64_t)ev * kBatch * 16)[threadIdx.x];
+    const float* h = hf + (int64_t)ev * kBatch * H + j;
+    float hv[kQuarter];
+#pragma unroll
+    for (int kk = 0; kk < kQuarter; ++kk) hv[kk] = h[(int64_t)(kq * kQuarter + kk) * H];
+    float w2[CP], gw2[CP];
+#pragma unroll
+    for (int c = 0; c < CP; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
+    (&dl[0][0])[threadIdx.x] = dmine;
     __syncthreads();
-    if (blockIdx.x == 0 && threadIdx.x < C) {
+    if (blockIdx.x == 0 && threadIdx.x < 32) {             // gb2: two halves of the batch, lower half first
+        const int c = threadIdx.x & 15, half = threadIdx.x >> 4;
+        const float* dlf = reinterpret_cast<const float*>(&dl[0][0]);
         float s = 0.f;
-        for (int k = 0; k < kBatch; ++k) s += dl[k * C + threadIdx.x];
-        g[ob2 + threadIdx.x] = s + l2 * x[row + ob2 + threadIdx.x];
+        for (int k = half * (kBatch / 2); k < (half + 1) * (kBatch / 2); ++k) s += dlf[k * 16 + c];
+        const float o = __shfl_down_sync(0xffffffffu, s, 16);
+        if (threadIdx.x < C) g[ob2 + c] = (s + o) + l2 * x[row + ob2 + c];
     }
-    const int jl = threadIdx.x & 127, kq = threadIdx.x >> 7;
-    const int j = blockIdx.x * 128 + jl;
-    float w2[16], gw2[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
     float gb1 = 0.f;
-    __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch;
-    constexpr int kQuarter = kBatch / 4;
-    for (int k0 = kq * kQuarter; k0 < (kq + 1) * kQuarter; k0 += 8) {
-        __align__(16) __nv_bfloat16 pack[8];
-        float hv[8];
+    __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch + kq * kQuarter;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) hv[kk] = h[(int64_t)(k0 + kk) * H + j];
+    for (int k0 = 0; k0 < kQuarter; k0 += 8) {
+        uint32_t pk[4];
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-            const int k = k0 + kk;
+            const int k = kq * kQuarter + k0 + kk;
+            float d[CP];
+#pragma unroll
+            for (int cq = 0; cq < CQ; ++cq) {
+                const float4 t = dl[k][cq];
+                d[cq * 4] = t.x; d[cq * 4 + 1] = t.y; d[cq * 4 + 2] = t.z; d[cq * 4 + 3] = t.w;
+            }
             float dh = 0.f;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) if (c < C) dh = fmaf(dl[k * C + c], w2[c], dh);
-            const float dp = hv[kk] > 0.f ? dh : 0.f;
+            for (int c = 0; c < CP; ++c) dh = fmaf(d[c], w2[c], dh);
+            const float dp = hv[k0 + kk] > 0.f ? dh : 0.f;
             gb1 += dp;
-            pack[kk] = __float2bfloat16_rn(dp);
+            const uint32_t b = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(dp));
+            if (kk & 1) pk[kk >> 1] |= b << 16; else pk[kk >> 1] = b;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) if (c < C) gw2[c] = fmaf(dl[k * C + c], hv[kk], gw2[c]);
+            for (int c = 0; c < CP; ++c) gw2[c] = fmaf(d[c], hv[k0 + kk], gw2[c]);
         }
-        *reinterpret_cast<uint4*>(drow + k0) = *reinterpret_cast<const uint4*>(pack);
+        *reinterpret_cast<uint4*>(drow + k0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
-    float* mine = part + ((int64_t)kq * 128 + jl) * 17;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) mine[c] = gw2[c];
-    mine[16] = gb1;
+    for (int c = 0; c < CP; ++c) part[kq][jl][c] = gw2[c];
+    part[kq][jl][CP] = gb1;
     __syncthreads();
-    if (kq == 0) {
-        float tot[17];
-#pragma unroll
-        for (int c = 0; c < 17; ++c) tot[c] = part[(int64_t)jl * 17 + c];
-        for (int qd = 1; qd < 4; ++qd)
-#pragma unroll
-            for (int c = 0; c < 17; ++c) tot[c] += part[((int64_t)qd * 128 + jl) * 17 + c];
-        g[(int64_t)H * F + j] = tot[16] + l2 * x[row + (int64_t)H * F + j];
-#pragma unroll
-        for (int c = 0; c < 16; ++c)
-            if (c < C) g[oW2 + (int64_t)c * H + j] = tot[c] + l2 * x[row + oW2 + (int64_t)c * H + j];
+    // (C + 1) x 64 outputs, consecutive threads on consecutive hidden units
+    for (int o = threadIdx.x; o < (C + 1) * kSlab; o += 256) {
+        const int c = o >> 6, jj = o & (kSlab - 1);        // c == C: gb1
+        const int pc = c < C ? c : CP;
+        const float tot = ((part[0][jj][pc] + part[1][jj][pc]) + part[2][jj][pc]) + part[3][jj][pc];
+        const int64_t at = c < C ? oW2 + (int64_t)c * H + blockIdx.x * kSlab + jj : (int64_t)H * F + blockIdx.x * kSlab + jj;
+        g[at] = tot + l2 * x[row + at];
     }
 }
 
@@ -520,6 +551,10 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
         err = "MLP: the tensor-core path needs batch = 64, n_hidden a multiple of 128, n_features a multiple of 16, 2 <= n_classes <= 16";
         return RFAST_EINVAL;
     }
+    if ((size_t)C * H * sizeof(float) > 200 * 1024) {
+        err = "MLP: n_classes * n_hidden floats must fit in 200 KB of shared memory";
+        return RFAST_EINVAL;
+    }
     MlpPlan* p = new MlpPlan();
     p->n = n; p->rows = rows; p->F = F; p->H = H; p->C = C; p->B = B; p->stride = stride; p->maxev = max_events;
     p->Fp = (F + kKBlock - 1) / kKBlock * kKBlock;
@@ -561,7 +596,9 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
         }
     }
     if (cudaFuncSetAttribute(k_mlp_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDw1Smem) != cudaSuccess) {
+        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDw1Smem) != cudaSuccess ||
+        ((size_t)C * H * sizeof(float) > 48 * 1024 &&
+         cudaFuncSetAttribute(k_mlp_logits, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)C * H * sizeof(float))) != cudaSuccess)) {
         mlp_plan_destroy(p);
         err = "MLP: cannot reserve shared memory";
         return RFAST_ECUDA;
@@ -584,10 +621,19 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
     k_mlp_gather<<<dim3(p->Fp / kKBlock, n_events), 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
     k_mlp_fwd<<<dim3(p->H / kMTile, n_events), kGemmThreads, kFwdSmem, st>>>(
         p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
-    k_mlp_logits<<<dim3(kBatch / 8, n_events), 256, 0, st>>>(
+    k_mlp_logits<<<dim3(kBatch / 8, n_events), 256, (size_t)p->C * p->H * sizeof(float), st>>>(
         g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dlog, p->rows, p->F, p->H, p->C);
-    k_mlp_back<<<dim3(p->H / 128, n_events), 512, (kBatch * p->C + 4 * 128 * 17) * sizeof(float), st>>>(
-        g.ev, g.x, g.stride, p->hf, p->dlog, p->dpqT, g.gbuf, g.gplane, p->F, p->H, p->C, g.l2);
+    {
+        const dim3 grid(p->H / 64, n_events);
+#define RFAST_BACK(CQ) k_mlp_back<CQ><<<grid, 256, 0, st>>>(g.ev, g.x, g.stride, p->hf, p->dlog, p->dpqT, g.gbuf, g.gplane, p->F, p->H, p->C, g.l2)
+        switch ((p->C + 3) / 4) {
+            case 1: RFAST_BACK(1); break;
+            case 2: RFAST_BACK(2); break;
+            case 3: RFAST_BACK(3); break;
+            default: RFAST_BACK(4); break;
+        }
+#undef RFAST_BACK
+    }
     k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
         p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);
     *launches += 5;
