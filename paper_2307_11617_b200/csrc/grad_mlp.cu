@@ -163,30 +163,43 @@ __global__ void k_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restri
 // Sampled rows of one activation, as the two GEMMs want them:
 //   Ab  [ev][B][Fp]  row k = features of sample k, zero beyond F (K-major operand of pre)
 //   AbT [ev][F][B]   the transpose                      (K-major operand of gW1, K = batch)
-// One CTA moves a 64 x 64 tile and transposes it through shared memory.  grid = (Fp / 64, events)
+// One CTA moves a 64 x 64 tile with 16-byte accesses and transposes it through shared memory
+// (F is a multiple of 16, so a group of 8 features never straddles F).  grid = (Fp / 64, events)
 __global__ void __launch_bounds__(256)
 k_mlp_gather(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx,
              const __nv_bfloat16* __restrict__ featb, __nv_bfloat16* __restrict__ Ab,
              __nv_bfloat16* __restrict__ AbT, int rows, int F, int Fp) {
-    __shared__ __nv_bfloat16 tile[kBatch][kKBlock + 2];
-    __shared__ int idx[kBatch];
+    __shared__ __align__(16) __nv_bfloat16 tile[kBatch][kKBlock + 8];   // row pitch 144 B: 16-byte aligned rows
     const int ev = blockIdx.y, f0 = blockIdx.x * kKBlock;
     const EvDesc e = evs[ev];
-    if (threadIdx.x < kBatch) idx[threadIdx.x] = batch_idx[(int64_t)e.sample * kBatch + threadIdx.x];
-    __syncthreads();
     const __nv_bfloat16* shard = featb + (int64_t)e.node * rows * F;
     __nv_bfloat16* ab = Ab + (int64_t)ev * kBatch * Fp;
     __nv_bfloat16* abt = AbT + (int64_t)ev * F * kBatch;
-    for (int q = threadIdx.x; q < kBatch * kKBlock; q += 256) {
-        const int k = q / kKBlock, f = q % kKBlock;
-        const __nv_bfloat16 v = (f0 + f < F) ? shard[(int64_t)idx[k] * F + f0 + f] : __float2bfloat16_rn(0.f);
-        ab[(int64_t)k * Fp + f0 + f] = v;
-        tile[k][f] = v;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {                          // 64 rows x 8 groups of 8 features
+        const int q = threadIdx.x + u * 256;
+        const int k = q >> 3, f = (q & 7) * 8;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (f0 + f < F) {
+            const int r = batch_idx[(int64_t)e.sample * kBatch + k];
+            v = *reinterpret_cast<const uint4*>(shard + (int64_t)r * F + f0 + f);
+        }
+        *reinterpret_cast<uint4*>(ab + (int64_t)k * Fp + f0 + f) = v;
+        *reinterpret_cast<uint4*>(&tile[k][f]) = v;
     }
     __syncthreads();
-    for (int q = threadIdx.x; q < kBatch * kKBlock; q += 256) {
-        const int f = q / kBatch, k = q % kBatch;
-        if (f0 + f < F) abt[(int64_t)(f0 + f) * kBatch + k] = tile[k][f];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {                          // 64 features x 8 groups of 8 samples
+        const int q = threadIdx.x + u * 256;
+        const int f = q & 63, k0 = (q >> 6) * 8;
+        if (f0 + f < F) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int kk = 0; kk < 8; kk += 2)
+                pk[kk >> 1] = (uint32_t)__bfloat16_as_ushort(tile[k0 + kk][f]) |
+                              ((uint32_t)__bfloat16_as_ushort(tile[k0 + kk + 1][f]) << 16);
+            *reinterpret_cast<uint4*>(abt + (int64_t)(f0 + f) * kBatch + k0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
     }
 }
 
@@ -477,22 +490,39 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
         const int j = h0 + q * 32 + lane;
         const int64_t row = (int64_t)e.node * stride;
         float* grow = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row + (int64_t)j * F + f0;
-        const float* xrow = x + row + (int64_t)j * F + f0;
+        const float4* xrow = reinterpret_cast<const float4*>(x + row + (int64_t)j * F + f0);
+        // The regulariser's x does not depend on the product: its loads run two 16-column chunks
+        // ahead of the accumulator read-back, the first two while the operands are still arriving.
+        const bool reg = l2 != 0.f;
+        float4 xa[4], xb[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            xa[i] = reg ? xrow[i] : make_float4(0, 0, 0, 0);
+            xb[i] = (reg && 16 < NT) ? xrow[4 + i] : make_float4(0, 0, 0, 0);
+        }
         const bool ok = mbar_wait(&acc_full, 0);
         tc_fence_after();
         if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
         else if (!aborted) {
-            for (int c0 = 0; c0 < NT; c0 += 16) {
+            for (int c0 = 0; c0 < NT; c0 += 32) {
                 float v[16];
                 tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
 #pragma unroll
-                for (int i = 0; i < 16; i += 4) {
-                    float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                    if (l2 != 0.f) {
-                        const float4 xv = *reinterpret_cast<const float4*>(xrow + c0 + i);
-                        o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
+                for (int i = 0; i < 4; ++i) {
+                    float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    if (reg) { o.x = fmaf(l2, xa[i].x, o.x); o.y = fmaf(l2, xa[i].y, o.y); o.z = fmaf(l2, xa[i].z, o.z); o.w = fmaf(l2, xa[i].w, o.w); }
+                    *reinterpret_cast<float4*>(grow + c0 + 4 * i) = o;
+                    if (reg && c0 + 32 < NT) xa[i] = xrow[(c0 + 32) / 4 + i];
+                }
+                if (c0 + 16 < NT) {
+                    tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0 + 16, v);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        if (reg) { o.x = fmaf(l2, xb[i].x, o.x); o.y = fmaf(l2, xb[i].y, o.y); o.z = fmaf(l2, xb[i].z, o.z); o.w = fmaf(l2, xb[i].w, o.w); }
+                        *reinterpret_cast<float4*>(grow + c0 + 16 + 4 * i) = o;
+                        if (reg && c0 + 48 < NT) xb[i] = xrow[(c0 + 48) / 4 + i];
                     }
-                    *reinterpret_cast<float4*>(grow + c0 + i) = o;
                 }
             }
         }
