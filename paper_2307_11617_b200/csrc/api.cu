@@ -19,8 +19,8 @@ namespace rfast {
 // MLP gradient (tensor-core path), defined in grad_mlp.cu
 struct MlpPlan;
 int  mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride, int max_events,
-                     const float* d_feat, const __nv_bfloat16* xb, cudaStream_t st, MlpPlan** out,
-                     size_t* dev_bytes, std::string& err);
+                     const float* d_feat, const __nv_bfloat16* xb, const float* x, float* gbuf, cudaStream_t st,
+                     MlpPlan** out, size_t* dev_bytes, std::string& err);
 int  mlp_plan_status(MlpPlan* plan, cudaStream_t st);
 void mlp_plan_destroy(MlpPlan* plan);
 int  mlp_grad_launch(MlpPlan* plan, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
@@ -433,7 +433,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
         CK(cudaMemsetAsync(ctx->xb, 0, plane * sizeof(__nv_bfloat16), ctx->stream));
         size_t mb = 0;
         rc = mlp_plan_create(ctx->n, ctx->rows, ctx->F, ctx->H, ctx->C, ctx->batch, ctx->stride, ctx->n,
-                             ctx->feat, ctx->xb, ctx->stream, &ctx->mlp, &mb, err);
+                             ctx->feat, ctx->xb, ctx->x, ctx->gbuf, ctx->stream, &ctx->mlp, &mb, err);
         if (rc != RFAST_OK) return set_err(ctx, rc, err);
         ctx->dev_bytes += mb;
     }

@@ -77,6 +77,18 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+// Tile store shared -> global; completion is tracked by the thread's bulk async-group.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// until the stores of all committed groups have read their shared-memory source
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// makes this thread's shared-memory writes visible to the async (TMA) proxy
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {     // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -147,7 +159,7 @@ struct MlpPlan {
     float* hf = nullptr;               // [ev][B][H] hidden activations
     float* dlog = nullptr;             // [ev][B][16] gradient w.r.t. the logits, zero beyond C
     int* status = nullptr;
-    CUtensorMap tmW1, tmA, tmD, tmAT;
+    CUtensorMap tmW1, tmA, tmD, tmAT, tmX, tmG;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -205,7 +217,7 @@ k_mlp_gather(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx,
 
 // pre^T slab = W1[h0 .. h0+128) x A^T, then h = relu(pre + b1), stored in hf[ev][k][j].
 // grid = (H / 128, events)
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kGemmThreads, 2)
 k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmA,
           const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
           float* __restrict__ hf, int F, int H, int kblocks, int* status) {
@@ -435,26 +447,35 @@ k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t 
     }
 }
 
-// One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A).
-// grid = (H / 128, F / NT, events)
+// One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A),
+// plus l2 * W1.  The fp32 side of the epilogue also goes through TMA: the W1 tile of x arrives in
+// shared memory as NT/16 pieces of 128 rows x 16 floats (64-byte swizzle) while the product runs,
+// each epilogue thread adds its accumulator row to its own row of every piece in place, and each
+// warp stores its 32 rows of a piece back with a TMA tile store.  (A thread owns a whole row of
+// the tile, so plain stores would touch 32 different cache lines per instruction.)
+// grid = (H / 128, F / NT, events); dynamic shared memory dw1_smem(NT)
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmAT,
-          const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
-          float* __restrict__ gbuf, int64_t gplane, int F, int H, int NT, float l2, int* status) {
+          const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
+          const EvDesc* __restrict__ evs, int n, int F, int H, int NT, float l2, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kABytes = kMTile * kKBlock * 2;          // q(dpre)^T slab
+    constexpr int kPiece = kMTile * 16 * 4;                // 128 rows x 16 floats
     uint8_t* sA = smem;
-    uint8_t* sB = smem + kABytes;                          // [NT][64] bf16 tile of A^T
-    __shared__ uint64_t ab_full, acc_full;
+    uint8_t* sB = smem + kABytes;                          // [NT][64] bf16 tile of A^T (at most 16 KB)
+    uint8_t* sX = smem + 2 * kABytes;                      // [NT / 16] pieces
+    __shared__ uint64_t ab_full, acc_full, x_full;
     __shared__ uint32_t tmem_base;
     __shared__ volatile int aborted;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ev = blockIdx.z, h0 = blockIdx.x * kMTile, f0 = blockIdx.y * NT;
     const EvDesc e = evs[ev];
+    const bool reg = l2 != 0.f;
     if (threadIdx.x == 0) {
         mbar_init(&ab_full, 1);
         mbar_init(&acc_full, 1);
+        mbar_init(&x_full, 1);
         aborted = 0;
         fence_barrier_init();
     }
@@ -468,6 +489,11 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
         mbar_expect_tx(&ab_full, kABytes + NT * kKBlock * 2);
         tma_load_2d(sA, &tmD, &ab_full, 0, ev * H + h0);
         tma_load_2d(sB, &tmAT, &ab_full, 0, ev * F + f0);
+        if (reg) {
+            mbar_expect_tx(&x_full, (NT / 16) * kPiece);
+            for (int pc = 0; pc < NT / 16; ++pc)
+                tma_load_3d(sX + pc * kPiece, &tmX, &x_full, f0 + pc * 16, h0, e.node);
+        }
     } else if (warp == 1 && lane == 0) {                   // ---- MMA issuer
         const uint32_t idesc = umma_idesc_bf16(kMTile, NT);
         const bool ok = mbar_wait(&ab_full, 0);
@@ -485,46 +511,35 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
             __threadfence_block();
             mbar_arrive(&acc_full);
         }
-    } else if (warp >= 2) {                                // ---- epilogue: TMEM -> global
+    } else if (warp >= 2) {                                // ---- epilogue: TMEM (+ l2 x) -> shared -> TMA store
         const int q = warp & 3;
-        const int j = h0 + q * 32 + lane;
-        const int64_t row = (int64_t)e.node * stride;
-        float* grow = gbuf + (int64_t)(e.g_par ^ 1) * gplane + row + (int64_t)j * F + f0;
-        const float4* xrow = reinterpret_cast<const float4*>(x + row + (int64_t)j * F + f0);
-        // The regulariser's x does not depend on the product: its loads run two 16-column chunks
-        // ahead of the accumulator read-back, the first two while the operands are still arriving.
-        const bool reg = l2 != 0.f;
-        float4 xa[4], xb[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            xa[i] = reg ? xrow[i] : make_float4(0, 0, 0, 0);
-            xb[i] = (reg && 16 < NT) ? xrow[4 + i] : make_float4(0, 0, 0, 0);
-        }
-        const bool ok = mbar_wait(&acc_full, 0);
+        const int r = q * 32 + lane;                        // row of the tile = tensor-memory lane
+        bool ok = mbar_wait(&acc_full, 0);
         tc_fence_after();
+        if (reg) ok = mbar_wait(&x_full, 0) && ok;          // also on the way out: the copies must have landed
         if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
         else if (!aborted) {
-            for (int c0 = 0; c0 < NT; c0 += 32) {
+            const int plane = (e.g_par ^ 1) * n + e.node;
+            const int sw = (r >> 1) & 3;                    // 64-byte swizzle: 16-byte chunk index ^ address bits 7..8
+            for (int pc = 0; pc < NT / 16; ++pc) {
                 float v[16];
-                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
+                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + pc * 16, v);
+                float4* rowp = reinterpret_cast<float4*>(sX + pc * kPiece + r * 64);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                    if (reg) { o.x = fmaf(l2, xa[i].x, o.x); o.y = fmaf(l2, xa[i].y, o.y); o.z = fmaf(l2, xa[i].z, o.z); o.w = fmaf(l2, xa[i].w, o.w); }
-                    *reinterpret_cast<float4*>(grow + c0 + 4 * i) = o;
-                    if (reg && c0 + 32 < NT) xa[i] = xrow[(c0 + 32) / 4 + i];
-                }
-                if (c0 + 16 < NT) {
-                    tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0 + 16, v);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float4 o = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-                        if (reg) { o.x = fmaf(l2, xb[i].x, o.x); o.y = fmaf(l2, xb[i].y, o.y); o.z = fmaf(l2, xb[i].z, o.z); o.w = fmaf(l2, xb[i].w, o.w); }
-                        *reinterpret_cast<float4*>(grow + c0 + 16 + 4 * i) = o;
-                        if (reg && c0 + 48 < NT) xb[i] = xrow[(c0 + 48) / 4 + i];
+                for (int c = 0; c < 4; ++c) {
+                    float4 o = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                    float4* at = rowp + (c ^ sw);
+                    if (reg) {
+                        const float4 xv = *at;
+                        o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
                     }
+                    *at = o;
                 }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) tma_store_3d(&tmG, sX + pc * kPiece + q * 32 * 64, f0 + pc * 16, h0 + q * 32, plane);
             }
+            if (lane == 0) { tma_store_commit(); tma_store_wait_read(); }
         }
     }
     tc_fence_before();
@@ -553,28 +568,30 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor, innermost dimension first; strides in bytes for dimensions 1.. ; 128-byte swizzle
+// innermost dimension first; strides in bytes for dimensions 1.. ; bf16 with the 128-byte swizzle
+// (GEMM operands) or fp32 with the 64-byte swizzle (epilogue tiles of 16 floats per row)
 bool make_map(CUtensorMap* m, void* base, int rank, const uint64_t* dims, const uint64_t* strides,
-              const uint32_t* box) {
+              const uint32_t* box, bool f32 = false) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t d[3], s[2];
     cuuint32_t b[3], es[3] = {1, 1, 1};
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
     for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, base, d, s, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+    return fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, base, d, s, b, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 1024;
-constexpr size_t kDw1Smem = kMTile * kKBlock * 2 + 128 * kKBlock * 2 + 1024;
+constexpr size_t dw1_smem(int NT) { return 2 * (size_t)kMTile * kKBlock * 2 + (size_t)(NT / 16) * kMTile * 16 * 4 + 1024; }
 
 }  // namespace
 
 int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride, int max_events,
-                    const float* d_feat, const __nv_bfloat16* xb, cudaStream_t st, MlpPlan** out,
-                    size_t* dev_bytes, std::string& err) {
+                    const float* d_feat, const __nv_bfloat16* xb, const float* x, float* gbuf, cudaStream_t st,
+                    MlpPlan** out, size_t* dev_bytes, std::string& err) {
     *out = nullptr;
     *dev_bytes = 0;
     if (B != kBatch || H % kMTile != 0 || H <= 0 || F % 16 != 0 || F <= 0 || C < 2 || C > 16) {
@@ -618,15 +635,20 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
         const uint32_t bD[2] = {kKBlock, kMTile};
         const uint64_t dT[2] = {(uint64_t)kBatch, (uint64_t)max_events * F};
         const uint32_t bT[2] = {kKBlock, (uint32_t)p->NT};
+        // fp32 views of the W1 block: x [n][H][F] and the two gradient planes [2n][H][F]
+        const uint64_t dX[3] = {(uint64_t)F, (uint64_t)H, (uint64_t)n}, dG[3] = {(uint64_t)F, (uint64_t)H, (uint64_t)2 * n};
+        const uint64_t sX[2] = {(uint64_t)F * 4, (uint64_t)stride * 4};
+        const uint32_t bX[3] = {16, kMTile, 1}, bG[3] = {16, 32, 1};
         if (!make_map(&p->tmW1, (void*)xb, 3, dW, sW, bW) || !make_map(&p->tmA, p->Ab, 2, dA, sA, bA) ||
-            !make_map(&p->tmD, p->dpqT, 2, dD, sD, bD) || !make_map(&p->tmAT, p->AbT, 2, dT, sD, bT)) {
+            !make_map(&p->tmD, p->dpqT, 2, dD, sD, bD) || !make_map(&p->tmAT, p->AbT, 2, dT, sD, bT) ||
+            !make_map(&p->tmX, (void*)x, 3, dX, sX, bX, true) || !make_map(&p->tmG, gbuf, 3, dG, sX, bG, true)) {
             mlp_plan_destroy(p);
             err = "MLP: cuTensorMapEncodeTiled failed";
             return RFAST_ECUDA;
         }
     }
     if (cudaFuncSetAttribute(k_mlp_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDw1Smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw1_smem(p->NT)) != cudaSuccess ||
         ((size_t)C * H * sizeof(float) > 48 * 1024 &&
          cudaFuncSetAttribute(k_mlp_logits, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)C * H * sizeof(float))) != cudaSuccess)) {
         mlp_plan_destroy(p);
@@ -664,8 +686,8 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
         }
 #undef RFAST_BACK
     }
-    k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
-        p->tmD, p->tmAT, g.ev, g.x, g.stride, g.gbuf, g.gplane, p->F, p->H, p->NT, g.l2, p->status);
+    k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, dw1_smem(p->NT), st>>>(
+        p->tmD, p->tmAT, p->tmX, p->tmG, g.ev, p->n, p->F, p->H, p->NT, g.l2, p->status);
     *launches += 5;
     return RFAST_OK;
 }
