@@ -21,7 +21,9 @@ SHAPES = [
     dict(n=6, F=64, H=128, C=10, rows=128, K=20, batch=64),
     dict(n=5, F=48, H=256, C=3, rows=96, K=12, batch=64),
     dict(n=8, F=784, H=512, C=10, rows=256, K=15, batch=64),
+    dict(n=6, F=160, H=256, C=10, rows=128, K=12, batch=64, l2=1e-2),   # regulariser on: gW1 epilogue adds l2 * W1
 ]
+IDS = ["F64 H128", "F48 H256 C3", "F784 H512", "F160 H256 l2"]
 
 
 def _blocks(wl):
@@ -30,7 +32,7 @@ def _blocks(wl):
     return {"W1": (0, o1), "b1": (o1, o2), "W2": (o2, o3), "b2": (o3, wl.p)}
 
 
-@pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
+@pytest.mark.parametrize("ov", SHAPES, ids=IDS)
 def test_mlp_gradient_from_identical_state(rfast_lib, ov):
     """Initial gradients (same x0 on both sides).  b1, W2, b2 see no rounded computed operand
     and agree to fp32 accuracy.  gW1 = q(dpre)^T q(A) rounds the computed dpre to bf16: where
@@ -52,7 +54,7 @@ def test_mlp_gradient_from_identical_state(rfast_lib, ov):
     assert rel_l2(g, ref) <= 1e-4
 
 
-@pytest.mark.parametrize("ov", SHAPES, ids=["F64 H128", "F48 H256 C3", "F784 H512"])
+@pytest.mark.parametrize("ov", SHAPES, ids=IDS)
 def test_mlp_trajectory_and_gradient_at_device_iterate(rfast_lib, ov):
     import paper_2307_11617_b200 as pkg
     from paper_2307_11617_b200 import binding as B

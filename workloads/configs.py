@@ -144,6 +144,7 @@ def _mlp_tree(seed, ov):
     n = ov.get("n", 64); F = ov.get("F", 784); H = ov.get("H", 512); C = ov.get("C", 10)
     rows = ov.get("rows", 1024); K = ov.get("K", 500); B = ov.get("batch", 64)
     drop = ov.get("drop", 0.05); max_delay = ov.get("max_delay", 2); alpha = ov.get("alpha", 0.002)
+    l2 = ov.get("l2", 0.0)
     rd, rs = _rng(seed, 1), _rng(seed, 2)
     G_R, G_C = tree_graphs(random_tree_parents(n, rs), random_tree_parents(n, rs))
     feat, label = _gaussian_mixture(n, rows, F, C, 2, rd, 1.0 / np.sqrt(F))
@@ -155,7 +156,7 @@ def _mlp_tree(seed, ov):
     act = activation_durations(
         n, K, lambda i, t: max(1, int(np.rint(np.exp(rs.standard_normal())))))
     sch = make_schedule(G_R, G_C, act, drop, max_delay, rs, batch=B, rows_per_node=rows)
-    return Workload("mlp_tree64", n, p, 0, alpha, G_R, G_C, MODEL_MLP, B, 0.0, rows,
+    return Workload("mlp_tree64", n, p, 0, alpha, G_R, G_C, MODEL_MLP, B, l2, rows,
                     dims={"n_features": F, "n_hidden": H, "n_classes": C},
                     data={"feat": feat, "label": label}, x0=x0, schedule=sch,
                     meta={"K": K, "drop": drop, "max_delay": max_delay})
