@@ -10,7 +10,8 @@
 // tensor memory, and the epilogue reads the accumulator back with tcgen05.ld.  Both are
 // computed transposed (M = a 128-row slab of hidden units) so that M is the tensor core's
 // native 128.  The C <= 16 wide products in between are far too thin for an MMA tile and run
-// in fp32 on the CUDA cores of one CTA per activation.
+// in fp32 on the CUDA cores: the logits as per-slab shares in the forward kernel's epilogue,
+// while h is still in shared memory, the rest in the backward kernel.
 //
 // Every wait on an mbarrier is bounded: when it runs out the CTA records a code in a status
 // word, leaves its loops, frees its tensor memory and returns.
@@ -31,6 +32,9 @@ constexpr int kBatch = 64;          // rows per minibatch the tensor-core path i
 constexpr int kMTile = 128;         // hidden units per CTA (UMMA M)
 constexpr int kKBlock = 64;         // bf16 elements per 128-byte swizzle row
 constexpr int kStagesFwd = 4;
+constexpr int kFwdWorkers = 256;    // warps 2..9 of the forward kernel
+constexpr int kFwdThreads = 64 + kFwdWorkers;   // warp 0: TMA, warp 1: MMA + tensor memory
+constexpr int kHsPitch = 132;       // floats per staged row of 128 hidden activations (rows fall on different banks)
 constexpr int kGemmThreads = 192;   // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every mbarrier wait gives up after 2 s
 
@@ -157,7 +161,7 @@ struct MlpPlan {
     int64_t stride = 0;
     __nv_bfloat16 *featb = nullptr, *Ab = nullptr, *AbT = nullptr, *dpqT = nullptr;
     float* hf = nullptr;               // [ev][B][H] hidden activations
-    float* dlog = nullptr;             // [ev][B][16] gradient w.r.t. the logits, zero beyond C
+    float* share = nullptr;            // [ev][H / 128][B][16] logit shares of the slabs, zero beyond C
     int* status = nullptr;
     CUtensorMap tmW1, tmA, tmD, tmAT, tmX, tmG;
 };
@@ -215,27 +219,37 @@ k_mlp_gather(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx,
     }
 }
 
-// pre^T slab = W1[h0 .. h0+128) x A^T, then h = relu(pre + b1), stored in hf[ev][k][j].
-// grid = (H / 128, events)
-__global__ void __launch_bounds__(kGemmThreads, 2)
+// pre^T slab = W1[h0 .. h0+128) x A^T, then h = relu(pre + b1), stored in hf[ev][k][j], and the
+// slab's share of the logits, share[ev][slab][k][c] = sum over the slab's 128 hidden units of
+// h[k][j] W2[c][j]: h is still on chip when the product ends (it is staged in the operand
+// stages, which are free by then), so the output layer costs no second pass over h.  The shares
+// of the H / 128 slabs are added, in slab order, by the backward kernel.
+// grid = (H / 128, events), 320 threads; dynamic shared memory kFwdSmem
+template <int CQ>
+__global__ void __launch_bounds__(kFwdThreads, 2)
 k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmA,
           const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
-          float* __restrict__ hf, int F, int H, int kblocks, int* status) {
+          float* __restrict__ hf, float* __restrict__ share, int F, int H, int C, int kblocks, int* status) {
+    constexpr int CP = CQ * 4;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kABytes = kMTile * kKBlock * 2, kBBytes = kBatch * kKBlock * 2;
     uint8_t* sA = smem;                                   // [stages][128][64] bf16
     uint8_t* sB = smem + kStagesFwd * kABytes;            // [stages][64][64] bf16
+    float* hs = reinterpret_cast<float*>(smem);           // after the product: h [64][kHsPitch]
+    float* w2s = reinterpret_cast<float*>(smem + kStagesFwd * (kABytes + kBBytes));   // [16][kHsPitch]
     __shared__ uint64_t full[kStagesFwd], empty[kStagesFwd], acc_full;
     __shared__ uint32_t tmem_base;
-    __shared__ volatile int aborted;
+    __shared__ volatile int bad;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ev = blockIdx.y, h0 = blockIdx.x * kMTile;
     const EvDesc e = evs[ev];
+    const int64_t row = (int64_t)e.node * stride;
+    const int64_t ob1 = (int64_t)H * F, oW2 = ob1 + H;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesFwd; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         mbar_init(&acc_full, 1);
-        aborted = 0;
+        bad = 0;
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&tmem_base, 64);
@@ -243,6 +257,7 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
     __syncthreads();
     tc_fence_after();
     const uint32_t tacc = tmem_base;
+    const int wt = threadIdx.x - 64;                       // worker thread id, 0..255 in warps 2..9
 
     if (warp == 0 && lane == 0) {                          // ---- TMA producer
         int issued = 0;
@@ -258,6 +273,7 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
         }
         if (!ok) {
             atomicExch(status, kErrProducer);
+            bad = 1;
             // let the copies already issued land before the CTA's shared memory goes away
             for (int q = (issued > kStagesFwd ? issued - kStagesFwd : 0); q < issued; ++q)
                 mbar_wait(&full[q % kStagesFwd], (q / kStagesFwd) & 1);
@@ -278,105 +294,73 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
             umma_commit(&empty[s]);
         }
         if (ok) umma_commit(&acc_full);
-        else { atomicExch(status, kErrMma); aborted = 1; __threadfence_block(); mbar_arrive(&acc_full); }
-    } else if (warp >= 2) {                                // ---- epilogue: TMEM -> relu -> hf
+        else { atomicExch(status, kErrMma); bad = 1; __threadfence_block(); mbar_arrive(&acc_full); }
+    } else if (warp >= 2) {                                // ---- epilogue: TMEM -> relu -> hf and shared memory
+        // while the product runs: the W2 columns of the slab (rows C .. CP-1 zero) and the bias
+        for (int o = wt; o < CP * kMTile; o += kFwdWorkers) {
+            const int c = o >> 7, j = o & (kMTile - 1);
+            w2s[c * kHsPitch + j] = c < C ? x[row + oW2 + (int64_t)c * H + h0 + j] : 0.f;
+        }
+        const int q = warp & 3;                             // this warp owns tensor-memory lanes 32q .. 32q+31
+        const int colh = (warp - 2) >> 2;                   // and columns 32 colh .. 32 colh + 31
+        const int jl = q * 32 + lane;                       // hidden unit inside the slab
+        const float b1 = x[row + ob1 + h0 + jl];
         const bool ok = mbar_wait(&acc_full, 0);
         tc_fence_after();
-        if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
-        else if (!aborted) {
-            const int q = warp & 3;                         // this warp owns tensor-memory lanes 32q .. 32q+31
-            const int j = h0 + q * 32 + lane;               // hidden unit
-            const float b1 = x[(int64_t)e.node * stride + (int64_t)H * F + j];
-            float* out = hf + (int64_t)ev * kBatch * H + j;
+        if (!ok) { if (lane == 0) { atomicExch(status, kErrEpilogue); bad = 1; } }
+        else if (!bad) {
+            float* out = hf + (int64_t)ev * kBatch * H + h0 + jl;
 #pragma unroll
-            for (int c0 = 0; c0 < kBatch; c0 += 16) {
+            for (int c0 = 0; c0 < 32; c0 += 16) {
                 float v[16];
-                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + c0, v);
+                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + colh * 32 + c0, v);
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    out[(int64_t)(c0 + i) * H] = fmaxf(v[i] + b1, 0.f);
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 64); }
-}
-
-// Output layer forward, softmax and dlog = (softmax - onehot) / B: one warp per sampled row.
-// W2 is staged once per CTA in shared memory (the per-class loads of the dot products would
-// otherwise each wait on L2), the row of h is fetched with all its loads in flight together.
-// grid = (B / 8, events), 256 threads, dynamic shared memory C*H floats.  dlog: [events][B][16],
-// classes beyond C are zero.
-__global__ void __launch_bounds__(256)
-k_mlp_logits(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
-             const float* __restrict__ x, int64_t stride, const float* __restrict__ hf,
-             float* __restrict__ dlog, int rows, int F, int H, int C) {
-    extern __shared__ float4 w2s[];                        // [C][H / 4]
-    const int ev = blockIdx.y;
-    const EvDesc e = evs[ev];
-    const int64_t row = (int64_t)e.node * stride;
-    const int64_t oW2 = (int64_t)H * F + H, ob2 = oW2 + (int64_t)C * H;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k = blockIdx.x * 8 + warp;
-    const float4* h4 = reinterpret_cast<const float4*>(hf + ((int64_t)ev * kBatch + k) * H);
-    const float4* W2 = reinterpret_cast<const float4*>(x + row + oW2);
-    const int H4 = H / 4;
-    for (int q = threadIdx.x; q < C * H4; q += 256) w2s[q] = W2[q];
-    const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + k]];
-    const float bias = lane < C ? x[row + ob2 + lane] : 0.f;
-    float acc[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) acc[c] = 0.f;
-    for (int t0 = 0; t0 < H4; t0 += 128) {                 // H is a multiple of 128: lane-strided quads
-        float4 hv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            hv[u] = t0 + u * 32 < H4 ? h4[t0 + u * 32 + lane] : make_float4(0, 0, 0, 0);
-        if (t0 == 0) __syncthreads();                      // W2 is in shared memory
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (t0 + u * 32 < H4) {
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    if (c < C) {
-                        const float4 w = w2s[c * H4 + t0 + u * 32 + lane];
-                        acc[c] = fmaf(hv[u].w, w.w, fmaf(hv[u].z, w.z, fmaf(hv[u].y, w.y, fmaf(hv[u].x, w.x, acc[c]))));
-                    }
+                for (int i = 0; i < 16; ++i) {
+                    const float hval = fmaxf(v[i] + b1, 0.f);
+                    out[(int64_t)(colh * 32 + c0 + i) * H] = hval;
+                    hs[(colh * 32 + c0 + i) * kHsPitch + jl] = hval;
                 }
             }
         }
     }
-    float mine = 0.f, m = -3.0e38f;                        // lane c keeps the logit of class c
+    tc_fence_before();
+    __syncthreads();                                       // h and the W2 columns are in shared memory
+    if (warp >= 2 && bad == 0) {                           // ---- the slab's share of the logits
+        const int k = wt >> 2, cgp = wt & 3;                // sampled row; classes cgp, cgp + 4, ...
+        float acc[CQ];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        if (c < C) {
-            const float s = warp_sum(acc[c]);
-            if (lane == c) mine = s + bias;
+        for (int i = 0; i < CQ; ++i) acc[i] = 0.f;
+        const float4* h4 = reinterpret_cast<const float4*>(hs + k * kHsPitch);
+#pragma unroll 8
+        for (int j4 = 0; j4 < kMTile / 4; ++j4) {
+            const float4 hv = h4[j4];
+#pragma unroll
+            for (int i = 0; i < CQ; ++i) {
+                const float4 w = reinterpret_cast<const float4*>(w2s + (cgp + 4 * i) * kHsPitch)[j4];
+                acc[i] = fmaf(hv.w, w.w, fmaf(hv.z, w.z, fmaf(hv.y, w.y, fmaf(hv.x, w.x, acc[i]))));
+            }
         }
+        float* dst = share + (((int64_t)ev * gridDim.x + blockIdx.x) * kBatch + k) * 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[cgp + 4 * i] = i < CQ ? acc[i < CQ ? i : 0] : 0.f;
     }
-    const float lg = lane < C ? mine : -3.0e38f;
-    m = lg;
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));   // lanes 0..15 hold the classes
-    const float ex = lane < C ? expf(lg - m) : 0.f;
-    float den = 0.f;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) den += __shfl_sync(0xffffffffu, ex, c);   // class order, the same in every lane
-    if (lane < 16)
-        dlog[((int64_t)ev * kBatch + k) * 16 + lane] = lane < C ? (ex / den - (lane == lab ? 1.f : 0.f)) / (float)kBatch : 0.f;
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 64); }
 }
 
-// Backward through the output layer for a slab of 64 hidden units: gW2, gb1, dpre and its
-// bf16 transpose for the second big product; the first slab also sums gb2.  A thread owns one
-// hidden unit and a quarter of the batch; the four partial sums are added in a fixed order.
-// CQ = ceil(C / 4): the class dimension is processed in quads, dlog being zero beyond C.
+// Backward through the output layer for a slab of 64 hidden units.  Every CTA first finishes
+// the output layer for the whole batch (64 x C values: the logit shares of the forward kernel
+// added in slab order, bias, softmax, dlog = (softmax - onehot) / B; the four class quads of a
+// row sit in adjacent lanes and combine maximum and denominator by shuffles), then forms gW2,
+// gb1, dpre and its bf16 transpose for the second big product; the first slab also sums gb2.
+// A thread owns one hidden unit and a quarter of the batch; the four partial sums are added in
+// a fixed order.  CQ = ceil(C / 4): the class dimension is processed in quads, zero beyond C.
 // grid = (H / 64, events), 256 threads
 template <int CQ>
 __global__ void __launch_bounds__(256)
-k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t stride,
-           const float* __restrict__ hf, const float* __restrict__ dlog, __nv_bfloat16* __restrict__ dpqT,
-           float* __restrict__ gbuf, int64_t gplane, int F, int H, int C, float l2) {
+k_mlp_back(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, const int* __restrict__ label,
+           const float* __restrict__ x, int64_t stride, const float* __restrict__ hf,
+           const float* __restrict__ share, int R, __nv_bfloat16* __restrict__ dpqT,
+           float* __restrict__ gbuf, int64_t gplane, int rows, int F, int H, int C, float l2) {
     constexpr int CP = CQ * 4, kSlab = 64, kQuarter = kBatch / 4;
     __shared__ float4 dl[kBatch][4];                       // [B][16]
     __shared__ float part[4][kSlab][CP + 1];               // gw2[0..CP), gb1
@@ -389,7 +373,20 @@ k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t 
     const int jl = threadIdx.x & (kSlab - 1), kq = threadIdx.x >> 6;
     const int j = blockIdx.x * kSlab + jl;
     // everything this thread needs from global memory, all in flight together
-    const float4 dmine = reinterpret_cast<const float4*>(dlog + (int64_t)ev * kBatch * 16)[threadIdx.x];
+    const int ks = threadIdx.x >> 2, quad = threadIdx.x & 3;   // output layer: sampled row, class quad
+    const int lab = label[(int64_t)e.node * rows + batch_idx[(int64_t)e.sample * kBatch + ks]];
+    float4 lg = make_float4(0, 0, 0, 0);
+    if (quad < CQ) {
+        const float4* sh = reinterpret_cast<const float4*>(share + ((int64_t)ev * R * kBatch + ks) * 16) + quad;
+        lg = sh[0];
+        for (int r = 1; r < R; ++r) {                       // slab order
+            const float4 t = sh[(int64_t)r * kBatch * 4];
+            lg.x += t.x; lg.y += t.y; lg.z += t.z; lg.w += t.w;
+        }
+    }
+    float b2[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) b2[i] = 4 * quad + i < C ? x[row + ob2 + 4 * quad + i] : 0.f;
     const float* h = hf + (int64_t)ev * kBatch * H + j;
     float hv[kQuarter];
 #pragma unroll
@@ -397,7 +394,24 @@ k_mlp_back(const EvDesc* __restrict__ evs, const float* __restrict__ x, int64_t 
     float w2[CP], gw2[CP];
 #pragma unroll
     for (int c = 0; c < CP; ++c) { w2[c] = c < C ? W2[(int64_t)c * H + j] : 0.f; gw2[c] = 0.f; }
-    (&dl[0][0])[threadIdx.x] = dmine;
+    {
+        float l4[4] = {lg.x + b2[0], lg.y + b2[1], lg.z + b2[2], lg.w + b2[3]};
+        float m = -3.0e38f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) if (4 * quad + i < C) m = fmaxf(m, l4[i]);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        float ex[4], den = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { ex[i] = 4 * quad + i < C ? expf(l4[i] - m) : 0.f; den += ex[i]; }
+        den += __shfl_xor_sync(0xffffffffu, den, 1);       // the same tree in all four lanes
+        den += __shfl_xor_sync(0xffffffffu, den, 2);
+        float d[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            d[i] = 4 * quad + i < C ? (ex[i] / den - (4 * quad + i == lab ? 1.f : 0.f)) / (float)kBatch : 0.f;
+        dl[ks][quad] = make_float4(d[0], d[1], d[2], d[3]);
+    }
     __syncthreads();
     if (blockIdx.x == 0 && threadIdx.x < 32) {             // gb2: two halves of the batch, lower half first
         const int c = threadIdx.x & 15, half = threadIdx.x >> 4;
@@ -584,7 +598,7 @@ bool make_map(CUtensorMap* m, void* base, int rank, const uint64_t* dims, const 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 1024;
+constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 16 * kHsPitch * 4 + 1024;
 constexpr size_t dw1_smem(int NT) { return 2 * (size_t)kMTile * kKBlock * 2 + (size_t)(NT / 16) * kMTile * 16 * 4 + 1024; }
 
 }  // namespace
@@ -596,10 +610,6 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
     *dev_bytes = 0;
     if (B != kBatch || H % kMTile != 0 || H <= 0 || F % 16 != 0 || F <= 0 || C < 2 || C > 16) {
         err = "MLP: the tensor-core path needs batch = 64, n_hidden a multiple of 128, n_features a multiple of 16, 2 <= n_classes <= 16";
-        return RFAST_EINVAL;
-    }
-    if ((size_t)C * H * sizeof(float) > 200 * 1024) {
-        err = "MLP: n_classes * n_hidden floats must fit in 200 KB of shared memory";
         return RFAST_EINVAL;
     }
     MlpPlan* p = new MlpPlan();
@@ -618,7 +628,7 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
               alloc(&p->AbT, (size_t)max_events * F * kBatch) &&
               alloc(&p->dpqT, (size_t)max_events * H * kBatch) &&
               cudaMalloc((void**)&p->hf, (size_t)max_events * kBatch * H * sizeof(float)) == cudaSuccess &&
-              cudaMalloc((void**)&p->dlog, (size_t)max_events * kBatch * 16 * sizeof(float)) == cudaSuccess &&
+              cudaMalloc((void**)&p->share, (size_t)max_events * (H / kMTile) * kBatch * 16 * sizeof(float)) == cudaSuccess &&
               cudaMalloc((void**)&p->status, sizeof(int)) == cudaSuccess;
     if (!ok) { mlp_plan_destroy(p); err = "MLP: device allocation failed"; return RFAST_ENOMEM; }
     cudaMemsetAsync(p->status, 0, sizeof(int), st);
@@ -647,22 +657,24 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
             return RFAST_ECUDA;
         }
     }
-    if (cudaFuncSetAttribute(k_mlp_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw1_smem(p->NT)) != cudaSuccess ||
-        ((size_t)C * H * sizeof(float) > 48 * 1024 &&
-         cudaFuncSetAttribute(k_mlp_logits, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)C * H * sizeof(float))) != cudaSuccess)) {
+    if (cudaFuncSetAttribute(k_mlp_fwd<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_fwd<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_fwd<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_fwd<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw1_smem(p->NT)) != cudaSuccess) {
         mlp_plan_destroy(p);
         err = "MLP: cannot reserve shared memory";
         return RFAST_ECUDA;
     }
     *out = p;
-    *dev_bytes = total + sizeof(int) + (size_t)max_events * kBatch * H * sizeof(float);
+    *dev_bytes = total + sizeof(int) + (size_t)max_events * kBatch * H * sizeof(float) +
+                 (size_t)max_events * (H / kMTile) * kBatch * 16 * sizeof(float);
     return RFAST_OK;
 }
 
 void mlp_plan_destroy(MlpPlan* p) {
     if (!p) return;
-    void* ptrs[] = {p->featb, p->Ab, p->AbT, p->hf, p->dlog, p->dpqT, p->status};
+    void* ptrs[] = {p->featb, p->Ab, p->AbT, p->hf, p->share, p->dpqT, p->status};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete p;
 }
@@ -671,24 +683,25 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
                     int n_events, cudaStream_t st, int64_t* launches, std::string& err) {
     if (!p || n_events > p->maxev) { err = "MLP: too many events for the plan"; return RFAST_EINVAL; }
     k_mlp_gather<<<dim3(p->Fp / kKBlock, n_events), 256, 0, st>>>(g.ev, g.batch_idx, p->featb, p->Ab, p->AbT, p->rows, p->F, p->Fp);
-    k_mlp_fwd<<<dim3(p->H / kMTile, n_events), kGemmThreads, kFwdSmem, st>>>(
-        p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->F, p->H, p->Fp / kKBlock, p->status);
-    k_mlp_logits<<<dim3(kBatch / 8, n_events), 256, (size_t)p->C * p->H * sizeof(float), st>>>(
-        g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->dlog, p->rows, p->F, p->H, p->C);
     {
-        const dim3 grid(p->H / 64, n_events);
-#define RFAST_BACK(CQ) k_mlp_back<CQ><<<grid, 256, 0, st>>>(g.ev, g.x, g.stride, p->hf, p->dlog, p->dpqT, g.gbuf, g.gplane, p->F, p->H, p->C, g.l2)
+        const int R = p->H / kMTile;
+        const dim3 gf(R, n_events), gb(p->H / 64, n_events);
+#define RFAST_MID(CQ)                                                                                              \
+    k_mlp_fwd<CQ><<<gf, kFwdThreads, kFwdSmem, st>>>(p->tmW1, p->tmA, g.ev, g.x, g.stride, p->hf, p->share, p->F, \
+                                                     p->H, p->C, p->Fp / kKBlock, p->status);                      \
+    k_mlp_back<CQ><<<gb, 256, 0, st>>>(g.ev, g.batch_idx, label, g.x, g.stride, p->hf, p->share, R, p->dpqT,      \
+                                       g.gbuf, g.gplane, p->rows, p->F, p->H, p->C, g.l2)
         switch ((p->C + 3) / 4) {
-            case 1: RFAST_BACK(1); break;
-            case 2: RFAST_BACK(2); break;
-            case 3: RFAST_BACK(3); break;
-            default: RFAST_BACK(4); break;
+            case 1: RFAST_MID(1); break;
+            case 2: RFAST_MID(2); break;
+            case 3: RFAST_MID(3); break;
+            default: RFAST_MID(4); break;
         }
-#undef RFAST_BACK
+#undef RFAST_MID
     }
     k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, dw1_smem(p->NT), st>>>(
         p->tmD, p->tmAT, p->tmX, p->tmG, g.ev, p->n, p->F, p->H, p->NT, g.l2, p->status);
-    *launches += 5;
+    *launches += 4;
     return RFAST_OK;
 }
 
