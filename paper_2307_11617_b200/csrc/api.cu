@@ -71,9 +71,10 @@ struct rfast_ctx {
     int max_round_events = 0;
     int round = 0;
     int64_t launches = 0;
-    cudaGraphExec_t graph_exec = nullptr;   // recorded span of rounds [graph_r0, graph_r1)
+    // recorded span of rounds [graph_r0, graph_r1): a sequence of graphs of about a thousand kernels each
+    struct GraphChunk { cudaGraphExec_t exec; int64_t launches; };
+    std::vector<GraphChunk> graph_chunks;
     int graph_r0 = -1, graph_r1 = -1;
-    int64_t graph_launches = 0;
     size_t dev_bytes = 0, sched_bytes = 0;
     std::string err;
 };
@@ -122,7 +123,8 @@ int upload_rows(rfast_ctx* ctx, float* dst, const float* src, int64_t rows) {
 }
 
 void free_schedule(rfast_ctx* c) {
-    if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+    for (auto& gc : c->graph_chunks) cudaGraphExecDestroy(gc.exec);
+    c->graph_chunks.clear();
     c->graph_r0 = c->graph_r1 = -1;
     for (void* q : c->sched_allocs) cudaFree(q);
     c->sched_allocs.clear();
@@ -623,23 +625,38 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         CK(cudaLaunchCooperativeKernel(persist_kernel(ctx), dim3(ctx->persist_grid), dim3(kThreads), args,
                                        persist_smem(ctx), ctx->stream));
         ctx->launches += 1;
-    } else if (graph_ok && ctx->graph_exec && ctx->graph_r0 == r0 && ctx->graph_r1 == r1) {
-        CK(cudaGraphLaunch(ctx->graph_exec, ctx->stream));
-        ctx->launches += ctx->graph_launches;
+    } else if (graph_ok && !ctx->graph_chunks.empty() && ctx->graph_r0 == r0 && ctx->graph_r1 == r1) {
+        for (const auto& gc : ctx->graph_chunks) {
+            CK(cudaGraphLaunch(gc.exec, ctx->stream));
+            ctx->launches += gc.launches;
+        }
     } else if (graph_ok) {
-        if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
-        const int64_t l0 = ctx->launches;
-        CK(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
-        int rc = issue_rounds(ctx, r0, r1);
-        cudaGraph_t graph = nullptr;
-        cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
-        if (rc != RFAST_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
-        if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("cudaStreamEndCapture: ") + cudaGetErrorString(e));
-        e = cudaGraphInstantiate(&ctx->graph_exec, graph, 0);
-        cudaGraphDestroy(graph);
-        if (e != cudaSuccess) { ctx->graph_exec = nullptr; return set_err(ctx, RFAST_ECUDA, std::string("cudaGraphInstantiate: ") + cudaGetErrorString(e)); }
-        ctx->graph_r0 = r0; ctx->graph_r1 = r1; ctx->graph_launches = ctx->launches - l0;
-        CK(cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+        // The span is recorded as a sequence of graphs of about kChunkLaunches kernels, each
+        // launched as soon as it is instantiated: the device works on one chunk while the host
+        // records the next, so a first run does not wait for the whole span to be captured.
+        constexpr int64_t kChunkLaunches = 1024;
+        for (auto& gc : ctx->graph_chunks) cudaGraphExecDestroy(gc.exec);
+        ctx->graph_chunks.clear();
+        ctx->graph_r0 = ctx->graph_r1 = -1;
+        const int per_round = ctx->model == RFAST_MODEL_QUAD_DIAG ? 1 : ctx->model == RFAST_MODEL_MLP ? 6 : 4;
+        const int chunk_rounds = (int)std::max<int64_t>(2, kChunkLaunches / per_round);
+        for (int ra = r0; ra < r1; ra += chunk_rounds) {
+            const int rb = std::min(r1, ra + chunk_rounds);
+            const int64_t l0 = ctx->launches;
+            CK(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+            int rc = issue_rounds(ctx, ra, rb);
+            cudaGraph_t graph = nullptr;
+            cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+            if (rc != RFAST_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+            if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("cudaStreamEndCapture: ") + cudaGetErrorString(e));
+            cudaGraphExec_t exec = nullptr;
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("cudaGraphInstantiate: ") + cudaGetErrorString(e));
+            ctx->graph_chunks.push_back({exec, ctx->launches - l0});
+            CK(cudaGraphLaunch(exec, ctx->stream));
+        }
+        ctx->graph_r0 = r0; ctx->graph_r1 = r1;
     } else {
         int rc = issue_rounds(ctx, r0, r1);
         if (rc != RFAST_OK) return rc;
