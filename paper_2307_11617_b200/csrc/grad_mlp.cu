@@ -90,6 +90,8 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void*
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // until the stores of all committed groups have read their shared-memory source
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// the same, the most recent group excepted
+__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // makes this thread's shared-memory writes visible to the async (TMA) proxy
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -305,7 +307,7 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
         const int colh = (warp - 2) >> 2;                   // and columns 32 colh .. 32 colh + 31
         const int jl = q * 32 + lane;                       // hidden unit inside the slab
         const float b1 = x[row + ob1 + h0 + jl];
-        const bool ok = mbar_wait(&acc_full, 0);
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full, 0));   // one decision per warp
         tc_fence_after();
         if (!ok) { if (lane == 0) { atomicExch(status, kErrEpilogue); bad = 1; } }
         else if (!bad) {
@@ -462,12 +464,13 @@ k_mlp_back(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, co
 }
 
 // One tile of gW1: hidden units [h0, h0+128) x features [f0, f0+NT) = q(dpre)^T (K = batch) x q(A),
-// plus l2 * W1.  The fp32 side of the epilogue also goes through TMA: the W1 tile of x arrives in
-// shared memory as NT/16 pieces of 128 rows x 16 floats (64-byte swizzle) while the product runs,
-// each epilogue thread adds its accumulator row to its own row of every piece in place, and each
-// warp stores its 32 rows of a piece back with a TMA tile store.  (A thread owns a whole row of
-// the tile, so plain stores would touch 32 different cache lines per instruction.)
-// grid = (H / 128, F / NT, events); dynamic shared memory dw1_smem(NT)
+// plus l2 * W1.  The fp32 side of the epilogue also goes through TMA, in pieces of 32 rows x 16
+// floats (64-byte swizzle): a thread owns a whole row of the accumulator, so plain stores would
+// touch 32 different cache lines per instruction.  Each epilogue warp has a ring of two pieces
+// in shared memory: it adds its accumulator rows to the W1 piece loaded there (or just writes
+// them when there is no regulariser), stores the piece with a TMA tile store, and reuses the
+// slot once that store has read it.  The small footprint lets four CTAs share an SM.
+// grid = (H / 128, F / NT, events); dynamic shared memory kDw1Smem
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmAT,
           const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmG,
@@ -475,21 +478,22 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kABytes = kMTile * kKBlock * 2;          // q(dpre)^T slab
-    constexpr int kPiece = kMTile * 16 * 4;                // 128 rows x 16 floats
+    constexpr int kPiece = 32 * 16 * 4;                    // 32 rows x 16 floats
     uint8_t* sA = smem;
     uint8_t* sB = smem + kABytes;                          // [NT][64] bf16 tile of A^T (at most 16 KB)
-    uint8_t* sX = smem + 2 * kABytes;                      // [NT / 16] pieces
-    __shared__ uint64_t ab_full, acc_full, x_full;
+    uint8_t* ring = smem + 2 * kABytes;                    // [4 warps][2 slots] pieces
+    __shared__ uint64_t ab_full, acc_full, x_full[4][2];
     __shared__ uint32_t tmem_base;
     __shared__ volatile int aborted;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ev = blockIdx.z, h0 = blockIdx.x * kMTile, f0 = blockIdx.y * NT;
     const EvDesc e = evs[ev];
     const bool reg = l2 != 0.f;
+    const int np = NT / 16;
     if (threadIdx.x == 0) {
         mbar_init(&ab_full, 1);
         mbar_init(&acc_full, 1);
-        mbar_init(&x_full, 1);
+        for (int q = 0; q < 4; ++q) { mbar_init(&x_full[q][0], 1); mbar_init(&x_full[q][1], 1); }
         aborted = 0;
         fence_barrier_init();
     }
@@ -503,11 +507,6 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
         mbar_expect_tx(&ab_full, kABytes + NT * kKBlock * 2);
         tma_load_2d(sA, &tmD, &ab_full, 0, ev * H + h0);
         tma_load_2d(sB, &tmAT, &ab_full, 0, ev * F + f0);
-        if (reg) {
-            mbar_expect_tx(&x_full, (NT / 16) * kPiece);
-            for (int pc = 0; pc < NT / 16; ++pc)
-                tma_load_3d(sX + pc * kPiece, &tmX, &x_full, f0 + pc * 16, h0, e.node);
-        }
     } else if (warp == 1 && lane == 0) {                   // ---- MMA issuer
         const uint32_t idesc = umma_idesc_bf16(kMTile, NT);
         const bool ok = mbar_wait(&ab_full, 0);
@@ -526,35 +525,58 @@ k_mlp_dw1(const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUten
             mbar_arrive(&acc_full);
         }
     } else if (warp >= 2) {                                // ---- epilogue: TMEM (+ l2 x) -> shared -> TMA store
-        const int q = warp & 3;
-        const int r = q * 32 + lane;                        // row of the tile = tensor-memory lane
-        bool ok = mbar_wait(&acc_full, 0);
-        tc_fence_after();
-        if (reg) ok = mbar_wait(&x_full, 0) && ok;          // also on the way out: the copies must have landed
-        if (!ok) { if (lane == 0) atomicExch(status, kErrEpilogue); }
-        else if (!aborted) {
-            const int plane = (e.g_par ^ 1) * n + e.node;
-            const int sw = (r >> 1) & 3;                    // 64-byte swizzle: 16-byte chunk index ^ address bits 7..8
-            for (int pc = 0; pc < NT / 16; ++pc) {
-                float v[16];
-                tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + pc * 16, v);
-                float4* rowp = reinterpret_cast<float4*>(sX + pc * kPiece + r * 64);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float4 o = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-                    float4* at = rowp + (c ^ sw);
-                    if (reg) {
-                        const float4 xv = *at;
-                        o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
-                    }
-                    *at = o;
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) tma_store_3d(&tmG, sX + pc * kPiece + q * 32 * 64, f0 + pc * 16, h0 + q * 32, plane);
+        const int q = warp & 3;                             // rows 32q .. 32q+31 of the tile = tensor-memory lanes
+        uint8_t* slot0 = ring + q * 2 * kPiece;
+        const int sw = (lane >> 1) & 3;                     // 64-byte swizzle: 16-byte chunk index ^ address bits 7..8
+        // W1 pieces are requested two ahead: pieces 0 and 1 here, piece pc + 2 when piece pc is stored
+        if (reg && lane == 0)
+            for (int pc = 0; pc < 2 && pc < np; ++pc) {
+                mbar_expect_tx(&x_full[q][pc], kPiece);
+                tma_load_3d(slot0 + pc * kPiece, &tmX, &x_full[q][pc], f0 + pc * 16, h0 + q * 32, e.node);
             }
-            if (lane == 0) { tma_store_commit(); tma_store_wait_read(); }
+        bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full, 0));         // one decision per warp
+        tc_fence_after();
+        const bool run = ok && !aborted;
+        const int plane = (e.g_par ^ 1) * n + e.node;
+        int pc = 0;
+        for (; pc < np; ++pc) {
+            const int s = pc & 1;
+            uint8_t* slot = slot0 + s * kPiece;
+            if (reg) ok = __all_sync(0xffffffffu, mbar_wait(&x_full[q][s], (pc >> 1) & 1)) && ok;
+            if (!run || !ok) break;
+            if (!reg && pc >= 2) {                          // the store of piece pc - 2 has read this slot
+                if (lane == 0) tma_store_wait_read_1();
+                __syncwarp();
+            }
+            float v[16];
+            tmem_ld16(tacc + ((uint32_t)(q * 32) << 16) + pc * 16, v);
+            float4* rowp = reinterpret_cast<float4*>(slot + lane * 64);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float4 o = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                float4* at = rowp + (c ^ sw);
+                if (reg) {
+                    const float4 xv = *at;
+                    o.x = fmaf(l2, xv.x, o.x); o.y = fmaf(l2, xv.y, o.y); o.z = fmaf(l2, xv.z, o.z); o.w = fmaf(l2, xv.w, o.w);
+                }
+                *at = o;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tmG, slot, f0 + pc * 16, h0 + q * 32, plane);
+                tma_store_commit();
+                if (reg && pc + 2 < np) {                   // next W1 piece into this slot, once the store has read it
+                    tma_store_wait_read();
+                    mbar_expect_tx(&x_full[q][s], kPiece);
+                    tma_load_3d(slot, &tmX, &x_full[q][s], f0 + (pc + 2) * 16, h0 + q * 32, e.node);
+                }
+            }
         }
+        // left early: the one piece requested beyond the last one awaited must land before the CTA ends
+        if (reg && pc < np && pc + 1 < np) mbar_wait(&x_full[q][(pc + 1) & 1], ((pc + 1) >> 1) & 1);
+        if (!ok && lane == 0) atomicExch(status, kErrEpilogue);
+        if (lane == 0) tma_store_wait_read();
     }
     tc_fence_before();
     __syncthreads();
@@ -599,7 +621,7 @@ bool make_map(CUtensorMap* m, void* base, int rank, const uint64_t* dims, const 
 }
 
 constexpr size_t kFwdSmem = kStagesFwd * (kMTile * kKBlock * 2 + kBatch * kKBlock * 2) + 16 * kHsPitch * 4 + 1024;
-constexpr size_t dw1_smem(int NT) { return 2 * (size_t)kMTile * kKBlock * 2 + (size_t)(NT / 16) * kMTile * 16 * 4 + 1024; }
+constexpr size_t kDw1Smem = 2 * (size_t)kMTile * kKBlock * 2 + 4 * 2 * (32 * 16 * 4) + 1024;
 
 }  // namespace
 
@@ -648,7 +670,7 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
         // fp32 views of the W1 block: x [n][H][F] and the two gradient planes [2n][H][F]
         const uint64_t dX[3] = {(uint64_t)F, (uint64_t)H, (uint64_t)n}, dG[3] = {(uint64_t)F, (uint64_t)H, (uint64_t)2 * n};
         const uint64_t sX[2] = {(uint64_t)F * 4, (uint64_t)stride * 4};
-        const uint32_t bX[3] = {16, kMTile, 1}, bG[3] = {16, 32, 1};
+        const uint32_t bX[3] = {16, 32, 1}, bG[3] = {16, 32, 1};
         if (!make_map(&p->tmW1, (void*)xb, 3, dW, sW, bW) || !make_map(&p->tmA, p->Ab, 2, dA, sA, bA) ||
             !make_map(&p->tmD, p->dpqT, 2, dD, sD, bD) || !make_map(&p->tmAT, p->AbT, 2, dT, sD, bT) ||
             !make_map(&p->tmX, (void*)x, 3, dX, sX, bX, true) || !make_map(&p->tmG, gbuf, 3, dG, sX, bG, true)) {
@@ -661,7 +683,7 @@ int mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride,
         cudaFuncSetAttribute(k_mlp_fwd<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
         cudaFuncSetAttribute(k_mlp_fwd<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
         cudaFuncSetAttribute(k_mlp_fwd<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFwdSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dw1_smem(p->NT)) != cudaSuccess) {
+        cudaFuncSetAttribute(k_mlp_dw1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDw1Smem) != cudaSuccess) {
         mlp_plan_destroy(p);
         err = "MLP: cannot reserve shared memory";
         return RFAST_ECUDA;
@@ -699,7 +721,7 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
         }
 #undef RFAST_MID
     }
-    k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, dw1_smem(p->NT), st>>>(
+    k_mlp_dw1<<<dim3(p->H / kMTile, p->F / p->NT, n_events), kGemmThreads, kDw1Smem, st>>>(
         p->tmD, p->tmAT, p->tmX, p->tmG, g.ev, p->n, p->F, p->H, p->NT, g.l2, p->status);
     *launches += 4;
     return RFAST_OK;
