@@ -23,8 +23,10 @@ SHAPES = [
     dict(n=8, F=784, H=512, C=10, rows=256, K=15, batch=64),
     dict(n=6, F=160, H=256, C=10, rows=128, K=12, batch=64, l2=1e-2),   # regulariser on: gW1 epilogue adds l2 * W1
     dict(n=3, F=32, H=1152, C=4, rows=64, K=6, batch=64),               # 9 slabs of hidden units share the logits
+    dict(n=4, F=32, H=128, C=16, rows=64, K=6, batch=64),               # the widest output layer (four class quads)
+    dict(n=4, F=32, H=256, C=7, rows=64, K=6, batch=64, l2=1e-3),       # two class quads, the second ragged
 ]
-IDS = ["F64 H128", "F48 H256 C3", "F784 H512", "F160 H256 l2", "F32 H1152"]
+IDS = ["F64 H128", "F48 H256 C3", "F784 H512", "F160 H256 l2", "F32 H1152", "C16", "C7 l2"]
 
 
 def _blocks(wl):
