@@ -202,8 +202,9 @@ int64_t rfast_query(rfast_ctx* ctx, int what);
  *                         the kernel returns and the next synchronising call reports
  *                         RFAST_ETIMEOUT (the state is then undefined, the device healthy:
  *                         rfast_reset starts over).
- *   RFAST_OPT_GRAPHS      1 (default): spans of rounds are recorded into a CUDA graph and
- *                         replayed (non-default streams only); 0: direct launches.
+ *   RFAST_OPT_GRAPHS      1 (default): spans of rounds are recorded into CUDA graphs (chunks of
+ *                         about a thousand kernels, each launched as soon as it is instantiated)
+ *                         and replayed (non-default streams only); 0: direct launches.
  *   RFAST_OPT_WAIT_LIMIT_MS     bound of every device-side barrier wait, 1..60000 (default 2000).
  *   RFAST_OPT_PHANTOM_ARRIVALS  failure injection for tests, made on the host: the grid barrier
  *                         expects this many arrivals that nobody makes, so its bounded wait runs

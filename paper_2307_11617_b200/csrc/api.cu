@@ -599,7 +599,7 @@ int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync) {
         return set_err(ctx, RFAST_ESTATE, "run would pass the end of the schedule");
     const int r0 = ctx->round, r1 = ctx->round + rounds;
     // Many short kernels per round make the launch path the bottleneck of the small problems:
-    // the rounds of one call are recorded once into a CUDA graph and replayed when the same
+    // the rounds of one call are recorded once into CUDA graphs and replayed when the same
     // span is run again (after a reset).  The legacy default stream cannot be captured; there
     // the kernels are launched directly.
     const bool graph_ok = ctx->opt_graphs && ctx->stream != nullptr && rounds >= 2;
