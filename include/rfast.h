@@ -101,7 +101,23 @@ typedef struct rfast_problem {
                               /* 2 = the running sums rho are two floats as well (their fp32         */
                               /* resolution otherwise limits what a receiver sees once they have     */
                               /* grown; doubles the rho traffic)                                     */
+    int32_t     tracker;      /* how the mass in transit over G_C is kept (same mathematics):         */
+                              /* RFAST_TRACKER_RUNNING_SUMS: rho_ji and rho~_ij as Algorithm 1 prints  */
+                              /* them; RFAST_TRACKER_BUCKETS: the edge masses of the augmented system   */
+                              /* (Appendix F), see below                                               */
 } rfast_problem;
+
+/* RFAST_TRACKER_BUCKETS.  S2b consumes rho_ij^{tau_new} - rho~_ij = the sum of a_ij z^{t+1/2}_j over
+ * the sender's local iterations tau_prev < t <= tau_new: the mass that is on the edge, the quantity
+ * the augmented system of Appendix F carries instead of ever-growing running sums.  The schedule is
+ * known in full before the run, so the host knows for every sender activation which receiver
+ * activation will consume its contribution; with this option the sender adds it to a row that
+ * holds exactly the contributions of one such consumption ("bucket") and the receiver adds that
+ * row.  Same result as the running sums in exact arithmetic; in fp32 the subtraction of two
+ * large running sums falls away (no loss of resolution over long horizons), a consumption reads
+ * one row instead of two and a sender reads a row only when the bucket is not empty.  The views
+ * RFAST_STATE_RHO_LATEST and RFAST_STATE_RHO_BUF do not exist with this option (RFAST_ESTATE). */
+enum { RFAST_TRACKER_RUNNING_SUMS = 0, RFAST_TRACKER_BUCKETS = 1 };
 
 /* Raw schedule (value independent).  Round r activates the nodes
  * act_node[act_ptr[r] .. act_ptr[r+1]) (strictly ascending).  Every activation is an

@@ -46,7 +46,7 @@ class _Problem(C.Structure):
                 ("quad_d", C.c_void_p), ("quad_b", C.c_void_p), ("feat", C.c_void_p),
                 ("target", C.c_void_p), ("label", C.c_void_p), ("sp_rowptr", C.c_void_p),
                 ("sp_col", C.c_void_p), ("sp_val", C.c_void_p), ("x0", C.c_void_p),
-                ("compensated", C.c_int32)]
+                ("compensated", C.c_int32), ("tracker", C.c_int32)]
 
 
 class _Schedule(C.Structure):
@@ -117,6 +117,7 @@ def _problem(wl, keep):
     P.model = MODEL_IDS[wl.model] if isinstance(wl.model, str) else int(wl.model)
     P.batch, P.rows = int(wl.batch), int(wl.rows)
     P.compensated = int(getattr(wl, "compensated", 0) or 0)     # False/True/2 -> 0/1/2
+    P.tracker = int(getattr(wl, "tracker", 0) or 0)             # 0 running sums, 1 mass buckets
     dims = getattr(wl, "dims", {}) or {}
     P.n_features = int(dims.get("n_features", 0))
     P.n_classes = int(dims.get("n_classes", 0))

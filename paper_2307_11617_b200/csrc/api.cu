@@ -39,6 +39,7 @@ struct rfast_ctx {
     float *x = nullptr, *z = nullptr, *zc = nullptr, *gbuf = nullptr, *x0 = nullptr;
     bool compensated = false;
     bool rho2 = false;                // compensation level 2: two-float running sums
+    bool buckets = false;             // mass on the G_C edges kept per consumption instead of as running sums
     int64_t rlo_off() const { return rho2 ? (int64_t)comp.n_rho_slots * stride : 0; }
     float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
     int* label = nullptr;
@@ -352,6 +353,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
     ctx->F = prob->n_features; ctx->C = prob->n_classes; ctx->H = prob->n_hidden;
     ctx->compensated = prob->compensated != 0;
     ctx->rho2 = prob->compensated >= 2;
+    ctx->buckets = prob->tracker == RFAST_TRACKER_BUCKETS;
     ctx->stride = (prob->p + 31) / 32 * 32;
     if (ctx->stride / 4 > 0x7fffffff) return set_err(ctx, RFAST_EINVAL, "p too large");
     if ((rc = build_host_graph(prob->G_R, ctx->n, true, ctx->R, err)) != RFAST_OK) return set_err(ctx, rc, "G_R: " + err);
@@ -454,7 +456,7 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     CK(cudaStreamSynchronize(ctx->stream));
     Compiled comp;
     std::string err;
-    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated), comp, err);
+    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated), ctx->buckets, comp, err);
     if (rc != RFAST_OK) return set_err(ctx, rc, err);
     free_schedule(ctx);
     ctx->alpha_round.clear();
@@ -783,6 +785,8 @@ int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
         }
         case RFAST_STATE_RHO_LATEST:
         case RFAST_STATE_RHO_BUF: {
+            if (ctx->buckets)
+                return set_err(ctx, RFAST_ESTATE, "read_state: the bucket tracker keeps no running sums (rho, rho~ views do not exist)");
             std::vector<int> idx(ctx->Cg.E, -1);
             for (int ev = 0; ev < ev_end; ++ev) {
                 const EvDesc& d = c.ev[ev];
@@ -814,7 +818,8 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32
     if ((rc = build_host_graph(prob->G_C, prob->n, false, C, err)) != RFAST_OK) return done(rc);
     if ((rc = check_roots(R, C, prob->root, err)) != RFAST_OK) return done(rc);
     Compiled c;
-    if ((rc = compile_schedule(R, C, s, prob->batch, prob->rows, traffic_of(prob->model, prob->compensated != 0), c, err)) != RFAST_OK) return done(rc);
+    if ((rc = compile_schedule(R, C, s, prob->batch, prob->rows, traffic_of(prob->model, prob->compensated != 0),
+                               prob->tracker == RFAST_TRACKER_BUCKETS, c, err)) != RFAST_OK) return done(rc);
     if (used_tau_v) std::copy(c.used_tau_v.begin(), c.used_tau_v.end(), used_tau_v);
     if (used_tau_rho) std::copy(c.used_tau_rho.begin(), c.used_tau_rho.end(), used_tau_rho);
     if (v_ver)
@@ -865,6 +870,7 @@ CkptHeader make_header(rfast_ctx* c) {
     h.p = c->p; h.stride = c->stride; h.n_events = c->comp.n_events;
     h.n = c->n; h.model = c->model; h.compensated = c->compensated + (c->rho2 ? 1 : 0); h.K = c->comp.K;
     h.n_v_slots = c->comp.n_v_slots; h.n_rho_slots = c->comp.n_rho_slots; h.round = c->round;
+    h.pad = c->buckets ? 1 : 0;
     return h;
 }
 
@@ -923,15 +929,27 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     if (!ctx || !out || n_out != 5) return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5") : RFAST_EINVAL;
     if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
     const Compiled& c = ctx->comp;
-    const int n = ctx->n, E = ctx->Cg.E;
+    const int n = ctx->n;
+    int E = ctx->Cg.E;
     // which rows hold the current g, the latest rho and the buffered rho of every edge
     std::vector<int> gsel(n), latest(std::max(E, 1), -1), buf(std::max(E, 1), -1), t(n, 0);
     const int ev_end = c.act_ptr[ctx->round];
     for (int ev = 0; ev < ev_end; ++ev) {
         const EvDesc& d = c.ev[ev];
         t[d.node]++;
+        if (ctx->buckets) continue;
         for (int k = 0; k < d.out_cnt; ++k) latest[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
         for (int k = 0; k < d.news_cnt; ++k) buf[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
+    }
+    if (ctx->buckets) {
+        // the mass in transit is the content of the buckets begun and not yet consumed
+        latest.clear();
+        for (size_t v = 0; v < c.rho_leader.size(); ++v)
+            if (c.rho_leader[v] == (int64_t)v && c.rho_write[v] < ctx->round && c.rho_last[v] >= ctx->round)
+                latest.push_back(c.rho_slot[v]);
+        E = (int)latest.size();
+        if (latest.empty()) latest.push_back(-1);
+        buf.assign(latest.size(), -1);
     }
     for (int i = 0; i < n; ++i) gsel[i] = (t[i] & 1) * n + i;
     const int blocks = (int)((ctx->p + kThreads - 1) / kThreads);

@@ -128,7 +128,7 @@ inline int deliver(std::vector<Pend>& q, int r, int tau) {
 }  // namespace
 
 int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedule* s, int batch,
-                     int rows, const ModelTraffic& mt, Compiled& out, std::string& err) {
+                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err) {
     const int n = R.n;
     if (!s || s->K < 0 || !s->act_ptr) return fail(err, RFAST_ESCHED, "schedule: null or K < 0");
     const int K = s->K;
@@ -141,6 +141,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     Compiled c;
     c.K = K;
     c.n_events = nE;
+    c.buckets = buckets;
     c.act_ptr.assign(s->act_ptr, s->act_ptr + K + 1);
     c.act_node.assign(s->act_node, s->act_node + nE);
     c.in_r_off.assign(nE + 1, 0);
@@ -190,6 +191,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     const int64_t nRho = c.out_c_off[nE];
     c.rho_write.assign(nRho, 0);
     std::vector<int> rho_last_sender(nRho, 0), rho_last_recv(nRho, -1);
+    if (buckets) c.rho_leader.assign(nRho, -1);
     for (int r = 0; r < K; ++r) {
         for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
             const int i = c.act_node[ev];
@@ -207,7 +209,12 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
                 int tau = deliver(pend_c[e], r, prev);
                 c.used_tau_rho.push_back(tau);
                 c.prev_tau_rho.push_back(prev);
-                if (tau > prev) {                      // news: rho[tau] - rho[prev] is read
+                if (tau > prev && buckets) {           // news: the contributions of stamps prev+1 .. tau, one row
+                    const auto& evs = ev_of[C.col[e]];
+                    const int64_t lead = c.out_c_off[evs[prev]] + C.opos[e];
+                    for (int st = prev + 1; st <= tau; ++st) c.rho_leader[c.out_c_off[evs[st - 1]] + C.opos[e]] = lead;
+                    rho_last_recv[lead] = r;
+                } else if (tau > prev) {               // news: rho[tau] - rho[prev] is read
                     const auto& evs = ev_of[C.col[e]];
                     int64_t vn = c.out_c_off[evs[tau - 1]] + C.opos[e];
                     rho_last_recv[vn] = std::max(rho_last_recv[vn], r);
@@ -219,7 +226,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
                 tau_rho[e] = tau;
             }
             const int stamp = ++t[i];
-            if (stamp >= 2) {                          // S2c reads the sender's current running sums
+            if (stamp >= 2 && !buckets) {              // S2c reads the sender's current running sums
                 int64_t base = c.out_c_off[ev_of[i][stamp - 2]];
                 for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = r;
             }
@@ -245,6 +252,18 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     c.tau_v_end = tau_v;
     c.tau_rho_end = tau_rho;
     c.t_end = t;
+    if (buckets) {
+        // contributions nobody consumes inside the schedule: one last bucket per edge, kept
+        for (int e = 0; e < C.E; ++e) {
+            const int j = C.col[e];
+            if (t[j] <= tau_rho[e]) continue;
+            const int64_t lead = c.out_c_off[ev_of[j][tau_rho[e]]] + C.opos[e];
+            for (int st = tau_rho[e] + 1; st <= t[j]; ++st) c.rho_leader[c.out_c_off[ev_of[j][st - 1]] + C.opos[e]] = lead;
+            rho_last_recv[lead] = INF;
+        }
+        c.rho_last.resize(nRho);
+        for (int64_t v = 0; v < nRho; ++v) c.rho_last[v] = rho_last_recv[c.rho_leader[v]];
+    } else {
     // what is current at the end of the schedule stays readable: each sender's latest running
     // sums and each receiver's buffered version
     for (int i = 0; i < n; ++i)
@@ -257,6 +276,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             rho_last_recv[c.out_c_off[ev_of[C.col[e]][tau_rho[e] - 1]] + C.opos[e]] = INF;
     c.rho_last.resize(nRho);
     for (int64_t v = 0; v < nRho; ++v) c.rho_last[v] = std::max(rho_last_sender[v], rho_last_recv[v]);
+    }
 
     // ---- pass 2: rows.  A row is free again in the round after its version's last read -------
     c.v_slot.assign(nE, -1);
@@ -284,6 +304,15 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             for (int k = 0; k < C.outdeg(i); ++k) {
                 int64_t vid = c.out_c_off[ev] + k;
                 int slot = -1;
+                if (buckets) {                         // the first contribution of a bucket takes a row, the others share it
+                    const int64_t lead = c.rho_leader[vid];
+                    if (lead != vid) { c.rho_slot[vid] = c.rho_slot[lead]; continue; }
+                    if (!free_c.empty()) { slot = free_c.back(); free_c.pop_back(); }
+                    else slot = c.n_rho_slots++;
+                    c.rho_slot[vid] = slot;
+                    if (c.rho_last[vid] != INF && c.rho_last[vid] + 1 < K) rel_c[c.rho_last[vid] + 1].push_back(vid);
+                    continue;
+                }
                 if (stamp_of[ev] >= 2) {
                     // in place: the previous version is read for the last time here, by this
                     // very update, and no receiver reads it in this round or later
@@ -337,9 +366,10 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
                 if (tau <= prev) continue;             // nothing newer: rho[tau] - rho~ = 0
                 const auto& evs = ev_of[C.col[e]];
                 c.news_new.push_back(c.rho_slot[c.out_c_off[evs[tau - 1]] + C.opos[e]]);
-                c.news_prev.push_back(prev >= 1 ? c.rho_slot[c.out_c_off[evs[prev - 1]] + C.opos[e]] : -1);
+                const bool sub = !buckets && prev >= 1;   // a bucket holds the difference itself
+                c.news_prev.push_back(sub ? c.rho_slot[c.out_c_off[evs[prev - 1]] + C.opos[e]] : -1);
                 c.news_edge.push_back(e);
-                news_streams += 1 + (prev >= 1);
+                news_streams += 1 + sub;
             }
             d.news_cnt = (int32_t)c.news_new.size() - d.news_beg;
             d.out_beg = (int32_t)c.out_new.size();
@@ -347,7 +377,10 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             for (int k = 0; k < C.outdeg(i); ++k) {
                 int e = C.oeid[C.optr[i] + k];
                 int cur = -1;
-                if (stamp_of[ev] >= 2) cur = c.rho_slot[c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k];
+                if (buckets) {                         // add to the bucket unless this is its first contribution
+                    const int64_t vid = c.out_c_off[ev] + k;
+                    if (c.rho_leader[vid] != vid) cur = c.rho_slot[vid];
+                } else if (stamp_of[ev] >= 2) cur = c.rho_slot[c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k];
                 c.out_cur.push_back(cur);
                 c.out_new.push_back(c.rho_slot[c.out_c_off[ev] + k]);
                 c.out_a.push_back(C.w[e]);

@@ -49,6 +49,10 @@ struct Compiled {
     std::vector<int> v_slot, v_write, v_last;
     std::vector<int> rho_slot, rho_write, rho_last;
     int n_v_slots = 0, n_rho_slots = 0;
+    // mass-bucket tracker: the contributions consumed together share a row; rho_leader[v] is the
+    // first of them (it owns the row; rho_write / rho_last of a leader: first write, consumption)
+    bool buckets = false;
+    std::vector<int64_t> rho_leader;
     // device descriptors
     std::vector<EvDesc> ev;
     std::vector<int>    mix_slot;  std::vector<float> mix_w;
@@ -80,6 +84,6 @@ struct ModelTraffic {
 int build_host_graph(const rfast_graph& g, int n, bool row_stochastic, HostGraph& out, std::string& err);
 int check_roots(const HostGraph& R, const HostGraph& C, int root, std::string& err);
 int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedule* s, int batch,
-                     int rows, const ModelTraffic& mt, Compiled& out, std::string& err);
+                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err);
 
 }  // namespace rfast

@@ -164,3 +164,58 @@ def test_create_fails_loudly_without_a_device(rfast_lib):
     with pytest.raises(RFastError) as ei:
         pkg.rfast_create(wl)
     assert ei.value.code == ECUDA
+
+
+@pytest.mark.parametrize("name,ov", CASES)
+def test_bucket_tracker_rows_hold_exactly_one_consumption(rfast_lib, name, ov):
+    """Mass-bucket tracker: the contributions a receiver consumes together (sender stamps
+    tau_prev < t <= tau_new, Algorithm 1 S2b) share one row from the first of them to the
+    consumption and no other bucket uses that row meanwhile; what nobody consumes inside the
+    schedule forms one last bucket per edge that is kept.  The stamps are the brute-force ones."""
+    import paper_2307_11617_b200 as pkg
+    wl = build_config(name, seed=5, tracker=1, **ov)
+    s = wl.schedule
+    r = pkg.rfast_compile_host(wl, s)
+    ref = pkg.rfast_compile_host(build_config(name, seed=5, **ov), s)
+    assert list(r["used_tau_rho"]) == list(ref["used_tau_rho"]) and list(r["used_tau_v"]) == list(ref["used_tau_v"])
+    assert r["streams"] <= ref["streams"]
+    rho = r["rho_ver"]
+    ev_round = np.repeat(np.arange(s.K), np.diff(s.act_ptr))
+    outC = out_edges(wl.G_C)
+    off = np.concatenate([[0], np.cumsum([len(outC[i]) for i in s.act_node])])
+    pos = {f: k for i in range(wl.n) for k, f in enumerate(outC[i])}
+    ev_of = [[] for _ in range(wl.n)]
+    for ev, i in enumerate(s.act_node):
+        ev_of[i].append(ev)
+    vid = lambda e, stamp: off[ev_of[wl.G_C.col[e]][stamp - 1]] + pos[e]
+    sr, _ = brute_force_stamps(wl.G_C, s, s.send_c)
+    INF = np.iinfo(np.int32).max
+    buckets = []                                       # (row, first write round, consume round)
+    k = 0
+    prev = [0] * wl.G_C.n_edges
+    for ev, i in enumerate(s.act_node):
+        for e in range(wl.G_C.rowptr[i], wl.G_C.rowptr[i + 1]):
+            tau = sr[k]; k += 1
+            if tau > prev[e]:
+                members = [vid(e, st) for st in range(prev[e] + 1, tau + 1)]
+                rows = {int(rho[m][0]) for m in members}
+                assert len(rows) == 1
+                assert all(int(rho[m][2]) == ev_round[ev] for m in members)
+                assert all(int(rho[m][1]) < ev_round[ev] for m in members)
+                buckets.append((rows.pop(), int(rho[members[0]][1]), int(ev_round[ev])))
+                prev[e] = tau
+    t = [len(a) for a in ev_of]
+    for e in range(wl.G_C.n_edges):
+        j = int(wl.G_C.col[e])
+        if t[j] > prev[e]:
+            members = [vid(e, st) for st in range(prev[e] + 1, t[j] + 1)]
+            rows = {int(rho[m][0]) for m in members}
+            assert len(rows) == 1 and all(int(rho[m][2]) == INF for m in members)
+            buckets.append((rows.pop(), int(rho[members[0]][1]), INF))
+    assert sum(1 for _ in buckets) > 0
+    by_row = {}
+    for row, first, last in sorted(buckets, key=lambda b: b[1]):
+        assert 0 <= row < r["rho_rows"]
+        if row in by_row:
+            assert by_row[row] < first, "bucket row reused before its consumption"
+        by_row[row] = last

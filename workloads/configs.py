@@ -50,6 +50,8 @@ class Workload:
     meta: dict = field(default_factory=dict)
     compensated: int = 0            # tracker arithmetic asked of the engine: 0 plain fp32, 1 two-float
                                     # tracker, 2 two-float tracker and running sums
+    tracker: int = 0                # how the engine keeps the mass on the G_C edges: 0 running sums
+                                    # (Algorithm 1 as printed), 1 one row per consumption ("buckets")
 
     def __post_init__(self):
         # scalars are handed to every consumer as the fp32-representable value
@@ -82,18 +84,12 @@ def _gaussian_mixture(n, rows, F, C, classes_per_node, rng, scale):
 
 def build_config(name: str, seed: int = 0, **ov) -> Workload:
     """ov overrides: n, p, rows, K, F (features), H (hidden), C (classes), batch, drop,
-    max_delay, alpha, nnz (per sparse row)."""
-    if name == "ls_ring4":
-        return _ls_ring(seed, ov)
-    if name == "softmax_exp16":
-        return _softmax_exp(seed, ov)
-    if name == "mlp_tree64":
-        return _mlp_tree(seed, ov)
-    if name == "quad_tree64":
-        return _quad_tree(seed, ov)
-    if name == "logistic_tree1024":
-        return _logistic_tree(seed, ov)
-    raise KeyError(name)
+    max_delay, alpha, nnz (per sparse row), compensated, tracker."""
+    builders = {"ls_ring4": _ls_ring, "softmax_exp16": _softmax_exp, "mlp_tree64": _mlp_tree,
+                "quad_tree64": _quad_tree, "logistic_tree1024": _logistic_tree}
+    wl = builders[name](seed, ov)
+    wl.tracker = int(ov.get("tracker", 0))
+    return wl
 
 
 # -- config 1: n=4 directed ring, heterogeneous least squares, full batch ---------------------
