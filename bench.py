@@ -123,14 +123,14 @@ def whole_job_rate(units_per_rank: int, world: int, seconds: float) -> float:
     return world * units_per_rank / seconds
 
 
-def build_workload(name, small=False):
+def build_workload(name, small=False, tracker="sums"):
     from workloads import build_config
+    ov = {}
     if small:
         ov = {"quad_tree64": dict(p=1_500_000, K=20), "softmax_exp16": dict(K=200, rows=128),
               "logistic_tree1024": dict(K=20, rows=8), "mlp_tree64": dict(K=10, rows=128),
               "ls_ring4": {}}[name]
-        return build_config(name, seed=0, **ov)
-    return build_config(name, seed=0)
+    return build_config(name, seed=0, tracker=1 if tracker == "buckets" else 0, **ov)
 
 
 def oracle_sample(wl, budget_s=15.0):
@@ -171,7 +171,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = build_workload(args.config, args.small)
+    wl = build_workload(args.config, args.small, getattr(args, "tracker", "sums"))
     vals, desc = [], ""
     for _ in range(args.warmup + args.steps):
         v, desc, _dt = oracle_sample(wl, budget_s=8.0)
@@ -195,6 +195,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--config", default="quad_tree64")
     ap.add_argument("--small", action="store_true", help="reduced size (profiling captures)")
+    ap.add_argument("--tracker", default="sums", choices=["sums", "buckets"],
+                    help="running sums as Algorithm 1 prints them (default) or one row per consumption")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -217,7 +219,7 @@ def main():
     from paper_2307_11617_b200 import binding as B
 
     t_gen = time.perf_counter()
-    wl = build_workload(args.config, args.small)
+    wl = build_workload(args.config, args.small, getattr(args, "tracker", "sums"))
     t_gen = time.perf_counter() - t_gen
     stream = torch.cuda.Stream()
     t_create = time.perf_counter()
@@ -305,7 +307,7 @@ def main():
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": wl.name, "n": wl.n, "p": wl.p, "rounds": K_rounds,
-                           "activations_per_step": events, "small": bool(args.small),
+                           "activations_per_step": events, "small": bool(args.small), "tracker": args.tracker,
                            "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
                            "reset_between_steps": "untimed", "parallelism": f"replicas x{world}"},
                 "param_updates_per_s": value * wl.p, "gpu_launches": int(launches),
