@@ -197,6 +197,9 @@ def main():
     ap.add_argument("--small", action="store_true", help="reduced size (profiling captures)")
     ap.add_argument("--tracker", default="sums", choices=["sums", "buckets"],
                     help="running sums as Algorithm 1 prints them (default) or one row per consumption")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "coords"],
+                    help="with N GPUs: N independent replicas (default), or the coordinates of the "
+                         "element-wise problem split over the GPUs (no exchange; strong scaling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -220,6 +223,11 @@ def main():
 
     t_gen = time.perf_counter()
     wl = build_workload(args.config, args.small, getattr(args, "tracker", "sums"))
+    full_p = wl.p
+    sharded = args.shard == "coords" and world > 1
+    if sharded:
+        from workloads import shard_coordinates
+        wl = shard_coordinates(wl, rank, world)      # same schedule, this rank's slice of every vector
     t_gen = time.perf_counter() - t_gen
     stream = torch.cuda.Stream()
     t_create = time.perf_counter()
@@ -261,7 +269,8 @@ def main():
     ms = [a.elapsed_time(b) for a, b in pairs]
     ms_step = float(sum(ms) / len(ms))
     ms_step = max_over_ranks(ms_step, "cuda")
-    value = whole_job_rate(events, world, ms_step * 1e-3)
+    # coordinate shards: every rank runs every activation on its slice, the job's rate is one rank's
+    value = whole_job_rate(events, 1 if sharded else world, ms_step * 1e-3)
 
     # end to end through the C ABI with host buffers: schedule arrays in (compiled and uploaded),
     # the run, x and y back into pinned host memory
@@ -283,7 +292,7 @@ def main():
         barrier()
         dt = (time.perf_counter() - t0) / reps
         dt = max_over_ranks(dt, "cuda")
-        e2e = {"value": whole_job_rate(events, world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        e2e = {"value": whole_job_rate(events, 1 if sharded else world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3}
 
     peak, peak_kind = measured_peaks()
@@ -305,12 +314,12 @@ def main():
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": wl.name, "n": wl.n, "p": wl.p, "rounds": K_rounds,
+                "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": wl.name, "n": wl.n, "p": full_p, "rounds": K_rounds,
                            "activations_per_step": events, "small": bool(args.small), "tracker": args.tracker,
                            "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
-                           "reset_between_steps": "untimed", "parallelism": f"replicas x{world}"},
-                "param_updates_per_s": value * wl.p, "gpu_launches": int(launches),
+                           "reset_between_steps": "untimed", "parallelism": f"coordinate shards x{world}" if sharded else f"replicas x{world}"},
+                "param_updates_per_s": value * full_p, "gpu_launches": int(launches),
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                 "setup_s": {"generate": t_gen, "create": t_create, "load_schedule": t_load},
                 "device_bytes": eng.query(B.Q_DEVICE_BYTES),

@@ -18,6 +18,14 @@ def _worker(rank, world, port, out):
     import bench
     dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
     ms = bench.max_over_ranks(10.0 + 5.0 * rank)            # rank 1 is the slow replica
+    # coordinate shards: each rank builds its own slice from (rank, world); the slices tile p
+    from workloads import build_config, shard_coordinates
+    wl = build_config("quad_tree64", seed=0, n=8, p=1001, K=4)
+    lo, hi = shard_coordinates(wl, rank, world).meta["coordinates"]
+    import torch
+    spans = [torch.zeros(2, dtype=torch.int64) for _ in range(world)]
+    dist.all_gather(spans, torch.tensor([lo, hi]))
+    assert spans[0][0] == 0 and spans[-1][1] == wl.p and all(int(a[1]) == int(b[0]) for a, b in zip(spans, spans[1:]))
     out.put((rank, ms, bench.whole_job_rate(1000, world, ms * 1e-3)))
     dist.barrier()
     dist.destroy_process_group()

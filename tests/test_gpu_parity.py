@@ -321,3 +321,26 @@ def test_parity_on_general_digraphs(rfast_lib, name, ov, comp):
         d = eng.diagnostics()
     scale = np.abs(orc.G()).sum(axis=0).max()
     assert d["conservation_residual"] <= 2e-5 * scale
+
+
+def test_coordinate_shards_reproduce_the_whole_bit_for_bit(rfast_lib):
+    """The element-wise problem split by coordinate (what `bench.py --shard coords` gives each
+    GPU) needs no exchange: three ragged slices run one after the other on this GPU give, side
+    by side, exactly the state of the whole problem."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    from workloads import shard_coordinates
+    wl = build_config("quad_tree64", seed=6, n=16, p=70_001, K=30)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        X, Y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+    xs, ys = [], []
+    for k in range(3):
+        sub = shard_coordinates(wl, k, 3)
+        with pkg.Engine(sub) as eng:
+            eng.load_schedule(sub.schedule)
+            eng.run()
+            xs.append(eng.read(B.STATE_X)); ys.append(eng.read(B.STATE_Y))
+    assert np.array_equal(np.concatenate(xs, axis=1), X)
+    assert np.array_equal(np.concatenate(ys, axis=1), Y)

@@ -107,3 +107,29 @@ def test_ack_gated_schedule_never_has_two_unacknowledged_packets():
                     recv = int(np.searchsorted(G_R.rowptr, e, side="right") - 1)
                     later = [q for q in act_rounds[recv] if q >= r + 1 + code]
                     pending[e] = later[0] if later else K + 1
+
+
+def test_coordinate_shards_partition_the_problem_and_the_oracle_agrees():
+    """The element-wise objective splits by coordinate with no exchange: the slices cover p
+    exactly once, and the oracle run slice by slice equals the oracle run on the whole."""
+    from oracle import from_workload, make_model, run_schedule
+    from workloads import shard_coordinates
+    wl = build_config("quad_tree64", seed=4, n=12, p=1003, K=25)
+    parts = [shard_coordinates(wl, k, 7) for k in range(7)]
+    spans = [q.meta["coordinates"] for q in parts]
+    assert spans[0][0] == 0 and spans[-1][1] == wl.p
+    assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+    assert max(hi - lo for lo, hi in spans) - min(hi - lo for lo, hi in spans) <= 1
+    whole = from_workload(wl, make_model(wl).grad)
+    whole.init_gradients()
+    run_schedule(whole, wl.schedule)
+    X, Z = [], []
+    for q in parts:
+        o = from_workload(q, make_model(q).grad)
+        o.init_gradients()
+        run_schedule(o, q.schedule)
+        X.append(o.X()); Z.append(o.Z())
+    assert np.array_equal(np.concatenate(X, axis=1), whole.X())
+    assert np.array_equal(np.concatenate(Z, axis=1), whole.Z())
+    with pytest.raises(ValueError):
+        shard_coordinates(build_config("ls_ring4", seed=0), 0, 2)

@@ -14,12 +14,12 @@ from .graphs import (Graph, graph_from_edges, ring_graphs, tree_graphs,
 from .schedules import (Schedule, make_schedule, make_schedule_ack_gated, activation_bernoulli,
                         activation_uniform_subset, activation_durations,
                         activation_all, realised_T_D)
-from .configs import CONFIG_NAMES, build_config, Workload
+from .configs import CONFIG_NAMES, build_config, shard_coordinates, Workload
 
 __all__ = [
     "Graph", "graph_from_edges", "ring_graphs", "tree_graphs",
     "binary_tree_parents", "exponential_tree_parents", "random_tree_parents",
     "sender_csr", "Schedule", "make_schedule", "make_schedule_ack_gated", "activation_bernoulli",
     "activation_uniform_subset", "activation_durations", "activation_all",
-    "realised_T_D", "CONFIG_NAMES", "build_config", "Workload",
+    "realised_T_D", "CONFIG_NAMES", "build_config", "shard_coordinates", "Workload",
 ]

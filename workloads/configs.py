@@ -211,3 +211,27 @@ def _logistic_tree(seed, ov):
                           "label": label},
                     schedule=sch, meta={"K": K, "drop": drop, "max_delay": max_delay,
                                         "stragglers": sorted(strag)})
+
+
+def shard_coordinates(wl: Workload, part: int, parts: int) -> Workload:
+    """The slice of an element-wise problem that one of `parts` devices owns.
+
+    Every step of an activation (S1, S2a, the gradient d^2 (x - b), S2b, S2c) acts coordinate by
+    coordinate when the objective is the diagonal quadratic, so the problem splits by
+    coordinate with no exchange at all: each part runs the same schedule on its slice and the
+    concatenation of the parts' states is the state of the whole.  Slices are contiguous, as
+    equal as possible, the first p mod parts of them one coordinate longer."""
+    if wl.model != MODEL_QUAD_DIAG:
+        raise ValueError("only the element-wise objective splits by coordinate without exchange")
+    if not (0 <= part < parts <= wl.p):
+        raise ValueError("need 0 <= part < parts <= p")
+    base, extra = divmod(wl.p, parts)
+    lo = part * base + min(part, extra)
+    hi = lo + base + (1 if part < extra else 0)
+    data = {k: np.ascontiguousarray(v[:, lo:hi]) for k, v in wl.data.items()}
+    x0 = None if wl.x0 is None else np.ascontiguousarray(wl.x0[:, lo:hi])
+    sub = Workload(wl.name, wl.n, hi - lo, wl.root, wl.alpha, wl.G_R, wl.G_C, wl.model, wl.batch, wl.l2,
+                   wl.rows, dims=dict(wl.dims), data=data, x0=x0, schedule=wl.schedule,
+                   meta=dict(wl.meta, coordinates=(lo, hi)), compensated=wl.compensated)
+    sub.tracker = wl.tracker
+    return sub
