@@ -247,7 +247,9 @@ int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
  *   out[0] consensus error  || x - 1 xbar^T ||_F        (xbar = mean of the x_i)
  *   out[1] || xbar ||_2
  *   out[2] conservation residual of Lemma 3:
- *          max_c | sum_i z_i + sum_e (rho_e - rho~_e) - sum_i g_i |   (0 up to rounding)
+ *          max_c | sum_i z_i + sum_e (rho_e - rho~_e) - sum_i g_i |   (0 up to rounding; with
+ *          RFAST_TRACKER_BUCKETS the mass in transit sum_e (rho_e - rho~_e) is the content of the
+ *          buckets begun and not yet consumed)
  *   out[3] max_c | sum_i g_i |   (the scale of out[2])
  *   out[4] || z ||_F
  * n_out must be 5 (RFAST_EINVAL otherwise); out is a caller-owned HOST array of doubles. */
