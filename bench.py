@@ -303,7 +303,7 @@ def main():
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
                 "algorithmic_bytes_per_launch": bytes_step / max(1, launches // max(1, args.steps)),
                 "traffic": (fused_traffic_ratio() and fused_traffic_ratio() * bytes_step / max(1, launches // max(1, args.steps)))
-                if wl.model == "quad_diag" else None,
+                if wl.model == "quad_diag" and args.tracker == "sums" else None,   # the counters were taken on that workload
                 "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
 
     cpu = None
