@@ -116,3 +116,47 @@ def test_bucket_tracker_checkpoint_resume_and_stepping(rfast_lib):
         eng.load_schedule(wl.schedule)
         with pytest.raises(pkg.binding.RFastError):
             eng.restore(foreign)
+
+
+def _sweep_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for it in range(count):
+        model = ["quad_tree64", "ls_ring4", "softmax_exp16", "logistic_tree1024"][it % 4]
+        ov = dict(K=int(rng.integers(1, 40)), drop=float(rng.choice([0.0, 0.3, 0.6])),
+                  max_delay=int(rng.choice([0, 3, 10])), tracker=int(rng.integers(0, 2)),
+                  compensated=int(rng.integers(0, 3)))
+        if model == "quad_tree64":
+            ov.update(n=int(rng.integers(1, 24)), p=int(rng.choice([1, 3, 5, 1023, 1024, 1025, 4097, 9001])))
+        elif model == "ls_ring4":
+            ov.update(n=int(rng.integers(1, 10)), p=int(rng.choice([1, 7, 10, 33, 300, 1030])), rows=int(rng.integers(2, 40)))
+        elif model == "softmax_exp16":
+            ov.update(n=int(2 ** rng.integers(0, 5)), F=int(rng.choice([5, 16, 96, 100])), C=int(rng.integers(2, 9)),
+                      rows=int(rng.integers(8, 40)), batch=int(rng.integers(1, 9)))
+        else:
+            p = int(rng.choice([50, 999, 4096, 5000, 9000]))
+            ov.update(n=int(rng.integers(2, 40)), p=p, rows=int(rng.integers(2, 10)), batch=int(rng.integers(1, 5)),
+                      nnz=int(rng.integers(1, min(p, 60))))
+        cases.append((model, ov, int(rng.integers(0, 1000))))
+    return cases
+
+
+@pytest.mark.parametrize("model,ov,seed", _sweep_cases(32, 2024),
+                         ids=[f"{i}-{c[0].split('_')[0]}" for i, c in enumerate(_sweep_cases(32, 2024))])
+def test_seeded_sweep_of_shapes_losses_trackers_and_arithmetics(rfast_lib, model, ov, seed):
+    """Ragged and degenerate shapes (one node, one coordinate, tile size +- 1, one sampled row),
+    no loss to 60 % loss, delays up to 10 rounds, both trackers, the three tracker arithmetics:
+    x and y at 1e-5, stamps bit-exact, Lemma 3 on the device state."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config(model, seed=seed, **ov)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        x, y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        assert eng.read(B.STATE_USED_TAU_V).tolist() == orc.used_tau_v
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
+        d = eng.diagnostics()
+    assert rel_l2(x, orc.X(), ref0[0]) <= TOL and rel_l2(y, orc.Z(), ref0[1]) <= TOL
+    assert d["conservation_residual"] <= 1e-5 * max(np.abs(orc.G()).sum(axis=0).max(), 1e-30)
