@@ -336,6 +336,9 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     // ---- pass 3: device descriptors and the method's traffic ---------------------------------
     c.ev.resize(nE);
     c.round_streams.assign(K + 1, 0);
+    c.mix_slot.reserve(c.in_r_off[nE]);  c.mix_w.reserve(c.in_r_off[nE]);
+    c.news_new.reserve(c.in_c_off[nE]);  c.news_prev.reserve(c.in_c_off[nE]);  c.news_edge.reserve(c.in_c_off[nE]);
+    c.out_cur.reserve(nRho);  c.out_new.reserve(nRho);  c.out_a.reserve(nRho);  c.out_edge.reserve(nRho);
     for (int r = 0; r < K; ++r) {
         int64_t streams = 0;
         for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
