@@ -569,6 +569,8 @@ k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restri
 // tile_ptr[r][t] = index of the first entry of shard row r with column >= t * kLogitTile
 // (computed once per problem on the host), so no search is needed here.
 // grid = (tiles, events), 256 threads
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 constexpr int kLogitSub = 4;                               // passes of kThreads float4 per tile
 constexpr int kLogitTile = kLogitSub * 4 * kThreads;
 template <bool COMP>
@@ -587,6 +589,33 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int
     const int64_t row = (int64_t)e.node * g.stride;
     const int64_t c0 = (int64_t)blockIdx.x * kLogitTile;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // The tracking part at the end is a chain of dependent loads per sub-pass (edge lists -> row
+    // ids -> rows); its operands are requested into L2 now, while the tile is assembled: the
+    // lists into shared memory (the later reads then hit L1), the rows by prefetch, one request
+    // per 128-byte line.
+    constexpr int kPre = 16;
+    __shared__ int pre_row[3 * kPre];
+    const float* gold = g.gbuf + (int64_t)e.g_par * g.gplane + row;
+    if (!init_only) {
+        if (threadIdx.x < 3 * kPre) {
+            const int m = threadIdx.x % kPre, what = threadIdx.x / kPre;
+            int id = -1;
+            if (what == 0 && m < e.news_cnt) id = a.news_new[e.news_beg + m];
+            if (what == 1 && m < e.news_cnt) id = a.news_prev[e.news_beg + m];
+            if (what == 2 && m < e.out_cnt) id = a.out_cur[e.out_beg + m];
+            pre_row[threadIdx.x] = id;
+        }
+        if ((lane & 7) == 0) {
+#pragma unroll
+            for (int sub = 0; sub < kLogitSub; ++sub) {
+                const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
+                if (i4 < a.n4) {
+                    prefetch_l2(a.z + row + (int64_t)i4 * 4);
+                    prefetch_l2(gold + (int64_t)i4 * 4);
+                }
+            }
+        }
+    }
 #pragma unroll
     for (int sub = 0; sub < kLogitSub; ++sub) {
         const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
@@ -613,6 +642,18 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int
         }
         __syncthreads();
         const int total = pref_s[nb];
+        if (k0 == 0 && !init_only && (lane & 7) == 0) {          // pre_row is visible since the barriers above
+            for (int m = 0; m < 3 * kPre; ++m) {
+                const int id = pre_row[m];
+                if (id < 0) continue;
+                const float* rr = a.rbuf + (int64_t)id * a.stride;
+#pragma unroll
+                for (int sub = 0; sub < kLogitSub; ++sub) {
+                    const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
+                    if (i4 < a.n4) prefetch_l2(rr + (int64_t)i4 * 4);
+                }
+            }
+        }
         if (total <= kStage) {
             // all entries of this tile are fetched at once (one memory latency), then one warp
             // adds them row after row so that the order of additions is the same on every run
@@ -641,7 +682,6 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int
     }
     __syncthreads();
     float* zr = a.z + row;
-    const float* gold = g.gbuf + (int64_t)e.g_par * g.gplane + row;
     float* gnew = g.gbuf + (int64_t)(e.g_par ^ 1) * g.gplane + row;
     for (int sub = 0; sub < kLogitSub; ++sub) {
         const int base = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
