@@ -44,8 +44,8 @@ struct rfast_ctx {
     float *quad_d = nullptr, *quad_b = nullptr, *feat = nullptr, *target = nullptr;
     int* label = nullptr;
     int64_t* sp_ptr = nullptr;
-    int64_t* sp_tile_ptr = nullptr;   // [n*rows][tiles+1] first entry of each shard row in each coordinate tile
-    int sp_tiles = 0;
+    int64_t* sp_tile_ptr = nullptr;   // [n*rows][ranges+1] first entry of each shard row in each range of 512 coordinates
+    int sp_tiles = 0, sp_ranges = 0;
     int* sp_col = nullptr;
     float* sp_val = nullptr;
     __nv_bfloat16* xb = nullptr;
@@ -204,9 +204,9 @@ int launch_logit_track(rfast_ctx* ctx, const RoundArgs& a, const EvDesc* d_ev, i
     GradArgs g = grad_args(ctx, d_ev);
     const dim3 grid(ctx->sp_tiles, nev);
     if (ctx->compensated)
-        k_logit_track<true><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_tiles, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
+        k_logit_track<true><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_ranges, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
     else
-        k_logit_track<false><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_tiles, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
+        k_logit_track<false><<<grid, kThreads, 0, ctx->stream>>>(a, g, ctx->sp_tile_ptr, ctx->sp_ranges, ctx->sp_col, ctx->sp_val, ctx->scratch, init_only);
     ctx->launches += 1;
     CK(cudaGetLastError());
     return RFAST_OK;
@@ -403,15 +403,16 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
                 }
                 if (prob->label[r] != 1 && prob->label[r] != -1) return set_err(ctx, RFAST_EINVAL, "labels must be -1 or +1");
             }
-            {   // per shard row, where each tile of kLogitTile coordinates starts (one walk over the entries)
+            {   // per shard row, where each range of kLogitRange coordinates starts (one walk over the entries)
                 ctx->sp_tiles = (int)((ctx->p + kLogitTile - 1) / kLogitTile);
-                std::vector<int64_t> tp((size_t)nrows * (ctx->sp_tiles + 1));
+                ctx->sp_ranges = (int)((ctx->p + kLogitRange - 1) / kLogitRange);
+                std::vector<int64_t> tp((size_t)nrows * (ctx->sp_ranges + 1));
                 for (size_t r = 0; r < nrows; ++r) {
                     int64_t q = prob->sp_rowptr[r];
                     const int64_t qe = prob->sp_rowptr[r + 1];
-                    int64_t* dst = tp.data() + r * (ctx->sp_tiles + 1);
-                    for (int t = 0; t <= ctx->sp_tiles; ++t) {
-                        const int64_t bound = (int64_t)t * kLogitTile;
+                    int64_t* dst = tp.data() + r * (ctx->sp_ranges + 1);
+                    for (int t = 0; t <= ctx->sp_ranges; ++t) {
+                        const int64_t bound = (int64_t)t * kLogitRange;
                         while (q < qe && prob->sp_col[q] < bound) ++q;
                         dst[t] = q;
                     }

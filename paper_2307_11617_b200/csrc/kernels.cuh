@@ -562,33 +562,31 @@ k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restri
 
 // Sparse logistic regression, phase 2, fused with S2b/S2c.  A CTA owns a tile of kLogitTile
 // coordinates of one activation: it forms g = l2 x + sum_k coef_k a_k for the tile in shared
-// memory (the sampled rows are added one after the other, so repeated columns add up in batch
-// order on every run; the entries of one row land on distinct coordinates), stores it as the
-// new remembered gradient and, unless init_only, runs the tracking update on the tile, 1024
-// coordinates at a time.
-// tile_ptr[r][t] = index of the first entry of shard row r with column >= t * kLogitTile
-// (computed once per problem on the host), so no search is needed here.
+// memory, stores it as the new remembered gradient and, unless init_only, runs the tracking
+// update on the tile, 1024 coordinates at a time.
+// Assembly: warp w owns the coordinates [512 w, 512 (w+1)) of the tile and fetches, for every
+// sampled row, exactly the entries that fall there: range_ptr[r][j] = index of the first entry of
+// shard row r with column >= 512 j (computed once per problem on the host), so nothing is
+// searched and the warps never wait for one another.  The entries are taken 32 at a time in
+// row-major order; entries of different rows that hit the same coordinate (rare) are found with
+// a warp match and added in row order, so the sum is the same on every run.
 // grid = (tiles, events), 256 threads
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 constexpr int kLogitSub = 4;                               // passes of kThreads float4 per tile
 constexpr int kLogitTile = kLogitSub * 4 * kThreads;
+constexpr int kLogitRange = kLogitTile / (kThreads / 32);  // coordinates a warp assembles
 template <bool COMP>
 __global__ void __launch_bounds__(kThreads)
-k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int ntiles,
+k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ range_ptr, int nranges,
               const int* __restrict__ sp_col, const float* __restrict__ sp_val,
               const float* __restrict__ coef, int init_only) {
-    constexpr int kStage = 2048;           // staged entries per pass (about 40 per row and tile are typical)
     __shared__ float tile[kLogitTile];
-    __shared__ int64_t lo_s[64];
-    __shared__ int cnt_s[64], pref_s[65];
-    __shared__ float ck_s[64];
-    __shared__ int st_col[kStage];
-    __shared__ float st_val[kStage];
     const EvDesc e = g.ev[blockIdx.y];
     const int64_t row = (int64_t)e.node * g.stride;
     const int64_t c0 = (int64_t)blockIdx.x * kLogitTile;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr unsigned kFull = 0xffffffffu;
     // The tracking part at the end is a chain of dependent loads per sub-pass (edge lists -> row
     // ids -> rows); its operands are requested into L2 now, while the tile is assembled: the
     // lists into shared memory (the later reads then hit L1), the rows by prefetch, one request
@@ -616,6 +614,19 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int
             }
         }
     }
+    // the warp's first batch of rows: batch index -> entry range, started before the x tile is stored
+    const int rg = blockIdx.x * (kThreads / 32) + warp;      // this warp's coordinate range inside a row
+    const bool mine = rg < nranges;
+    int64_t lo = 0;
+    int cnt = 0;
+    float ck = 0.f;
+    if (mine && lane < min(32, g.B)) {
+        const int rrow = g.batch_idx[(int64_t)e.sample * g.B + lane];
+        const int64_t r = (int64_t)e.node * g.rows + rrow;
+        lo = range_ptr[r * (nranges + 1) + rg];
+        cnt = (int)(range_ptr[r * (nranges + 1) + rg + 1] - lo);
+        ck = coef[(int64_t)blockIdx.y * g.B + lane];
+    }
 #pragma unroll
     for (int sub = 0; sub < kLogitSub; ++sub) {
         const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
@@ -623,60 +634,64 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ tile_ptr, int
         if (i4 < a.n4) xv = reinterpret_cast<const float4*>(g.x + row)[i4];
         reinterpret_cast<float4*>(tile)[sub * kThreads + threadIdx.x] = f4_scale(g.l2, xv);
     }
-    for (int k0 = 0; k0 < g.B; k0 += 64) {                       // up to 64 sampled rows per pass
-        const int nb = min(64, g.B - k0);
-        __syncthreads();
-        if (threadIdx.x < nb) {
-            const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k0 + threadIdx.x];
-            const int64_t r = (int64_t)e.node * g.rows + rrow;
-            const int64_t lo = tile_ptr[r * (ntiles + 1) + blockIdx.x];
-            lo_s[threadIdx.x] = lo;
-            cnt_s[threadIdx.x] = (int)(tile_ptr[r * (ntiles + 1) + blockIdx.x + 1] - lo);
-            ck_s[threadIdx.x] = coef[(int64_t)blockIdx.y * g.B + k0 + threadIdx.x];
-        }
-        __syncthreads();
-        if (threadIdx.x <= nb) {
-            int s = 0;
-            for (int u = 0; u < threadIdx.x; ++u) s += cnt_s[u];
-            pref_s[threadIdx.x] = s;
-        }
-        __syncthreads();
-        const int total = pref_s[nb];
-        if (k0 == 0 && !init_only && (lane & 7) == 0) {          // pre_row is visible since the barriers above
-            for (int m = 0; m < 3 * kPre; ++m) {
-                const int id = pre_row[m];
-                if (id < 0) continue;
-                const float* rr = a.rbuf + (int64_t)id * a.stride;
+    __syncthreads();                                        // tile = l2 x; pre_row is visible
+    if (!init_only && (lane & 7) == 0) {
+        for (int m = 0; m < 3 * kPre; ++m) {
+            const int id = pre_row[m];
+            if (id < 0) continue;
+            const float* rr = a.rbuf + (int64_t)id * a.stride;
 #pragma unroll
-                for (int sub = 0; sub < kLogitSub; ++sub) {
-                    const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
-                    if (i4 < a.n4) prefetch_l2(rr + (int64_t)i4 * 4);
+            for (int sub = 0; sub < kLogitSub; ++sub) {
+                const int i4 = (blockIdx.x * kLogitSub + sub) * kThreads + threadIdx.x;
+                if (i4 < a.n4) prefetch_l2(rr + (int64_t)i4 * 4);
+            }
+        }
+    }
+    if (mine) {
+        for (int k0 = 0; k0 < g.B; k0 += 32) {              // up to 32 sampled rows per pass, one per lane
+            const int nb = min(32, g.B - k0);
+            if (k0 > 0) {
+                lo = 0; cnt = 0; ck = 0.f;
+                if (lane < nb) {
+                    const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k0 + lane];
+                    const int64_t r = (int64_t)e.node * g.rows + rrow;
+                    lo = range_ptr[r * (nranges + 1) + rg];
+                    cnt = (int)(range_ptr[r * (nranges + 1) + rg + 1] - lo);
+                    ck = coef[(int64_t)blockIdx.y * g.B + k0 + lane];
                 }
             }
-        }
-        if (total <= kStage) {
-            // all entries of this tile are fetched at once (one memory latency), then one warp
-            // adds them row after row so that the order of additions is the same on every run
-            for (int t = threadIdx.x; t < total; t += kThreads) {
-                int k = 0;
-                while (pref_s[k + 1] <= t) ++k;
-                const int64_t q = lo_s[k] + (t - pref_s[k]);
-                st_col[t] = sp_col[q] - (int)c0;
-                st_val[t] = ck_s[k] * sp_val[q];
+            int incl = cnt;                                 // entries of rows 0 .. lane (this pass, this range)
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += v;
             }
-            __syncthreads();
-            if (warp == 0)
-                for (int k = 0; k < nb; ++k) {
-                    for (int t = pref_s[k] + lane; t < pref_s[k + 1]; t += 32) tile[st_col[t]] += st_val[t];
+            const int total = __shfl_sync(kFull, incl, 31);
+            for (int t0 = 0; t0 < total; t0 += 32) {        // entry t of the row-major list
+                const int t = t0 + lane;
+                const bool act = t < total;
+                int k = 0;
+                for (int j = 0; j < nb; ++j) k += (__shfl_sync(kFull, incl, j) <= t) ? 1 : 0;
+                k = min(k, nb - 1);
+                const int64_t lo_k = __shfl_sync(kFull, lo, k);
+                const int excl_k = __shfl_sync(kFull, incl - cnt, k);
+                const float ck_k = __shfl_sync(kFull, ck, k);
+                int col = -1 - lane;                        // inactive lanes: distinct dummies
+                float val = 0.f;
+                if (act) {
+                    const int64_t q = lo_k + (t - excl_k);
+                    col = sp_col[q] - (int)c0;
+                    val = ck_k * sp_val[q];
+                }
+                const unsigned same = __match_any_sync(kFull, col);
+                const int rank = __popc(same & ((1u << lane) - 1u));   // earlier rows on the same coordinate
+                int maxr = rank;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) maxr = max(maxr, __shfl_xor_sync(kFull, maxr, o));
+                for (int rr = 0; rr <= maxr; ++rr) {        // almost always one turn
+                    if (act && rank == rr) tile[col] += val;
                     __syncwarp();
                 }
-        } else {
-            for (int k = 0; k < nb; ++k) {
-                for (int64_t q = lo_s[k] + threadIdx.x; q < lo_s[k] + cnt_s[k]; q += kThreads) {
-                    const int c = sp_col[q] - (int)c0;
-                    tile[c] += ck_s[k] * sp_val[q];
-                }
-                __syncthreads();
             }
         }
     }
