@@ -564,6 +564,7 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
     a.out_cur = ctx->d_out_cur; a.out_new = ctx->d_out_new; a.out_a = ctx->d_out_a;
     a.x = ctx->x; a.z = ctx->z; a.zc = ctx->zc; a.vbuf = ctx->vbuf; a.rbuf = ctx->rbuf; a.rlo_off = ctx->rlo_off();
     a.stride = ctx->stride; a.n4 = (int)(ctx->stride / 4); a.alpha = ctx->alpha;
+    const bool pf = (size_t)ctx->n * ctx->stride * sizeof(float) > ((size_t)64 << 20);   // one state array against half of L2
     for (int r = r0; r < r1; ++r) {
         const int nev = c.act_ptr[r + 1] - c.act_ptr[r];
         if (nev == 0) continue;
@@ -575,18 +576,27 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
             ctx->launches += 1;
         } else {
             const int64_t gplane = (int64_t)ctx->n * ctx->stride;
-            if (ctx->model == RFAST_MODEL_MLP)
-                k_mix<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->xb);
-            else
-                k_mix<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, nullptr);
+            const dim3 tg = tile_grid(a.n4, 1, nev);
+            if (ctx->model == RFAST_MODEL_MLP) {
+                if (pf) k_mix<1, true, true><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->xb);
+                else k_mix<1, true, false><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->xb);
+            } else {
+                if (pf) k_mix<1, false, true><<<tg, kThreads, 0, ctx->stream>>>(a, nullptr);
+                else k_mix<1, false, false><<<tg, kThreads, 0, ctx->stream>>>(a, nullptr);
+            }
             ctx->launches += 1;
             int rc = launch_gradients(ctx, a.ev, nev);
             if (rc != RFAST_OK) return rc;
             if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {
                 if ((rc = launch_logit_track(ctx, a, a.ev, nev, 0)) != RFAST_OK) return rc;
             } else {
-                if (ctx->compensated) k_track<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
-                else k_track<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                if (ctx->compensated) {
+                    if (pf) k_track<1, true, true><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                    else k_track<1, true, false><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                } else {
+                    if (pf) k_track<1, false, true><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                    else k_track<1, false, false><<<tg, kThreads, 0, ctx->stream>>>(a, ctx->gbuf, gplane);
+                }
                 ctx->launches += 1;
             }
         }

@@ -31,6 +31,9 @@ struct RoundArgs {
     float   alpha;
 };
 
+// one request brings the 128-byte line into L2; issued by one lane in eight (8 x 16 bytes)
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ float4 ld_stream(const float* row, int i4) {
     return __ldcs(reinterpret_cast<const float4*>(row) + i4);
 }
@@ -371,17 +374,23 @@ __device__ __forceinline__ void mix_tile(const RoundArgs& a, const EvDesc& e, in
     }
 }
 
-template <int U, bool BF16>
+// PF: the state does not fit L2; the rows read behind an edge-list entry are requested into L2 first
+template <int U, bool BF16, bool PF = false>
 __global__ void __launch_bounds__(kThreads)
 k_mix(RoundArgs a, __nv_bfloat16* __restrict__ xb) {
-    mix_tile<U, BF16, false>(a, a.ev[blockIdx.y], blockIdx.x, xb);
+    const EvDesc e = a.ev[blockIdx.y];
+    const int base = blockIdx.x * (kThreads * U) + threadIdx.x;
+    if (PF && U == 1 && (threadIdx.x & 7) == 0 && base < a.n4)
+        for (int m = 0; m < e.mix_cnt; ++m)
+            prefetch_l2(a.vbuf + (int64_t)a.mix_slot[e.mix_beg + m] * a.stride + (int64_t)base * 4);
+    mix_tile<U, BF16, false>(a, e, blockIdx.x, xb);
 }
 
 // ---------------------------------------------------------------------------------------------
 // S2b + S2c (+ S4 by row id) with the gradients taken from the two gradient buffers:
 // g_old = gbuf[par][node], g_new = gbuf[par^1][node].  grid = (tiles, events)
 // ---------------------------------------------------------------------------------------------
-template <int U, bool COMP>
+template <int U, bool COMP, bool PF = false>
 __global__ void __launch_bounds__(kThreads)
 k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
     const EvDesc e = a.ev[blockIdx.y];
@@ -396,6 +405,19 @@ k_track(RoundArgs a, const float* __restrict__ gbuf, int64_t gplane) {
         const int i4 = base + u * kThreads;
         zh[u] = gnv[u] = gov[u] = make_float4(0, 0, 0, 0);
         if (i4 < a.n4) { zh[u] = ld_stream(zr, i4); gnv[u] = ld_stream(gn, i4); gov[u] = ld_stream(go, i4); }
+    }
+    // the news and running-sum rows are read behind the list entries that name them
+    if (PF && U == 1 && (threadIdx.x & 7) == 0 && base < a.n4) {
+        const int64_t off = (int64_t)base * 4;
+        for (int m = 0; m < e.news_cnt; ++m) {
+            prefetch_l2(a.rbuf + (int64_t)a.news_new[e.news_beg + m] * a.stride + off);
+            const int prev = a.news_prev[e.news_beg + m];
+            if (prev >= 0) prefetch_l2(a.rbuf + (int64_t)prev * a.stride + off);
+        }
+        for (int m = 0; m < e.out_cnt; ++m) {
+            const int cur = a.out_cur[e.out_beg + m];
+            if (cur >= 0) prefetch_l2(a.rbuf + (int64_t)cur * a.stride + off);
+        }
     }
     track_and_push<U, COMP>(a, e, base, zr, zh, gnv, gov);
 }
@@ -571,7 +593,6 @@ k_logit_coef(GradArgs g, const int64_t* __restrict__ sp_ptr, const int* __restri
 // row-major order; entries of different rows that hit the same coordinate (rare) are found with
 // a warp match and added in row order, so the sum is the same on every run.
 // grid = (tiles, events), 256 threads
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 constexpr int kLogitSub = 4;                               // passes of kThreads float4 per tile
 constexpr int kLogitTile = kLogitSub * 4 * kThreads;
