@@ -421,7 +421,7 @@ k_mlp_back(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, co
         float s = 0.f;
         for (int k = half * (kBatch / 2); k < (half + 1) * (kBatch / 2); ++k) s += dlf[k * 16 + c];
         const float o = __shfl_down_sync(0xffffffffu, s, 16);
-        if (threadIdx.x < C) g[ob2 + c] = (s + o) + l2 * x[row + ob2 + c];
+        if (threadIdx.x < C) g[ob2 + c] = l2 != 0.f ? (s + o) + l2 * x[row + ob2 + c] : (s + o);   // no load without a regulariser
     }
     float gb1 = 0.f;
     __nv_bfloat16* drow = dpqT + ((int64_t)ev * H + j) * kBatch + kq * kQuarter;
@@ -459,7 +459,7 @@ k_mlp_back(const EvDesc* __restrict__ evs, const int* __restrict__ batch_idx, co
         const int pc = c < C ? c : CP;
         const float tot = ((part[0][jj][pc] + part[1][jj][pc]) + part[2][jj][pc]) + part[3][jj][pc];
         const int64_t at = c < C ? oW2 + (int64_t)c * H + blockIdx.x * kSlab + jj : (int64_t)H * F + blockIdx.x * kSlab + jj;
-        g[at] = tot + l2 * x[row + at];
+        g[at] = l2 != 0.f ? tot + l2 * x[row + at] : tot;
     }
 }
 
