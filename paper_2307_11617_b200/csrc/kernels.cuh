@@ -517,17 +517,19 @@ k_softmax_logits(GradArgs g, const float* __restrict__ feat, float* __restrict__
 template <bool CG>
 __device__ __forceinline__ void softmax_delta_block(const GradArgs& g, const EvDesc& e, int ev_local,
                                                     const int* label, const float* logit, float* delta, int* rowid) {
-    for (int k = threadIdx.x; k < g.B; k += 256) {
+    // one thread per (row, class): every thread forms the row's maximum and denominator itself
+    // (same order of operations for all classes of a row), so nothing waits for a reduction
+    for (int t = threadIdx.x; t < g.B * g.C; t += 256) {
+        const int k = t / g.C, c = t - k * g.C;
         const int rrow = g.batch_idx[(int64_t)e.sample * g.B + k];
-        rowid[k] = rrow;
+        if (c == 0) rowid[k] = rrow;
+        const int lab = label[(int64_t)e.node * g.rows + rrow];
         const float* lg = logit + ((int64_t)ev_local * g.B + k) * g.C;
         float m = ld_sel1<CG>(lg);
-        for (int c = 1; c < g.C; ++c) m = fmaxf(m, ld_sel1<CG>(lg + c));
+        for (int cc = 1; cc < g.C; ++cc) m = fmaxf(m, ld_sel1<CG>(lg + cc));
         float den = 0.f;
-        for (int c = 0; c < g.C; ++c) den += expf(ld_sel1<CG>(lg + c) - m);
-        const int lab = label[(int64_t)e.node * g.rows + rrow];
-        for (int c = 0; c < g.C; ++c)
-            delta[k * g.C + c] = (expf(ld_sel1<CG>(lg + c) - m) / den - (c == lab ? 1.f : 0.f)) / (float)g.B;
+        for (int cc = 0; cc < g.C; ++cc) den += expf(ld_sel1<CG>(lg + cc) - m);
+        delta[t] = (expf(ld_sel1<CG>(lg + c) - m) / den - (c == lab ? 1.f : 0.f)) / (float)g.B;
     }
     __syncthreads();
 }
@@ -539,8 +541,15 @@ __device__ __forceinline__ float softmax_grad_coord(const GradArgs& g, const EvD
     if (q < (int64_t)g.C * g.F) {
         const int c = (int)(q / g.F), f = (int)(q % g.F);
         const float* abase = feat + (int64_t)e.node * g.rows * g.F;
-#pragma unroll 8
-        for (int k = 0; k < g.B; ++k) s = fmaf(delta[k * g.C + c], abase[(int64_t)rowid[k] * g.F + f], s);
+        int k = 0;
+        for (; k + 16 <= g.B; k += 16) {                   // sixteen feature loads in flight, summed in order
+            float av[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) av[u] = abase[(int64_t)rowid[k + u] * g.F + f];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) s = fmaf(delta[(k + u) * g.C + c], av[u], s);
+        }
+        for (; k < g.B; ++k) s = fmaf(delta[k * g.C + c], abase[(int64_t)rowid[k] * g.F + f], s);
     } else {
         const int c = (int)(q - (int64_t)g.C * g.F);
         for (int k = 0; k < g.B; ++k) s += delta[k * g.C + c];
