@@ -328,23 +328,48 @@ k_mlp_fwd(const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();                                       // h and the W2 columns are in shared memory
     if (warp >= 2 && bad == 0) {                           // ---- the slab's share of the logits
-        const int k = wt >> 2, cgp = wt & 3;                // sampled row; classes cgp, cgp + 4, ...
-        float acc[CQ];
+        // Register tile of 4 rows x CQ classes per thread over a quarter of the hidden units: every
+        // value read from shared memory feeds 4 (W2) or CQ (h) products, a third of the reads of
+        // one row per thread.  Lane bits: jq = quarter of the units (interleaved: float4 4t + jq),
+        // kg = rows kg, kg + 16, kg + 32, kg + 48; cgp = classes cgp, cgp + 4, ...  The four
+        // quarters sit in adjacent lanes and are added in a fixed tree.
+        const int jq = wt & 3, kg = (wt >> 2) & 15, cgp = wt >> 6;
+        float acc[4][CQ];
 #pragma unroll
-        for (int i = 0; i < CQ; ++i) acc[i] = 0.f;
-        const float4* h4 = reinterpret_cast<const float4*>(hs + k * kHsPitch);
-#pragma unroll 8
-        for (int j4 = 0; j4 < kMTile / 4; ++j4) {
-            const float4 hv = h4[j4];
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int i = 0; i < CQ; ++i) acc[r][i] = 0.f;
+#pragma unroll 2
+        for (int t = 0; t < kMTile / 16; ++t) {
+            const int j4 = 4 * t + jq;
+            float4 hv[4], wv[CQ];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) hv[r] = reinterpret_cast<const float4*>(hs + (kg + 16 * r) * kHsPitch)[j4];
+#pragma unroll
+            for (int i = 0; i < CQ; ++i) wv[i] = reinterpret_cast<const float4*>(w2s + (cgp + 4 * i) * kHsPitch)[j4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int i = 0; i < CQ; ++i)
+                    acc[r][i] = fmaf(hv[r].w, wv[i].w, fmaf(hv[r].z, wv[i].z, fmaf(hv[r].y, wv[i].y, fmaf(hv[r].x, wv[i].x, acc[r][i]))));
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
 #pragma unroll
             for (int i = 0; i < CQ; ++i) {
-                const float4 w = reinterpret_cast<const float4*>(w2s + (cgp + 4 * i) * kHsPitch)[j4];
-                acc[i] = fmaf(hv.w, w.w, fmaf(hv.z, w.z, fmaf(hv.y, w.y, fmaf(hv.x, w.x, acc[i]))));
+                float v = acc[r][i];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                acc[r][i] = v;
+            }
+        if (jq == 0) {
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                float* dst = share + (((int64_t)ev * gridDim.x + blockIdx.x) * kBatch + kg + 16 * r) * 16;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) dst[cgp + 4 * i] = i < CQ ? acc[r][i < CQ ? i : 0] : 0.f;
             }
         }
-        float* dst = share + (((int64_t)ev * gridDim.x + blockIdx.x) * kBatch + k) * 16;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) dst[cgp + 4 * i] = i < CQ ? acc[i < CQ ? i : 0] : 0.f;
     }
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tacc, 64); }
 }
