@@ -282,29 +282,27 @@ def main():
         h2d = sum(a.nbytes for a in (s.act_ptr, s.act_node, s.send_r, s.send_c, s.batch_idx)) + \
             64 * events
         reps = max(1, min(args.steps, 3))
-        barrier()
-        t0 = time.perf_counter()
-        for _ in range(reps):
-            eng.load_schedule(s)
-            eng.run(sync=False)
-            eng.read(B.STATE_X, xo)
-            eng.read(B.STATE_Y, yo)
-        barrier()
-        dt = (time.perf_counter() - t0) / reps
-        dt = max_over_ranks(dt, "cuda")
+        def timed_reps(result):
+            """Median over the repetitions of one whole pass (host timer; every pass ends with a
+            synchronous read, so nothing is in flight between two of them)."""
+            times = []
+            for _ in range(reps):
+                barrier()
+                t0 = time.perf_counter()
+                eng.load_schedule(s)
+                eng.run(sync=False)
+                result()
+                torch.cuda.synchronize()
+                times.append(time.perf_counter() - t0)
+            return max_over_ranks(sorted(times)[len(times) // 2], "cuda")
+
+        dt = timed_reps(lambda: (eng.read(B.STATE_X, xo), eng.read(B.STATE_Y, yo)))
         e2e = {"value": whole_job_rate(events, 1 if sharded else world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3,
                "result": "x and y of every node into pinned host memory"}
         # the same with the run's metrics as the result instead of the whole state (consensus
         # error, Lemma 3 residual, tracker norm: computed on the device, a few numbers come back)
-        barrier()
-        t0 = time.perf_counter()
-        for _ in range(reps):
-            eng.load_schedule(s)
-            eng.run(sync=False)
-            eng.diagnostics()
-        barrier()
-        dm = max_over_ranks((time.perf_counter() - t0) / reps, "cuda")
+        dm = timed_reps(eng.diagnostics)
         e2e["metrics_only"] = {"value": whole_job_rate(events, 1 if sharded else world, dm), "ms_per_step": dm * 1e3,
                                "d2h_bytes_per_step": int(5 * 8 * ((wl.p + 255) // 256))}
 
