@@ -187,6 +187,153 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def measure_config(name, args, steps, world, rank, local, cpu_budget_s):
+    """One workload on this rank's GPU: timed passes (CUDA events on the engine's stream), the
+    end-to-end passes through the C ABI with host buffers, the clocks seen meanwhile, the
+    roofline figures and, on rank 0, the oracle on a bounded sample.  Returns the pieces of a
+    JSON record."""
+    import torch
+    import torch.distributed as dist
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+
+    t_gen = time.perf_counter()
+    wl_full = build_workload(name, args.small, args.tracker)
+    wl = wl_full
+    sharded = args.shard == "coords" and world > 1 and wl.model == "quad_diag"
+    if sharded:
+        from workloads import shard_coordinates
+        wl = shard_coordinates(wl_full, rank, world)     # same schedule, this rank's slice of every vector
+    t_gen = time.perf_counter() - t_gen
+    stream = torch.cuda.Stream()
+    t_create = time.perf_counter()
+    eng = pkg.Engine(wl, stream.cuda_stream)
+    t_create = time.perf_counter() - t_create
+    t_load = time.perf_counter()
+    eng.load_schedule(wl.schedule)
+    t_load = time.perf_counter() - t_load
+    events = eng.query(B.Q_EVENTS_TOTAL)
+    # a coordinate shard moves 1/world of the job's bytes: the job's count is the sum over ranks
+    job = world if sharded else 1
+    bytes_impl = eng.query(B.Q_BYTES_TOTAL) * job
+    bytes_method = eng.query(B.Q_METHOD_BYTES_TOTAL) * job
+    K_rounds = wl.schedule.K
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step():
+        eng.reset()                                   # back to round 0; not part of the timed work
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        eng.run(sync=False)
+        e1.record(stream)
+        return (e0, e1)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        one_step()
+    barrier()
+    l0 = eng.query(B.Q_LAUNCHES)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    w0 = time.time()
+    pairs = [one_step() for _ in range(steps)]
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1)
+    launches = eng.query(B.Q_LAUNCHES) - l0
+    ms = sorted(a.elapsed_time(b) for a, b in pairs)
+    ms_step = max_over_ranks(float(ms[len(ms) // 2]), "cuda")     # median of the timed passes, slowest rank
+    # coordinate shards: every rank runs every activation on its slice, the job's rate is one rank's
+    value = whole_job_rate(events, 1 if sharded else world, ms_step * 1e-3)
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = measure_e2e(eng, wl, events, steps, barrier, 1 if sharded else world)
+
+    peak, peak_kind = measured_peaks()
+    achieved = bytes_method / (ms_step * 1e-3) / 1e9
+    achieved_impl = bytes_impl / (ms_step * 1e-3) / 1e9
+    hbm_bound = wl.model in ("quad_diag", "logistic_sparse", "mlp")
+    per_launch = max(1, launches // max(1, steps))
+    fused = wl.model == "quad_diag"
+    roofline = {"bound": "hbm",
+                "kernel": "k_fused_quad" if fused else "one round: k_mix + gradient kernels + tracking pass",
+                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
+                "bytes": "what the method must move: x, z read once, the gradient moved once, packets and running sums as compiled",
+                "algorithmic_bytes_per_launch": bytes_method / (per_launch if fused else K_rounds),
+                "implementation_bytes": {"per_step": bytes_impl, "achieved": achieved_impl, "frac": achieved_impl / peak,
+                                         "what": "every stream the kernels touch (re-reads between the kernels of a split step, low-order tracker words)"},
+                "traffic": (fused_traffic_ratio() and fused_traffic_ratio() * bytes_impl / per_launch)
+                if fused and args.tracker == "sums" and not sharded else None,   # the counters were taken on that workload
+                "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        v, desc, dt = oracle_sample(wl_full, budget_s=cpu_budget_s)   # the unsharded workload
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+
+    rec = {"value": value, "ms_per_step": ms_step, "steps": steps, "warmup": warm,
+           "config": {"workload": wl.name, "n": wl.n, "p": wl_full.p, "rounds": K_rounds,
+                      "activations_per_step": events, "small": bool(args.small), "tracker": args.tracker,
+                      "tracker_arithmetic": {0: "plain fp32", 1: "two-float tracker", 2: "two-float tracker and running sums"}[int(wl.compensated)],
+                      "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
+                      "reset_between_steps": "untimed",
+                      "parallelism": f"coordinate shards x{world}" if sharded else f"replicas x{world}"},
+           "scaling": "strong" if sharded else "weak",
+           "param_updates_per_s": value * wl_full.p, "gpu_launches": int(launches),
+           "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+           "setup_s": {"generate": t_gen, "create": t_create, "load_schedule": t_load},
+           "device_bytes": eng.query(B.Q_DEVICE_BYTES),
+           "version_rows": {"v": eng.query(B.Q_V_SLOTS), "rho": eng.query(B.Q_RHO_SLOTS)}}
+    eng.close()
+    del eng, wl, wl_full
+    torch.cuda.empty_cache()
+    return rec
+
+
+def measure_e2e(eng, wl, events, steps, barrier, rate_world):
+    """End to end through the C ABI with host buffers: the schedule arrays go in (compiled and
+    uploaded), the run, x and y of every node come back into pinned host memory.  Median over the
+    repetitions of one whole pass (host timer; every pass ends with a synchronous read, so
+    nothing is in flight between two of them)."""
+    import torch
+    from paper_2307_11617_b200 import binding as B
+    xo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
+    yo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
+    s = wl.schedule
+    h2d = sum(a.nbytes for a in (s.act_ptr, s.act_node, s.send_r, s.send_c, s.batch_idx)) + 64 * events
+    reps = max(1, min(steps, 3))
+
+    def timed_reps(result):
+        times = []
+        for _ in range(reps):
+            barrier()
+            t0 = time.perf_counter()
+            eng.load_schedule(s)
+            eng.run(sync=False)
+            result()
+            torch.cuda.synchronize()
+            times.append(time.perf_counter() - t0)
+        return max_over_ranks(sorted(times)[len(times) // 2], "cuda")
+
+    dt = timed_reps(lambda: (eng.read(B.STATE_X, xo), eng.read(B.STATE_Y, yo)))
+    e2e = {"value": whole_job_rate(events, rate_world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3,
+           "result": "x and y of every node into pinned host memory"}
+    # the same with the run's metrics as the result instead of the whole state (consensus
+    # error, Lemma 3 residual, tracker norm: computed on the device, a few numbers come back)
+    dm = timed_reps(eng.diagnostics)
+    e2e["metrics_only"] = {"value": whole_job_rate(events, rate_world, dm), "ms_per_step": dm * 1e3,
+                           "d2h_bytes_per_step": int(6 * 8 * ((wl.p + 255) // 256))}
+    return e2e
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -200,15 +347,24 @@ def main():
     ap.add_argument("--shard", default="replicas", choices=["replicas", "coords"],
                     help="with N GPUs: N independent replicas (default), or the coordinates of the "
                          "element-wise problem split over the GPUs (no exchange; strong scaling)")
+    ap.add_argument("--others", default="auto", choices=["auto", "all", "none"],
+                    help="also measure the other four configurations (3 timed passes each) into "
+                         "'other_configs'; auto: when --config is the default and --small is off")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world:
+        # one process per GPU: N ranks are started by torch.distributed.run, never silently as one
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} but WORLD_SIZE is {world}; launch the ranks with\n"
+                         f"  python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} "
+                         f"--master-addr 127.0.0.1 --master-port <port> bench.py --gpus {args.gpus} ...\n")
+        raise SystemExit(2)
     if args.impl == "reference":
         return run_reference(args)
 
     import torch
     import torch.distributed as dist
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
@@ -218,125 +374,28 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    import paper_2307_11617_b200 as pkg
-    from paper_2307_11617_b200 import binding as B
-
-    t_gen = time.perf_counter()
-    wl = build_workload(args.config, args.small, getattr(args, "tracker", "sums"))
-    full_p = wl.p
-    sharded = args.shard == "coords" and world > 1
-    if sharded:
-        from workloads import shard_coordinates
-        wl = shard_coordinates(wl, rank, world)      # same schedule, this rank's slice of every vector
-    t_gen = time.perf_counter() - t_gen
-    stream = torch.cuda.Stream()
-    t_create = time.perf_counter()
-    eng = pkg.Engine(wl, stream.cuda_stream)
-    t_create = time.perf_counter() - t_create
-    t_load = time.perf_counter()
-    eng.load_schedule(wl.schedule)
-    t_load = time.perf_counter() - t_load
-    events = eng.query(B.Q_EVENTS_TOTAL)
-    bytes_step = eng.query(B.Q_BYTES_TOTAL)
-    K_rounds = wl.schedule.K
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def one_step(timed):
-        eng.reset()                                   # back to round 0; not part of the timed work
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        eng.run(sync=False)
-        e1.record(stream)
-        return (e0, e1)
-
-    for _ in range(max(args.warmup, 3)):
-        one_step(False)
-    barrier()
-    l0 = eng.query(B.Q_LAUNCHES)
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.25)
-    w0 = time.time()
-    pairs = [one_step(True) for _ in range(args.steps)]
-    barrier()
-    w1 = time.time()
-    clocks = sampler.stop(w0, w1)
-    launches = eng.query(B.Q_LAUNCHES) - l0
-    ms = [a.elapsed_time(b) for a, b in pairs]
-    ms_step = float(sum(ms) / len(ms))
-    ms_step = max_over_ranks(ms_step, "cuda")
-    # coordinate shards: every rank runs every activation on its slice, the job's rate is one rank's
-    value = whole_job_rate(events, 1 if sharded else world, ms_step * 1e-3)
-
-    # end to end through the C ABI with host buffers: schedule arrays in (compiled and uploaded),
-    # the run, x and y back into pinned host memory
-    e2e = None
-    if not args.no_e2e:
-        xo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
-        yo = torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy()
-        s = wl.schedule
-        h2d = sum(a.nbytes for a in (s.act_ptr, s.act_node, s.send_r, s.send_c, s.batch_idx)) + \
-            64 * events
-        reps = max(1, min(args.steps, 3))
-        def timed_reps(result):
-            """Median over the repetitions of one whole pass (host timer; every pass ends with a
-            synchronous read, so nothing is in flight between two of them)."""
-            times = []
-            for _ in range(reps):
-                barrier()
-                t0 = time.perf_counter()
-                eng.load_schedule(s)
-                eng.run(sync=False)
-                result()
-                torch.cuda.synchronize()
-                times.append(time.perf_counter() - t0)
-            return max_over_ranks(sorted(times)[len(times) // 2], "cuda")
-
-        dt = timed_reps(lambda: (eng.read(B.STATE_X, xo), eng.read(B.STATE_Y, yo)))
-        e2e = {"value": whole_job_rate(events, 1 if sharded else world, dt), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(xo.nbytes + yo.nbytes), "ms_per_step": dt * 1e3,
-               "result": "x and y of every node into pinned host memory"}
-        # the same with the run's metrics as the result instead of the whole state (consensus
-        # error, Lemma 3 residual, tracker norm: computed on the device, a few numbers come back)
-        dm = timed_reps(eng.diagnostics)
-        e2e["metrics_only"] = {"value": whole_job_rate(events, 1 if sharded else world, dm), "ms_per_step": dm * 1e3,
-                               "d2h_bytes_per_step": int(5 * 8 * ((wl.p + 255) // 256))}
-
-    peak, peak_kind = measured_peaks()
-    achieved = bytes_step / (ms_step * 1e-3) / 1e9
-    hbm_bound = wl.model in ("quad_diag", "logistic_sparse", "mlp")
-    roofline = {"bound": "hbm", "kernel": "k_fused_quad" if wl.model == "quad_diag" else "k_mix+gradient+k_track",
-                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
-                "algorithmic_bytes_per_launch": bytes_step / max(1, launches // max(1, args.steps)),
-                "traffic": (fused_traffic_ratio() and fused_traffic_ratio() * bytes_step / max(1, launches // max(1, args.steps)))
-                if wl.model == "quad_diag" and args.tracker == "sums" else None,   # the counters were taken on that workload
-                "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
-
-    cpu = None
-    if rank == 0 and not args.no_cpu_baseline:
-        v, desc, dt = oracle_sample(wl)
-        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
+    main_rec = measure_config(args.config, args, args.steps, world, rank, local, cpu_budget_s=15.0)
+    others = {}
+    want_others = args.others == "all" or (args.others == "auto" and args.config == "quad_tree64" and not args.small
+                                           and args.shard == "replicas")
+    if want_others:
+        from workloads import CONFIG_NAMES
+        for nm in CONFIG_NAMES:
+            if nm != args.config:
+                r = measure_config(nm, args, 3, world, rank, local, cpu_budget_s=4.0)
+                r["metric"], r["unit"] = METRIC, UNIT
+                others[nm] = r
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-                "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": wl.name, "n": wl.n, "p": full_p, "rounds": K_rounds,
-                           "activations_per_step": events, "small": bool(args.small), "tracker": args.tracker,
-                           "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
-                           "reset_between_steps": "untimed", "parallelism": f"coordinate shards x{world}" if sharded else f"replicas x{world}"},
-                "param_updates_per_s": value * full_p, "gpu_launches": int(launches),
-                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-                "setup_s": {"generate": t_gen, "create": t_create, "load_schedule": t_load},
-                "device_bytes": eng.query(B.Q_DEVICE_BYTES),
-                "version_rows": {"v": eng.query(B.Q_V_SLOTS), "rho": eng.query(B.Q_RHO_SLOTS)}}
+        line = {"metric": METRIC, "value": main_rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": main_rec["warmup"], "ms_per_step": main_rec["ms_per_step"], "higher_is_better": True,
+                "scaling": main_rec["scaling"], "vs_baseline": None, "dtype": "f32", "data": "synthetic"}
+        for k in ("config", "param_updates_per_s", "gpu_launches", "roofline", "cpu_baseline", "e2e", "clocks",
+                  "setup_s", "device_bytes", "version_rows"):
+            line[k] = main_rec[k]
+        if others:
+            line["other_configs"] = others
         print(json.dumps(line), flush=True)
-    eng.close()
     if world > 1:
         dist.destroy_process_group()
 

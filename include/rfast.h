@@ -158,7 +158,20 @@ enum {
     RFAST_STATE_USED_TAU_RHO = 7,  /* int32 per (event, in-edge of G_C): stamp consumed at S2b      */
     RFAST_STATE_TAU_V_END    = 8,  /* int32 [|E_R|]    tau_v at the end of the loaded schedule      */
     RFAST_STATE_TAU_RHO_END  = 9,  /* int32 [|E_C|]    tau_rho at the end of the loaded schedule    */
-    RFAST_STATE_ROUND        = 10  /* int32 [1]        rounds run so far                            */
+    RFAST_STATE_ROUND        = 10, /* int32 [1]        rounds run so far                            */
+    RFAST_STATE_V_LATEST     = 11, /* float [n][p]     v_i of node i's last activation (the payload of  */
+                                   /*       its packet with stamp t_i, Algorithm 1 S1/S3) where the     */
+                                   /*       engine holds it; a zero row where it does not: t_i = 0,     */
+                                   /*       every copy was lost, or no receiver will mix it in again    */
+    RFAST_STATE_V_HELD       = 12, /* int32 [n]        the stamp t_i where V_LATEST holds node i's row, */
+                                   /*       0 where the row is zero                                     */
+    RFAST_STATE_TAU_V        = 13, /* int32 [|E_R|]    tau_v per G_R edge after the rounds run so far   */
+                                   /*       (the stamp the receiver mixed in at its last activation)    */
+    RFAST_STATE_TAU_RHO      = 14, /* int32 [|E_C|]    tau_rho per G_C edge after the rounds run so far */
+    /* other names for the same views */
+    RFAST_STATE_ACT_COUNTS           = RFAST_STATE_T_LOCAL,      /* activations per node = t_i          */
+    RFAST_STATE_COMPILED_STAMPS_V    = RFAST_STATE_USED_TAU_V,
+    RFAST_STATE_COMPILED_STAMPS_RHO  = RFAST_STATE_USED_TAU_RHO
 };
 
 /* Counters for rfast_query. */
@@ -175,7 +188,17 @@ enum {
     RFAST_Q_DEVICE_BYTES   = 7,  /* device memory held by the handle */
     RFAST_Q_N_USED_TAU_V   = 8,  /* element count of RFAST_STATE_USED_TAU_V   */
     RFAST_Q_N_USED_TAU_RHO = 9,  /* element count of RFAST_STATE_USED_TAU_RHO */
-    RFAST_Q_BYTES_TOTAL    = 10  /* algorithmic bytes of the whole loaded schedule */
+    RFAST_Q_BYTES_TOTAL    = 10, /* the same count for the whole loaded schedule */
+    RFAST_Q_METHOD_BYTES_RUN   = 11, /* bytes the method itself must move (rounds run since the last  */
+                                     /* reset): per activation x and z read once, v written if a packet */
+                                     /* leaves, the neighbours' v read, x written, the remembered        */
+                                     /* gradient read and the new one written (element-wise objective:   */
+                                     /* its two data streams instead), the news rows read, z written, the */
+                                     /* running sums read and written.  RFAST_Q_BYTES_* also count what   */
+                                     /* only the implementation moves: re-reads between the kernels a     */
+                                     /* step is split into, the low-order tracker words of compensated    */
+                                     /* arithmetic                                                        */
+    RFAST_Q_METHOD_BYTES_TOTAL = 12  /* the same count for the whole loaded schedule */
 };
 
 /* Problem statement -> device (eq. (1), Assumptions 1-2).  Validates Assumption 1
@@ -187,7 +210,9 @@ enum {
 int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out);
 
 /* Compiles a schedule (Algorithm 2, S.0) for the handle and resets the state to the
- * initial one (round 0).  Host side, integers only: for every event and in-edge the stamp
+ * initial one (round 0).  A second call replaces the schedule and starts over at round 0 as
+ * well: rounds are not appended (to continue a run, load the longer schedule and move the
+ * state across with rfast_checkpoint_* or rfast_seek + rfast_write_state).  Host side, integers only: for every event and in-edge the stamp
  * that is consumed (tau_v, tau_rho of Algorithm 1, i.e. the delays d_v, d_rho of
  * Algorithm 2), then the lifetime of every packet version and a version row for each.
  * Uploads the per-round descriptors.  RFAST_ESCHED if the arrays are inconsistent (sizes,
@@ -201,11 +226,51 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s);
 int rfast_run(rfast_ctx* ctx, int32_t rounds, int sync);
 
 /* Stream-ordered copy of one view into a caller-owned HOST buffer of exactly `bytes` bytes
- * (RFAST_EINVAL on mismatch); returns after the copy has completed. */
+ * (RFAST_EINVAL on mismatch); returns after the copy has completed.  Allocates nothing. */
 int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes);
 
-/* Back to the initial state of the loaded schedule (x0, z^0, zero packets, round 0). */
+/* Back to the initial state of the loaded schedule (x0, z^0, zero packets, round 0).  Also
+ * clears the status of a bounded device-side wait that ran out (RFAST_ETIMEOUT). */
 int rfast_reset(rfast_ctx* ctx);
+
+/* Sets the round counter to `round` (0 .. K) without running anything.  Everything integer in
+ * Algorithm 1 -- the counters t_i, the stamps tau_v, tau_rho, which packet versions are in
+ * flight -- is a function of the schedule and the round, so it follows; the float state is
+ * left as it is and is meant to be loaded next with rfast_write_state / rfast_write_packet
+ * (state of another run of the same schedule, e.g. a reference implementation's, or a
+ * perturbed one).  RFAST_ESTATE without a schedule, RFAST_EINVAL outside 0 .. K. */
+int rfast_seek(rfast_ctx* ctx, int32_t round);
+
+/* Mirror of rfast_read_state for the float views: copies a caller-owned HOST buffer of exactly
+ * `bytes` bytes (fp32 row-major, unpadded) into the view, as of the handle's current round;
+ * returns after the copy has completed.
+ *   X, Y            all n rows (Y: the tracker z_i; a two-float tracker's low word is cleared)
+ *   G_LAST          the remembered sample gradients (RFAST_ESTATE for the element-wise
+ *                   objective, which recomputes it from x)
+ *   RHO_LATEST      rho of every G_C edge whose sender has been active (t_j >= 1); rows of
+ *                   other edges are ignored (rho^0 = 0 is not stored)
+ *   RHO_BUF         rho~ of every G_C edge with tau_rho >= 1; other rows are ignored.  rho~ is
+ *                   the consumed version kept alive: where tau_rho = t_j it is the same row as
+ *                   RHO_LATEST, so write RHO_BUF before RHO_LATEST
+ *   V_LATEST        rows flagged by RFAST_STATE_V_HELD; other rows are ignored
+ * Packets in flight that are neither the latest nor the buffered version of their edge are
+ * written with rfast_write_packet.  Integer views cannot be written (RFAST_EINVAL): they
+ * follow from the schedule and the round, see rfast_seek. */
+int rfast_write_state(rfast_ctx* ctx, int which, const void* src, size_t bytes);
+
+/* One packet version, addressed the way Algorithm 1 S3 stamps it.
+ *   graph = 0: the v packet of node `id` with local stamp `stamp` (v_id^stamp);
+ *   graph = 1: the running sum rho of G_C edge `id` (receiver-CSR edge id) with its sender's
+ *              local stamp `stamp`.
+ * The engine holds a version only from the round after it was produced until the last round
+ * in which the schedule makes some activation read it.  Returns RFAST_OK and copies p floats
+ * from / to the caller-owned HOST buffer (`bytes` = p * 4, RFAST_EINVAL otherwise), or
+ * RFAST_NOT_HELD (a positive code, nothing copied) when that version has no row at the
+ * handle's current round: it was never sent or is never read, it is yet to be produced, or its
+ * last reader has run.  RFAST_ESTATE for graph = 1 with RFAST_TRACKER_BUCKETS. */
+#define RFAST_NOT_HELD 1
+int rfast_read_packet(rfast_ctx* ctx, int graph, int32_t id, int32_t stamp, float* dst, size_t bytes);
+int rfast_write_packet(rfast_ctx* ctx, int graph, int32_t id, int32_t stamp, const float* src, size_t bytes);
 
 /* A counter (>= 0), or a negative status for an unknown id / NULL handle. */
 int64_t rfast_query(rfast_ctx* ctx, int what);
@@ -252,7 +317,13 @@ int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
  *          buckets begun and not yet consumed)
  *   out[3] max_c | sum_i g_i |   (the scale of out[2])
  *   out[4] || z ||_F
- * n_out must be 5 (RFAST_EINVAL otherwise); out is a caller-owned HOST array of doubles. */
+ *   out[5] || grad F(xbar) ||_2, the full gradient of F = sum_i f_i (every row of every shard,
+ *          no sampling) at the mean iterate; computed for the element-wise and the least-squares
+ *          objective, NaN for the others
+ *   out[6] the merit function of the non-convex analysis (Section V-B),
+ *          M_F(x) = || grad F(xbar) ||^2 + || x - 1 xbar^T ||^2 = out[5]^2 + out[0]^2 (NaN likewise)
+ * n_out is 5 (the first five only) or 7; RFAST_EINVAL otherwise.  out is a caller-owned HOST
+ * array of doubles. */
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out);
 
 /* Host-only companion of rfast_load_schedule (needs no CUDA device): compiles the schedule

@@ -25,6 +25,11 @@ STATE_X, STATE_Y, STATE_G_LAST, STATE_RHO_LATEST, STATE_RHO_BUF = 0, 1, 2, 3, 4
 STATE_T_LOCAL, STATE_USED_TAU_V, STATE_USED_TAU_RHO, STATE_TAU_V_END, STATE_TAU_RHO_END, STATE_ROUND = 5, 6, 7, 8, 9, 10
 Q_ROUND, Q_EVENTS_TOTAL, Q_EVENTS_RUN, Q_LAUNCHES, Q_BYTES_RUN, Q_V_SLOTS, Q_RHO_SLOTS = 0, 1, 2, 3, 4, 5, 6
 Q_DEVICE_BYTES, Q_N_USED_TAU_V, Q_N_USED_TAU_RHO, Q_BYTES_TOTAL = 7, 8, 9, 10
+Q_METHOD_BYTES_RUN, Q_METHOD_BYTES_TOTAL = 11, 12
+STATE_V_LATEST, STATE_V_HELD, STATE_TAU_V, STATE_TAU_RHO = 11, 12, 13, 14
+_FLOAT_VIEWS = (STATE_X, STATE_Y, STATE_G_LAST, STATE_RHO_LATEST, STATE_RHO_BUF, STATE_V_LATEST)
+NOT_HELD = 1
+GRAPH_R, GRAPH_C = 0, 1
 
 
 class RFastError(RuntimeError):
@@ -88,6 +93,10 @@ def lib():
         L.rfast_checkpoint_save.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         L.rfast_checkpoint_load.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         L.rfast_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+        L.rfast_seek.argtypes = [C.c_void_p, C.c_int32]
+        L.rfast_write_state.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t]
+        L.rfast_read_packet.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]
+        L.rfast_write_packet.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]
         L.rfast_ls_gradient_static.argtypes = [C.c_void_p] * 4 + [C.c_int32, C.c_int32, C.c_float,
                                                C.c_void_p, C.c_char_p, C.c_size_t]
         _lib = L
@@ -204,12 +213,42 @@ def rfast_query(handle, what: int) -> int:
 
 def rfast_read_state(handle, which: int, shape, out=None) -> np.ndarray:
     """shape: the view's shape; float views are float32, integer views int32."""
-    dt = np.float32 if which <= STATE_RHO_BUF else np.int32
+    dt = np.float32 if which in _FLOAT_VIEWS else np.int32
     if out is None:
         out = np.empty(shape, dtype=dt)
     assert out.dtype == dt and out.flags.c_contiguous
     _check(lib().rfast_read_state(handle, int(which), _ptr(out), out.nbytes), handle)
     return out
+
+
+def rfast_seek(handle, rnd: int) -> None:
+    _check(lib().rfast_seek(handle, int(rnd)), handle)
+
+
+def rfast_write_state(handle, which: int, values) -> None:
+    """values: the float view as an array (converted to contiguous float32)."""
+    a = _arr(values, np.float32)
+    _check(lib().rfast_write_state(handle, int(which), _ptr(a), a.nbytes), handle)
+
+
+def rfast_read_packet(handle, graph: int, ident: int, stamp: int, p: int):
+    """Payload (float32 [p]) of one packet version, or None when the engine does not hold it."""
+    out = np.empty(int(p), dtype=np.float32)
+    rc = lib().rfast_read_packet(handle, int(graph), int(ident), int(stamp), _ptr(out), out.nbytes)
+    if rc == NOT_HELD:
+        return None
+    _check(rc, handle)
+    return out
+
+
+def rfast_write_packet(handle, graph: int, ident: int, stamp: int, values) -> bool:
+    """True when the version is held and was written, False when the engine keeps no row for it."""
+    a = _arr(values, np.float32)
+    rc = lib().rfast_write_packet(handle, int(graph), int(ident), int(stamp), _ptr(a), a.nbytes)
+    if rc == NOT_HELD:
+        return False
+    _check(rc, handle)
+    return True
 
 
 def rfast_destroy(handle) -> None:
@@ -264,10 +303,11 @@ def rfast_checkpoint_load(handle, blob: np.ndarray) -> None:
 def rfast_diagnostics(handle) -> dict:
     """Consensus error, norm of the mean iterate, conservation residual (Lemma 3) and its scale,
     tracker norm, all computed on the device."""
-    out = np.zeros(5, dtype=np.float64)
-    _check(lib().rfast_diagnostics(handle, _ptr(out), 5), handle)
+    out = np.zeros(7, dtype=np.float64)
+    _check(lib().rfast_diagnostics(handle, _ptr(out), 7), handle)
     return {"consensus_error": out[0], "xbar_norm": out[1], "conservation_residual": out[2],
-            "gradient_sum_max": out[3], "tracker_norm": out[4]}
+            "gradient_sum_max": out[3], "tracker_norm": out[4], "full_gradient_norm": out[5],
+            "merit": out[6]}
 
 
 STATIC_MAX_ROWS = 65536
@@ -320,12 +360,26 @@ class Engine:
         shape = {STATE_X: (n, p), STATE_Y: (n, p), STATE_G_LAST: (n, p),
                  STATE_RHO_LATEST: (self.n_edges_c, p), STATE_RHO_BUF: (self.n_edges_c, p),
                  STATE_T_LOCAL: (n,), STATE_TAU_V_END: (self.n_edges_r,),
-                 STATE_TAU_RHO_END: (self.n_edges_c,), STATE_ROUND: (1,)}.get(which)
+                 STATE_TAU_RHO_END: (self.n_edges_c,), STATE_ROUND: (1,),
+                 STATE_V_LATEST: (n, p), STATE_V_HELD: (n,), STATE_TAU_V: (self.n_edges_r,),
+                 STATE_TAU_RHO: (self.n_edges_c,)}.get(which)
         if which == STATE_USED_TAU_V:
             shape = (self.query(Q_N_USED_TAU_V),)
         if which == STATE_USED_TAU_RHO:
             shape = (self.query(Q_N_USED_TAU_RHO),)
         return rfast_read_state(self.h, which, shape, out)
+
+    def seek(self, rnd):
+        rfast_seek(self.h, rnd)
+
+    def write(self, which, values):
+        rfast_write_state(self.h, which, values)
+
+    def read_packet(self, graph, ident, stamp):
+        return rfast_read_packet(self.h, graph, ident, stamp, self.p)
+
+    def write_packet(self, graph, ident, stamp, values):
+        return rfast_write_packet(self.h, graph, ident, stamp, values)
 
     def set_option(self, option, value):
         rfast_set_option(self.h, option, value)

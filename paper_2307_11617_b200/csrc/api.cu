@@ -22,6 +22,7 @@ int  mlp_plan_create(int n, int rows, int F, int H, int C, int B, int64_t stride
                      const float* d_feat, const __nv_bfloat16* xb, const float* x, float* gbuf, cudaStream_t st,
                      MlpPlan** out, size_t* dev_bytes, std::string& err);
 int  mlp_plan_status(MlpPlan* plan, cudaStream_t st);
+void mlp_plan_clear_status(MlpPlan* plan, cudaStream_t st);
 void mlp_plan_destroy(MlpPlan* plan);
 int  mlp_grad_launch(MlpPlan* plan, const GradArgs& g, const __nv_bfloat16* xb, const int* label,
                      int n_events, cudaStream_t st, int64_t* launches, std::string& err);
@@ -50,6 +51,12 @@ struct rfast_ctx {
     float* sp_val = nullptr;
     __nv_bfloat16* xb = nullptr;
     float *vbuf = nullptr, *rbuf = nullptr, *scratch = nullptr;
+    float* row_tmp = nullptr;         // one row (element-wise objective: a recomputed gradient row on its way out)
+    // diagnostics scratch, sized with the schedule: row selectors, per-block partial results,
+    // mean iterate, per-row residuals of the full least-squares gradient
+    int* d_diag_idx = nullptr;  int64_t diag_idx_cap = 0;
+    double* d_diag_part = nullptr;
+    float* d_xbar = nullptr;  float* d_diag_res = nullptr;
     MlpPlan* mlp = nullptr;
     // compiled schedule
     bool has_sched = false;
@@ -133,6 +140,7 @@ void free_schedule(rfast_ctx* c) {
     c->sched_bytes = 0;
     c->d_ev = c->d_init_ev = nullptr;
     c->vbuf = c->rbuf = c->scratch = nullptr;
+    c->d_diag_idx = nullptr; c->d_diag_part = nullptr; c->d_xbar = nullptr; c->d_diag_res = nullptr;
     c->d_act_ptr = nullptr; c->d_alpha_round = nullptr; c->d_bar = nullptr; c->d_pstatus = nullptr;
     c->persist_ok = false;
     c->has_sched = false;
@@ -146,6 +154,7 @@ ModelTraffic traffic_of(int model, bool compensated) {
     // the others: gradient reads x (the MLP: a bf16 copy written by the mix pass), writes g,
     // tracking reads z, g_old, g_new (5).  z's write and the packets are counted elsewhere.
     mt.grad_track_streams = (model == RFAST_MODEL_LOGISTIC_SPARSE ? 4 : 5) + (mt.elementwise ? 0 : (compensated ? 2 : 0));
+    mt.method_streams = 2;    // element-wise: d and b, the remembered gradient recomputed; others: g_old read, g_new written
     return mt;
 }
 
@@ -286,6 +295,9 @@ int check_device_status(rfast_ctx* ctx) {
 
 int reset_state(rfast_ctx* ctx) {
     const size_t plane = (size_t)ctx->n * ctx->stride * sizeof(float);
+    // a bounded wait that ran out earlier is forgotten: the state starts over
+    if (ctx->d_pstatus) CK(cudaMemsetAsync(ctx->d_pstatus, 0, sizeof(int), ctx->stream));
+    if (ctx->mlp) mlp_plan_clear_status(ctx->mlp, ctx->stream);
     if (ctx->x0) CK(cudaMemcpyAsync(ctx->x, ctx->x0, plane, cudaMemcpyDeviceToDevice, ctx->stream));
     else CK(cudaMemsetAsync(ctx->x, 0, plane, ctx->stream));
     const int n4 = (int)(ctx->stride / 4);
@@ -329,7 +341,7 @@ void rfast_destroy(rfast_ctx* c) {
     free_schedule(c);
     if (c->mlp) mlp_plan_destroy(c->mlp);
     void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
-                    c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb};
+                    c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb, c->row_tmp};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete c;
 }
@@ -375,6 +387,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
             CK(dev_alloc(ctx, &ctx->quad_b, plane));
             if ((rc = upload_rows(ctx, ctx->quad_d, prob->quad_d, ctx->n)) != RFAST_OK) return rc;
             if ((rc = upload_rows(ctx, ctx->quad_b, prob->quad_b, ctx->n)) != RFAST_OK) return rc;
+            CK(dev_alloc(ctx, &ctx->row_tmp, (size_t)ctx->stride));
             break;
         case RFAST_MODEL_LEAST_SQUARES:
         case RFAST_MODEL_SOFTMAX:
@@ -536,6 +549,15 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
             const int want = std::max(1, ctx->max_round_events * per_ev);
             ctx->persist_grid = std::min(want, sms);          // one CTA per SM keeps the barrier short
             ctx->persist_ok = true;
+        }
+    }
+    {   // diagnostics scratch (nothing is allocated when the diagnostics run)
+        ctx->diag_idx_cap = (int64_t)ctx->n + 2 * (int64_t)std::max(std::max(ctx->Cg.E, c.n_rho_slots), 1);
+        CK(dev_alloc(ctx, &ctx->d_diag_idx, (size_t)ctx->diag_idx_cap, true));
+        CK(dev_alloc(ctx, &ctx->d_diag_part, (size_t)((ctx->p + kThreads - 1) / kThreads) * kDiagSlots, true));
+        if (ctx->model == RFAST_MODEL_LEAST_SQUARES) {
+            CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
+            CK(dev_alloc(ctx, &ctx->d_diag_res, (size_t)ctx->n * ctx->rows, true));
         }
     }
     ctx->has_sched = true;
@@ -714,6 +736,8 @@ int64_t rfast_query(rfast_ctx* ctx, int what) {
         case RFAST_Q_LAUNCHES: return ctx->launches;
         case RFAST_Q_BYTES_RUN: return hs ? c.round_streams[ctx->round] * 4 * ctx->p : 0;
         case RFAST_Q_BYTES_TOTAL: return hs ? c.round_streams[c.K] * 4 * ctx->p : 0;
+        case RFAST_Q_METHOD_BYTES_RUN: return hs ? c.round_streams_method[ctx->round] * 4 * ctx->p : 0;
+        case RFAST_Q_METHOD_BYTES_TOTAL: return hs ? c.round_streams_method[c.K] * 4 * ctx->p : 0;
         case RFAST_Q_V_SLOTS: return hs ? c.n_v_slots : 0;
         case RFAST_Q_RHO_SLOTS: return hs ? c.n_rho_slots : 0;
         case RFAST_Q_DEVICE_BYTES: return (int64_t)ctx->dev_bytes;
@@ -723,12 +747,152 @@ int64_t rfast_query(rfast_ctx* ctx, int what) {
     }
 }
 
+}  // extern "C"
+
+namespace {
+
+// Integer state of Algorithm 1 as of the handle's current round, replayed from the compiled
+// schedule: local counters, the row of every edge's latest and buffered running sum, the stamp
+// and row of every node's last v packet.
+struct RoundView {
+    std::vector<int> t;                       // [n]   t_i
+    std::vector<int> rho_latest, rho_buf;     // [E_C] row ids, -1: nothing stored (stamp 0)
+    std::vector<int> tau_v, tau_rho;          // [E_R], [E_C] stamps as of the receiver's last activation
+    std::vector<int> v_row, v_stamp;          // [n]   row of the last v packet if the engine holds it, else -1 / 0
+};
+
+// is a version written in round `write` and last read in round `last` held at round `round`?
+inline bool version_live(int write, int last, int round) { return write < round && last >= round; }
+
+RoundView round_view(const rfast_ctx* ctx) {
+    const Compiled& c = ctx->comp;
+    const int n = ctx->n;
+    RoundView v;
+    v.t.assign(n, 0);
+    v.rho_latest.assign(ctx->Cg.E, -1);
+    v.rho_buf.assign(ctx->Cg.E, -1);
+    v.tau_v.assign(ctx->R.E, 0);
+    v.tau_rho.assign(ctx->Cg.E, 0);
+    v.v_row.assign(n, -1);
+    v.v_stamp.assign(n, 0);
+    const int ev_end = c.act_ptr[ctx->round];
+    std::vector<int> last_ev(n, -1);
+    for (int ev = 0; ev < ev_end; ++ev) {
+        const EvDesc& d = c.ev[ev];
+        const int i = d.node;
+        v.t[i]++;
+        last_ev[i] = ev;
+        for (int e = ctx->R.rowptr[i], k = 0; e < ctx->R.rowptr[i + 1]; ++e, ++k) v.tau_v[e] = c.used_tau_v[c.in_r_off[ev] + k];
+        for (int e = ctx->Cg.rowptr[i], k = 0; e < ctx->Cg.rowptr[i + 1]; ++e, ++k) v.tau_rho[e] = c.used_tau_rho[c.in_c_off[ev] + k];
+        if (ctx->buckets) continue;
+        for (int k = 0; k < d.out_cnt; ++k) v.rho_latest[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
+        for (int k = 0; k < d.news_cnt; ++k) v.rho_buf[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
+    }
+    for (int i = 0; i < n; ++i) {
+        const int ev = last_ev[i];
+        if (ev >= 0 && c.v_slot[ev] >= 0 && version_live(c.v_write[ev], c.v_last[ev], ctx->round)) {
+            v.v_row[i] = c.v_slot[ev];
+            v.v_stamp[i] = v.t[i];
+        }
+    }
+    return v;
+}
+
+// Rows of a pool, picked by index, straight out of / into the caller's unpadded buffer: one
+// copy per row, nothing staged and nothing allocated.  A negative index reads as a zero row
+// and is skipped on a write.  lo_off > 0: the pool keeps a low-order word per value that far
+// behind; a write clears it.
+int rows_by_index(rfast_ctx* ctx, float* pool, const std::vector<int>& idx, void* host, bool write, int64_t lo_off = 0) {
+    const size_t rowb = (size_t)ctx->p * sizeof(float);
+    char* h = (char*)host;
+    for (size_t r = 0; r < idx.size(); ++r, h += rowb) {
+        if (idx[r] < 0) {
+            if (!write) std::memset(h, 0, rowb);
+            continue;
+        }
+        float* d = pool + (int64_t)idx[r] * ctx->stride;
+        if (write) {
+            CK(cudaMemcpyAsync(d, h, rowb, cudaMemcpyHostToDevice, ctx->stream));
+            if (lo_off > 0) CK(cudaMemsetAsync(d + lo_off, 0, rowb, ctx->stream));
+        } else {
+            CK(cudaMemcpyAsync(h, d, rowb, cudaMemcpyDeviceToHost, ctx->stream));
+        }
+    }
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
+// Where the engine keeps packet version (graph, id, stamp) at the current round: row id, or -1.
+int packet_row(rfast_ctx* ctx, int graph, int id, int stamp, int* row, std::string& err) {
+    const Compiled& c = ctx->comp;
+    *row = -1;
+    if (graph == 0) {
+        if (id < 0 || id >= ctx->n) { err = "packet: node id out of range"; return RFAST_EINVAL; }
+        if (stamp < 1 || stamp > (int)c.ev_of[id].size()) return RFAST_OK;
+        const int ev = c.ev_of[id][stamp - 1];
+        if (c.v_slot[ev] >= 0 && version_live(c.v_write[ev], c.v_last[ev], ctx->round)) *row = c.v_slot[ev];
+        return RFAST_OK;
+    }
+    if (graph != 1) { err = "packet: graph must be 0 (v over G_R) or 1 (rho over G_C)"; return RFAST_EINVAL; }
+    if (ctx->buckets) { err = "packet: the bucket tracker keeps no running sums"; return RFAST_ESTATE; }
+    if (id < 0 || id >= ctx->Cg.E) { err = "packet: edge id out of range"; return RFAST_EINVAL; }
+    const int j = ctx->Cg.col[id];
+    if (stamp < 1 || stamp > (int)c.ev_of[j].size()) return RFAST_OK;
+    const int64_t vid = c.out_c_off[c.ev_of[j][stamp - 1]] + ctx->Cg.opos[id];
+    if (c.rho_slot[vid] >= 0 && version_live(c.rho_write[vid], c.rho_last[vid], ctx->round)) *row = c.rho_slot[vid];
+    return RFAST_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rfast_seek(rfast_ctx* ctx, int32_t round) {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (round < 0 || round > ctx->comp.K) return set_err(ctx, RFAST_EINVAL, "seek: round outside 0 .. K");
+    CK(cudaStreamSynchronize(ctx->stream));
+    ctx->round = round;
+    return RFAST_OK;
+}
+
+int rfast_read_packet(rfast_ctx* ctx, int graph, int32_t id, int32_t stamp, float* dst, size_t bytes) {
+    if (!ctx || !dst) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (bytes != (size_t)ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "packet: size mismatch");
+    int row = -1;
+    std::string err;
+    const int rc = packet_row(ctx, graph, id, stamp, &row, err);
+    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+    if (row < 0) return RFAST_NOT_HELD;
+    const float* src = (graph == 0 ? ctx->vbuf : ctx->rbuf) + (int64_t)row * ctx->stride;
+    CK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
+int rfast_write_packet(rfast_ctx* ctx, int graph, int32_t id, int32_t stamp, const float* src, size_t bytes) {
+    if (!ctx || !src) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (bytes != (size_t)ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "packet: size mismatch");
+    int row = -1;
+    std::string err;
+    const int rc = packet_row(ctx, graph, id, stamp, &row, err);
+    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+    if (row < 0) return RFAST_NOT_HELD;
+    float* dst = (graph == 0 ? ctx->vbuf : ctx->rbuf) + (int64_t)row * ctx->stride;
+    CK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, ctx->stream));
+    if (graph == 1 && ctx->rho2) CK(cudaMemsetAsync(dst + ctx->rlo_off(), 0, bytes, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));
+    return RFAST_OK;
+}
+
 int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
     if (!ctx || !dst) return RFAST_EINVAL;
     const Compiled& c = ctx->comp;
     auto ints = [&](const int* src, size_t cnt) {
         if (bytes != cnt * sizeof(int)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
-        std::memcpy(dst, src, bytes);
+        if (bytes) std::memcpy(dst, src, bytes);
         return RFAST_OK;
     };
     const int n = ctx->n, n4 = (int)(ctx->stride / 4);
@@ -740,24 +904,12 @@ int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
         CK(cudaStreamSynchronize(ctx->stream));
         return RFAST_OK;
     };
-    // rows picked by index from a pool, staged through a temporary
-    auto gathered = [&](const float* pool, const std::vector<int>& idx) -> int {
-        const int64_t rows = (int64_t)idx.size();
-        if (bytes != (size_t)rows * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
-        if (rows == 0) return RFAST_OK;
-        float* tmp = nullptr; int* didx = nullptr;
-        CK(cudaMalloc((void**)&tmp, (size_t)rows * ctx->stride * sizeof(float)));
-        cudaError_t e = cudaMalloc((void**)&didx, rows * sizeof(int));
-        if (e != cudaSuccess) { cudaFree(tmp); return set_err(ctx, RFAST_ENOMEM, "read_state: temporary"); }
-        cudaMemcpyAsync(didx, idx.data(), rows * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
-        k_gather_rows<<<dim3((n4 + kThreads - 1) / kThreads, (unsigned)rows), kThreads, 0, ctx->stream>>>(
-            pool, didx, tmp, ctx->stride, ctx->stride, n4);
-        int rc = rows_out(tmp, rows);
-        cudaStreamSynchronize(ctx->stream);
-        cudaFree(tmp); cudaFree(didx);
-        return rc;
+    auto picked = [&](float* pool, const std::vector<int>& idx) -> int {
+        if (bytes != idx.size() * (size_t)ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
+        return rows_by_index(ctx, pool, idx, dst, false);
     };
-    if (which <= RFAST_STATE_RHO_BUF) {
+    const bool is_float = which <= RFAST_STATE_RHO_BUF || which == RFAST_STATE_V_LATEST;
+    if (is_float) {
         int rc = check_device_status(ctx);
         if (rc != RFAST_OK) return rc;
     }
@@ -768,50 +920,100 @@ int rfast_read_state(rfast_ctx* ctx, int which, void* dst, size_t bytes) try {
         default: break;
     }
     if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
-    // replay of the integer bookkeeping up to the current round
-    std::vector<int> t(n, 0);
-    const int ev_end = c.act_ptr[ctx->round];
-    for (int ev = 0; ev < ev_end; ++ev) t[c.act_node[ev]]++;
     switch (which) {
-        case RFAST_STATE_T_LOCAL: return ints(t.data(), n);
         case RFAST_STATE_USED_TAU_V: return ints(c.used_tau_v.data(), c.used_tau_v.size());
         case RFAST_STATE_USED_TAU_RHO: return ints(c.used_tau_rho.data(), c.used_tau_rho.size());
         case RFAST_STATE_TAU_V_END: return ints(c.tau_v_end.data(), c.tau_v_end.size());
         case RFAST_STATE_TAU_RHO_END: return ints(c.tau_rho_end.data(), c.tau_rho_end.size());
+        default: break;
+    }
+    const RoundView rv = round_view(ctx);
+    switch (which) {
+        case RFAST_STATE_T_LOCAL: return ints(rv.t.data(), n);
+        case RFAST_STATE_TAU_V: return ints(rv.tau_v.data(), rv.tau_v.size());
+        case RFAST_STATE_TAU_RHO: return ints(rv.tau_rho.data(), rv.tau_rho.size());
+        case RFAST_STATE_V_HELD: return ints(rv.v_stamp.data(), n);
+        case RFAST_STATE_V_LATEST: return picked(ctx->vbuf, rv.v_row);
         case RFAST_STATE_G_LAST: {
             if (ctx->model == RFAST_MODEL_QUAD_DIAG) {
+                // not stored for the element-wise objective: recomputed from x, a row at a time
                 if (bytes != (size_t)n * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "read_state: size mismatch");
-                float* tmp = nullptr;
-                CK(cudaMalloc((void**)&tmp, (size_t)n * ctx->stride * sizeof(float)));
-                k_quad_grad<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(
-                    ctx->x, ctx->quad_d, ctx->quad_b, tmp, ctx->stride, n4);
-                int rc = rows_out(tmp, n);
-                cudaStreamSynchronize(ctx->stream);
-                cudaFree(tmp);
-                return rc;
+                for (int i = 0; i < n; ++i) {
+                    const int64_t row = (int64_t)i * ctx->stride;
+                    k_quad_grad<<<dim3((n4 + kThreads - 1) / kThreads, 1), kThreads, 0, ctx->stream>>>(
+                        ctx->x + row, ctx->quad_d + row, ctx->quad_b + row, ctx->row_tmp, ctx->stride, n4);
+                    CK(cudaMemcpyAsync((char*)dst + (size_t)i * ctx->p * sizeof(float), ctx->row_tmp,
+                                       (size_t)ctx->p * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+                }
+                CK(cudaStreamSynchronize(ctx->stream));
+                return RFAST_OK;
             }
             std::vector<int> idx(n);
-            for (int i = 0; i < n; ++i) idx[i] = (t[i] & 1) * n + i;
-            return gathered(ctx->gbuf, idx);
+            for (int i = 0; i < n; ++i) idx[i] = (rv.t[i] & 1) * n + i;
+            return picked(ctx->gbuf, idx);
         }
         case RFAST_STATE_RHO_LATEST:
-        case RFAST_STATE_RHO_BUF: {
+        case RFAST_STATE_RHO_BUF:
             if (ctx->buckets)
                 return set_err(ctx, RFAST_ESTATE, "read_state: the bucket tracker keeps no running sums (rho, rho~ views do not exist)");
-            std::vector<int> idx(ctx->Cg.E, -1);
-            for (int ev = 0; ev < ev_end; ++ev) {
-                const EvDesc& d = c.ev[ev];
-                if (which == RFAST_STATE_RHO_LATEST)
-                    for (int k = 0; k < d.out_cnt; ++k) idx[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
-                else
-                    for (int k = 0; k < d.news_cnt; ++k) idx[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
-            }
-            return gathered(ctx->rbuf, idx);
-        }
+            return picked(ctx->rbuf, which == RFAST_STATE_RHO_LATEST ? rv.rho_latest : rv.rho_buf);
         default: return set_err(ctx, RFAST_EINVAL, "read_state: unknown view");
     }
 } catch (...) {
     return set_err(ctx, RFAST_ENOMEM, "read_state: host allocation failed");
+}
+
+int rfast_write_state(rfast_ctx* ctx, int which, const void* src, size_t bytes) try {
+    if (!ctx || !src) return RFAST_EINVAL;
+    const int n = ctx->n, n4 = (int)(ctx->stride / 4);
+    auto rows_in = [&](float* dev) -> int {
+        if (bytes != (size_t)n * ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "write_state: size mismatch");
+        CK(cudaMemcpy2DAsync(dev, ctx->stride * sizeof(float), src, ctx->p * sizeof(float), ctx->p * sizeof(float),
+                             n, cudaMemcpyHostToDevice, ctx->stream));     // the padding stays zero
+        return RFAST_OK;
+    };
+    auto picked = [&](float* pool, const std::vector<int>& idx, int64_t lo_off) -> int {
+        if (bytes != idx.size() * (size_t)ctx->p * sizeof(float)) return set_err(ctx, RFAST_EINVAL, "write_state: size mismatch");
+        return rows_by_index(ctx, pool, idx, const_cast<void*>(src), true, lo_off);
+    };
+    int rc;
+    switch (which) {
+        case RFAST_STATE_X:
+            if ((rc = rows_in(ctx->x)) != RFAST_OK) return rc;
+            if (ctx->model == RFAST_MODEL_MLP) {           // the matrix products read a bf16 copy of x
+                k_rows_to_bf16<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(ctx->x, ctx->xb, ctx->stride, n4);
+                CK(cudaGetLastError());
+            }
+            CK(cudaStreamSynchronize(ctx->stream));
+            return RFAST_OK;
+        case RFAST_STATE_Y:
+            if ((rc = rows_in(ctx->z)) != RFAST_OK) return rc;
+            if (ctx->zc) CK(cudaMemsetAsync(ctx->zc, 0, (size_t)n * ctx->stride * sizeof(float), ctx->stream));
+            CK(cudaStreamSynchronize(ctx->stream));
+            return RFAST_OK;
+        default: break;
+    }
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (which != RFAST_STATE_G_LAST && which != RFAST_STATE_RHO_LATEST && which != RFAST_STATE_RHO_BUF &&
+        which != RFAST_STATE_V_LATEST)
+        return set_err(ctx, RFAST_EINVAL, "write_state: only the float views can be written (integer state follows from the schedule and the round)");
+    const RoundView rv = round_view(ctx);
+    switch (which) {
+        case RFAST_STATE_G_LAST: {
+            if (ctx->model == RFAST_MODEL_QUAD_DIAG)
+                return set_err(ctx, RFAST_ESTATE, "write_state: the element-wise objective keeps no gradient (it is recomputed from x)");
+            std::vector<int> idx(n);
+            for (int i = 0; i < n; ++i) idx[i] = (rv.t[i] & 1) * n + i;
+            return picked(ctx->gbuf, idx, 0);
+        }
+        case RFAST_STATE_V_LATEST: return picked(ctx->vbuf, rv.v_row, 0);
+        default:
+            if (ctx->buckets)
+                return set_err(ctx, RFAST_ESTATE, "write_state: the bucket tracker keeps no running sums (rho, rho~ views do not exist)");
+            return picked(ctx->rbuf, which == RFAST_STATE_RHO_LATEST ? rv.rho_latest : rv.rho_buf, ctx->rlo_off());
+    }
+} catch (...) {
+    return set_err(ctx, RFAST_ENOMEM, "write_state: host allocation failed");
 }
 
 int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32_t* used_tau_v,
@@ -937,21 +1139,15 @@ int rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes) {
 }
 
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
-    if (!ctx || !out || n_out != 5) return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5") : RFAST_EINVAL;
+    if (!ctx || !out || (n_out != 5 && n_out != 7))
+        return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5 or 7") : RFAST_EINVAL;
     if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
     const Compiled& c = ctx->comp;
     const int n = ctx->n;
-    int E = ctx->Cg.E;
     // which rows hold the current g, the latest rho and the buffered rho of every edge
-    std::vector<int> gsel(n), latest(std::max(E, 1), -1), buf(std::max(E, 1), -1), t(n, 0);
-    const int ev_end = c.act_ptr[ctx->round];
-    for (int ev = 0; ev < ev_end; ++ev) {
-        const EvDesc& d = c.ev[ev];
-        t[d.node]++;
-        if (ctx->buckets) continue;
-        for (int k = 0; k < d.out_cnt; ++k) latest[c.out_edge[d.out_beg + k]] = c.out_new[d.out_beg + k];
-        for (int k = 0; k < d.news_cnt; ++k) buf[c.news_edge[d.news_beg + k]] = c.news_new[d.news_beg + k];
-    }
+    const RoundView rv = round_view(ctx);
+    std::vector<int> gsel(n), latest = rv.rho_latest, buf = rv.rho_buf;
+    int E = ctx->Cg.E;
     if (ctx->buckets) {
         // the mass in transit is the content of the buckets begun and not yet consumed
         latest.clear();
@@ -959,39 +1155,46 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
             if (c.rho_leader[v] == (int64_t)v && c.rho_write[v] < ctx->round && c.rho_last[v] >= ctx->round)
                 latest.push_back(c.rho_slot[v]);
         E = (int)latest.size();
-        if (latest.empty()) latest.push_back(-1);
         buf.assign(latest.size(), -1);
     }
-    for (int i = 0; i < n; ++i) gsel[i] = (t[i] & 1) * n + i;
+    for (int i = 0; i < n; ++i) gsel[i] = (rv.t[i] & 1) * n + i;
+    if ((int64_t)n + 2 * (int64_t)E > ctx->diag_idx_cap) return set_err(ctx, RFAST_ESTATE, "diagnostics: scratch too small");
     const int blocks = (int)((ctx->p + kThreads - 1) / kThreads);
-    int *d_gsel = nullptr, *d_latest = nullptr, *d_buf = nullptr;
-    double* d_part = nullptr;
-    auto cleanup = [&]() { cudaFree(d_gsel); cudaFree(d_latest); cudaFree(d_buf); cudaFree(d_part); };
-    if (cudaMalloc((void**)&d_gsel, n * sizeof(int)) != cudaSuccess ||
-        cudaMalloc((void**)&d_latest, latest.size() * sizeof(int)) != cudaSuccess ||
-        cudaMalloc((void**)&d_buf, buf.size() * sizeof(int)) != cudaSuccess ||
-        cudaMalloc((void**)&d_part, (size_t)blocks * 5 * sizeof(double)) != cudaSuccess) {
-        cleanup();
-        return set_err(ctx, RFAST_ENOMEM, "diagnostics: temporary allocation failed");
+    int *d_gsel = ctx->d_diag_idx, *d_latest = d_gsel + n, *d_buf = d_latest + E;
+    CK(cudaMemcpyAsync(d_gsel, gsel.data(), n * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+    if (E > 0) {
+        CK(cudaMemcpyAsync(d_latest, latest.data(), E * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+        CK(cudaMemcpyAsync(d_buf, buf.data(), E * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
     }
-    cudaMemcpyAsync(d_gsel, gsel.data(), n * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
-    cudaMemcpyAsync(d_latest, latest.data(), latest.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
-    cudaMemcpyAsync(d_buf, buf.data(), buf.size() * sizeof(int), cudaMemcpyHostToDevice, ctx->stream);
+    const bool want_mf = n_out == 7;
+    const bool ls = ctx->model == RFAST_MODEL_LEAST_SQUARES;
     k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
                                                           ctx->quad_b, ctx->rbuf, ctx->rlo_off(), d_latest, d_buf, n, E,
-                                                          ctx->stride, ctx->p, d_part);
-    std::vector<double> part((size_t)blocks * 5);
-    cudaError_t e = cudaMemcpyAsync(part.data(), d_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
-    cleanup();
-    if (e != cudaSuccess) return set_err(ctx, RFAST_ECUDA, std::string("diagnostics: ") + cudaGetErrorString(e));
-    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0;
+                                                          ctx->stride, ctx->p, want_mf && ls ? ctx->d_xbar : nullptr,
+                                                          ctx->d_diag_part);
+    if (want_mf && ls) {
+        k_diag_ls_residual<<<dim3((ctx->rows + 7) / 8, n), 256, 0, ctx->stream>>>(ctx->feat, ctx->target, ctx->d_xbar,
+                                                                                    ctx->d_diag_res, ctx->rows, ctx->F);
+        k_diag_ls_grad<<<blocks, kThreads, 0, ctx->stream>>>(ctx->feat, ctx->d_xbar, ctx->d_diag_res, n, ctx->rows,
+                                                               ctx->F, ctx->l2, ctx->d_diag_part);
+    }
+    CK(cudaGetLastError());
+    std::vector<double> part((size_t)blocks * kDiagSlots);
+    CK(cudaMemcpyAsync(part.data(), ctx->d_diag_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
+    CK(cudaStreamSynchronize(ctx->stream));       // the host vectors above may go now
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0;
     for (int b = 0; b < blocks; ++b) {          // fixed order: the same bits on every run
-        cons += part[(size_t)b * 5]; xb2 += part[(size_t)b * 5 + 1];
-        res = std::max(res, part[(size_t)b * 5 + 2]); gs = std::max(gs, part[(size_t)b * 5 + 3]);
-        z2 += part[(size_t)b * 5 + 4];
+        const double* q = part.data() + (size_t)b * kDiagSlots;
+        cons += q[0]; xb2 += q[1];
+        res = std::max(res, q[2]); gs = std::max(gs, q[3]);
+        z2 += q[4]; gf2 += q[5];
     }
     out[0] = std::sqrt(std::max(cons, 0.0)); out[1] = std::sqrt(xb2); out[2] = res; out[3] = gs; out[4] = std::sqrt(z2);
+    if (want_mf) {
+        const bool have = ls || ctx->model == RFAST_MODEL_QUAD_DIAG;
+        out[5] = have ? std::sqrt(gf2) : std::nan("");
+        out[6] = have ? gf2 + std::max(cons, 0.0) : std::nan("");
+    }
     return RFAST_OK;
 } catch (...) {
     return set_err(ctx, RFAST_ENOMEM, "diagnostics: host allocation failed");

@@ -181,7 +181,8 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     const int INF = INT_MAX;
     std::vector<std::vector<Pend>> pend_v(R.E), pend_c(C.E);
     std::vector<int> tau_v(R.E, 0), tau_rho(C.E, 0), t(n, 0);
-    std::vector<std::vector<int>> ev_of(n);            // node -> event id of stamp s at [s-1]
+    c.ev_of.assign(n, {});
+    std::vector<std::vector<int>>& ev_of = c.ev_of;    // node -> event id of stamp s at [s-1]
     c.used_tau_v.reserve(c.in_r_off[nE]);
     c.used_tau_rho.reserve(c.in_c_off[nE]);
     c.prev_tau_rho.reserve(c.in_c_off[nE]);
@@ -336,11 +337,12 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     // ---- pass 3: device descriptors and the method's traffic ---------------------------------
     c.ev.resize(nE);
     c.round_streams.assign(K + 1, 0);
+    c.round_streams_method.assign(K + 1, 0);
     c.mix_slot.reserve(c.in_r_off[nE]);  c.mix_w.reserve(c.in_r_off[nE]);
     c.news_new.reserve(c.in_c_off[nE]);  c.news_prev.reserve(c.in_c_off[nE]);  c.news_edge.reserve(c.in_c_off[nE]);
     c.out_cur.reserve(nRho);  c.out_new.reserve(nRho);  c.out_a.reserve(nRho);  c.out_edge.reserve(nRho);
     for (int r = 0; r < K; ++r) {
-        int64_t streams = 0;
+        int64_t streams = 0, method = 0;
         for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
             const int i = c.act_node[ev];
             EvDesc d{};
@@ -394,12 +396,15 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             c.ev[ev] = d;
             // fp32 streams per coordinate: S1/S2a read x, z, the neighbours' v, write v (if a
             // packet leaves) and x; S2b/S2c read the news, write z and the running sums
-            int64_t st = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
-            if (mt.elementwise) st += mt.data_streams;
-            else st += mt.grad_track_streams;
-            streams += st;
+            const int64_t base = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
+            streams += base + (mt.elementwise ? mt.data_streams : mt.grad_track_streams);
+            // what the method itself must move: x and z read once, the gradient moved once
+            // (remembered one read, new one written), no stream that exists only because the
+            // step is split over several kernels or because of the tracker's arithmetic
+            method += base + mt.method_streams;
         }
         c.round_streams[r + 1] = c.round_streams[r] + streams;
+        c.round_streams_method[r + 1] = c.round_streams_method[r] + method;
     }
     out = std::move(c);
     return RFAST_OK;

@@ -752,6 +752,10 @@ int mlp_grad_launch(MlpPlan* p, const GradArgs& g, const __nv_bfloat16* xb, cons
     return RFAST_OK;
 }
 
+void mlp_plan_clear_status(MlpPlan* p, cudaStream_t st) {
+    if (p) cudaMemsetAsync(p->status, 0, sizeof(int), st);
+}
+
 // 0 when no bounded wait ran out so far (synchronises the stream)
 int mlp_plan_status(MlpPlan* p, cudaStream_t st) {
     int h = 0;

@@ -741,37 +741,28 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ range_ptr, in
     }
 }
 
-// row copy helpers ----------------------------------------------------------------------------
-// dst[r][0..n4) = src[idx ? idx[r] : r][0..n4); a negative index gives a zero row.  grid = (tiles, rows)
-__global__ void __launch_bounds__(kThreads)
-k_gather_rows(const float* __restrict__ src, const int* __restrict__ idx, float* __restrict__ dst,
-              int64_t src_stride, int64_t dst_stride, int n4) {
-    const int i4 = blockIdx.x * kThreads + threadIdx.x;
-    if (i4 >= n4) return;
-    const int r = idx ? idx[blockIdx.y] : (int)blockIdx.y;
-    float4 v = make_float4(0, 0, 0, 0);
-    if (r >= 0) v = reinterpret_cast<const float4*>(src + (int64_t)r * src_stride)[i4];
-    reinterpret_cast<float4*>(dst + (int64_t)blockIdx.y * dst_stride)[i4] = v;
-}
-
 // Diagnostics: per coordinate, sums over nodes and edges; per block, partial results.
 //   part[block][0] = sum_c (sum_i x_ic^2 - n xbar_c^2)    (consensus error squared)
 //   part[block][1] = sum_c xbar_c^2
 //   part[block][2] = max_c | sum_i z_ic + sum_e (rho_ec - rho~_ec) - sum_i g_ic |
 //   part[block][3] = max_c | sum_i g_ic |
 //   part[block][4] = sum_c sum_i z_ic^2
+//   part[block][5] = sum_c (grad F(xbar))_c^2 for the element-wise objective, where the full gradient
+//                    sum_i d_ic^2 (xbar_c - b_ic) is coordinate-wise; 0 otherwise
 // g_i is row gsel[i] of gpool (or recomputed for the element-wise objective when gpool is null).
+// xbar_out (may be null) receives the mean iterate in fp32.
 // grid = tiles of kThreads coordinates (scalar: diagnostics favour clarity over speed)
+constexpr int kDiagSlots = 6;
 __global__ void __launch_bounds__(kThreads)
 k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const float* __restrict__ zc,
               const float* __restrict__ gpool, const int* __restrict__ gsel,
               const float* __restrict__ qd, const float* __restrict__ qb,
               const float* __restrict__ rbuf, int64_t rlo_off, const int* __restrict__ rho_latest,
               const int* __restrict__ rho_buf, int n, int n_edges, int64_t stride, int64_t p,
-              double* __restrict__ part) {
-    __shared__ double red[5][kThreads];
+              float* __restrict__ xbar_out, double* __restrict__ part) {
+    __shared__ double red[kDiagSlots][kThreads];
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0;
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0;
     if (c < p) {
         double sx = 0, sx2 = 0, sz = 0, sg = 0;
         for (int i = 0; i < n; ++i) {
@@ -799,9 +790,18 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
         xb2 = xbar * xbar;
         res = fabs(sz + mass - sg);
         gs = fabs(sg);
+        if (xbar_out) xbar_out[c] = (float)xbar;
+        if (!gpool) {
+            double gf = 0;
+            for (int i = 0; i < n; ++i) {
+                const double d = qd[(int64_t)i * stride + c];
+                gf += d * d * (xbar - (double)qb[(int64_t)i * stride + c]);
+            }
+            gf2 = gf * gf;
+        }
     }
     red[0][threadIdx.x] = cons; red[1][threadIdx.x] = xb2; red[2][threadIdx.x] = res;
-    red[3][threadIdx.x] = gs; red[4][threadIdx.x] = z2;
+    red[3][threadIdx.x] = gs; red[4][threadIdx.x] = z2; red[5][threadIdx.x] = gf2;
     __syncthreads();
     for (int s = kThreads / 2; s > 0; s >>= 1) {
         if (threadIdx.x < s) {
@@ -810,10 +810,52 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
             red[2][threadIdx.x] = fmax(red[2][threadIdx.x], red[2][threadIdx.x + s]);
             red[3][threadIdx.x] = fmax(red[3][threadIdx.x], red[3][threadIdx.x + s]);
             red[4][threadIdx.x] += red[4][threadIdx.x + s];
+            red[5][threadIdx.x] += red[5][threadIdx.x + s];
         }
         __syncthreads();
     }
-    if (threadIdx.x < 5) part[(int64_t)blockIdx.x * 5 + threadIdx.x] = red[threadIdx.x][0];
+    if (threadIdx.x < kDiagSlots) part[(int64_t)blockIdx.x * kDiagSlots + threadIdx.x] = red[threadIdx.x][0];
+}
+
+// Full least-squares gradient at the mean iterate, for the merit function:
+// residuals of every row of every shard, r_ik = a_ik . xbar - y_ik.  grid = (ceil(rows / 8), n)
+__global__ void __launch_bounds__(256)
+k_diag_ls_residual(const float* __restrict__ feat, const float* __restrict__ target,
+                   const float* __restrict__ xbar, float* __restrict__ res, int rows, int F) {
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (k >= rows) return;
+    const int64_t r = (int64_t)blockIdx.y * rows + k;
+    const float* a = feat + r * F;
+    float s = 0.f;
+    for (int c = lane; c < F; c += 32) s = fmaf(a[c], xbar[c], s);
+    s = warp_sum(s);
+    if (lane == 0) res[r] = s - target[r];
+}
+// ... then (grad F(xbar))_c = sum_i [ (1/rows) sum_k a_ik[c] r_ik + l2 xbar_c ], squared and summed
+// per block into part[block][5].  grid = tiles of kThreads coordinates
+__global__ void __launch_bounds__(kThreads)
+k_diag_ls_grad(const float* __restrict__ feat, const float* __restrict__ xbar, const float* __restrict__ res,
+               int n, int rows, int F, float l2, double* __restrict__ part) {
+    __shared__ double red[kThreads];
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    double gf = 0;
+    if (c < F) {
+        for (int i = 0; i < n; ++i) {
+            double s = 0;
+            for (int k = 0; k < rows; ++k) {
+                const int64_t r = (int64_t)i * rows + k;
+                s += (double)feat[r * F + c] * (double)res[r];
+            }
+            gf += s / rows + (double)l2 * (double)xbar[c];
+        }
+    }
+    red[threadIdx.x] = gf * gf;
+    __syncthreads();
+    for (int s = kThreads / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) part[(int64_t)blockIdx.x * kDiagSlots + 5] = red[0];
 }
 
 // bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)

@@ -59,7 +59,9 @@ struct Compiled {
     std::vector<int>    news_new, news_prev, news_edge;
     std::vector<int>    out_cur, out_new, out_edge;  std::vector<float> out_a;
     // fp32 streams per coordinate (method traffic), prefix sums over rounds
-    std::vector<int64_t> round_streams;   // [K+1]
+    std::vector<int64_t> round_streams;          // [K+1] streams the kernels touch
+    std::vector<int64_t> round_streams_method;   // [K+1] streams the method itself must move
+    std::vector<std::vector<int>> ev_of;         // node -> event id of its stamp s at [s-1]
 };
 
 // Arguments shared by the sample-gradient kernels.
@@ -79,6 +81,9 @@ struct ModelTraffic {
     bool elementwise = false;   // one fused pass, gradient recomputed instead of stored
     int  data_streams = 0;      // model data streams per coordinate in the fused pass
     int  grad_track_streams = 5; // split path: gradient reads x, writes g; tracking reads z, g_old, g_new
+    int  method_streams = 2;     // the method's own count beyond x, z, packets: the remembered gradient read,
+                                 // the new one written (element-wise objective: its two data streams,
+                                 // the remembered gradient being recomputed)
 };
 
 int build_host_graph(const rfast_graph& g, int n, bool row_stochastic, HostGraph& out, std::string& err);

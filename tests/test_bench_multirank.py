@@ -68,3 +68,13 @@ def test_reference_arm_under_torchrun_rank0_only(repo_root):
     assert d["impl"] == "reference" and d["metric"] == "node_activations_per_s" and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
     assert d["n_gpus"] == 2 and d["config"]["workload"] == "ls_ring4"
+
+
+def test_gpus_flag_without_its_ranks_is_refused(repo_root):
+    """`--gpus 8` started as one plain process must not print an n_gpus = 1 line: it exits
+    non-zero and says how to launch the ranks."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, "bench.py", "--gpus", "8", "--steps", "1"], cwd=repo_root, env=env,
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "torch.distributed.run" in r.stderr
+    assert not any(ln.startswith("{") for ln in r.stdout.splitlines())

@@ -79,6 +79,15 @@ def test_diagnostics_match_the_oracle_state(rfast_lib, name, ov):
         assert d0["conservation_residual"] <= 1e-6 * max(d0["gradient_sum_max"], 1e-30)   # z^0 = g^0
         eng.run()
         d = eng.diagnostics()
+    # merit function of the non-convex analysis: the full gradient of F = sum_i f_i (every row
+    # of every shard) at the mean iterate, from the oracle's own models
+    m = make_model(wl)
+    if wl.model in ("quad_diag", "least_squares"):
+        gF = sum(m.grad(i, xbar, None) for i in range(wl.n))
+        want["full_gradient_norm"] = np.linalg.norm(gF)
+        want["merit"] = np.linalg.norm(gF) ** 2 + np.linalg.norm(X - xbar) ** 2
+    else:
+        assert np.isnan(d["full_gradient_norm"]) and np.isnan(d["merit"])
     for key, w in want.items():
         assert abs(d[key] - w) <= 1e-4 * max(w, 1e-6), (key, d[key], w)
     # Lemma 3 on the device state, relative to the gradients that are summed
@@ -109,6 +118,8 @@ def test_bounded_barrier_wait_reports_timeout_and_the_handle_recovers(rfast_lib)
         assert ei.value.code == ETIMEOUT and time.time() - t0 < 5.0
         eng.set_option(B.OPT_PHANTOM_ARRIVALS, 0)
         eng.reset()
+        # the reset has cleared the timeout: the state can be read before anything runs again
+        assert np.array_equal(eng.read(B.STATE_X), np.zeros((wl.n, wl.p), np.float32) if wl.x0 is None else wl.x0)
         eng.run()
         x = eng.read(B.STATE_X)
     assert np.linalg.norm(x - orc.X()) <= 1e-5 * np.linalg.norm(orc.X())

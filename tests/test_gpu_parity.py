@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 
 from conftest import has_cuda
+from forcing import assert_per_node as _per_node
 from oracle import from_workload, make_model, rel_l2, run_schedule
 from workloads import build_config
 
@@ -39,12 +40,14 @@ def _oracle(wl, K=None):
     return orc, ref0
 
 
-def _compare(eng, orc, ref0, tol=TOL):
+def _compare(eng, orc, ref0, tol=TOL, node_tol=None):
     from paper_2307_11617_b200 import binding as B
     x, y = eng.read(B.STATE_X), eng.read(B.STATE_Y)
     assert np.isfinite(x).all() and np.isfinite(y).all()
     ex, ey = rel_l2(x, orc.X(), ref0[0]), rel_l2(y, orc.Z(), ref0[1])
     assert ex <= tol and ey <= tol, (ex, ey)
+    _per_node(x, orc.X(), None, node_tol or tol, "x")
+    _per_node(y, orc.Z(), orc.G(), node_tol or tol, "y")
     g = eng.read(B.STATE_G_LAST)
     assert rel_l2(g, orc.G(), ref0[1]) <= 10 * tol
     if len(orc.rho):
@@ -118,7 +121,11 @@ def test_parity_in_every_tracker_arithmetic(rfast_lib, name, ov, level):
     with pkg.Engine(wl) as eng:
         eng.load_schedule(wl.schedule)
         eng.run()
-        _compare(eng, orc, ref0)
+        # fp32 running sums keep growing while the trackers do not: at levels 0 and 1 a receiver
+        # sees its in-neighbours' mass at the resolution of ulp(rho), which on the four-node
+        # least-squares problem (trackers several times smaller than the local gradients) costs a
+        # single node up to ~1.5e-5 of its tracker while the state as a whole stays inside 1e-5
+        _compare(eng, orc, ref0, node_tol=3e-5 if (name == "ls_ring4" and level < 2) else None)
         d = eng.diagnostics()
     if level == 2:                                   # Lemma 3 then holds to double-float accuracy
         assert d["conservation_residual"] <= 1e-9 * max(d["gradient_sum_max"], d["tracker_norm"])
@@ -321,6 +328,47 @@ def test_parity_on_general_digraphs(rfast_lib, name, ov, comp):
         d = eng.diagnostics()
     scale = np.abs(orc.G()).sum(axis=0).max()
     assert d["conservation_residual"] <= 2e-5 * scale
+
+
+@pytest.mark.parametrize("name,ov", [
+    ("logistic_tree1024", dict(n=28, p=9000, rows=8, K=40, batch=4, nnz=60)),
+    ("softmax_exp16", dict(n=28, F=40, C=5, rows=32, K=40, batch=8)),
+], ids=["logistic", "softmax"])
+def test_parity_with_many_in_neighbours(rfast_lib, name, ov):
+    """A hub: every node pushes to node 0 over G_C (in-degree n - 1 = 27 there, up to 27 rows of
+    news in one activation -- more than the sparse-logistic pass lists for prefetching, which
+    must not change what is summed) and pulls from node 0 over G_R, plus the ring so that
+    other nodes have in- and out-neighbours too."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    from workloads import activation_bernoulli, graph_from_edges, make_schedule
+    wl = build_config(name, seed=13, **ov)
+    n = wl.n
+    rng = np.random.default_rng(14)
+    ring = {(i, (i + 1) % n) for i in range(n)}
+    wl.G_R = graph_from_edges(n, ring | {(0, i) for i in range(1, n)}, "row")
+    wl.G_C = graph_from_edges(n, ring | {(i, 0) for i in range(1, n)}, "col")
+    wl.schedule = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, wl.schedule.K, 0.7, rng), 0.1, 2,
+                                rng, batch=wl.batch, rows_per_node=wl.rows)
+    orc, ref0 = _oracle(wl)
+    # the hub really consumes more than 16 newer running sums in one activation
+    s, news = wl.schedule, 0
+    used = np.asarray(orc.used_tau_rho)
+    pos, last = 0, {}
+    for ev in range(s.n_events):
+        i = int(s.act_node[ev])
+        deg = int(wl.G_C.rowptr[i + 1] - wl.G_C.rowptr[i])
+        cur = used[pos:pos + deg]
+        if i == 0:
+            news = max(news, int((cur > last.get(0, np.zeros(deg, int))).sum()))
+            last[0] = cur
+        pos += deg
+    assert news > 16, news
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(s)
+        eng.run()
+        _compare(eng, orc, ref0)
+        assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
 
 
 def test_coordinate_shards_reproduce_the_whole_bit_for_bit(rfast_lib):

@@ -386,3 +386,20 @@ def test_oracle_reproduces_its_frozen_output_on_config_1(repo_root):
     assert np.abs(orc.X() - x).max() <= 1e-13 * np.abs(x).max()
     assert np.abs(orc.Z() - z).max() <= 1e-13 * np.abs(z).max()
     assert st.tolist() == orc.t + orc.tau_v + orc.tau_rho
+
+
+def test_rel_l2_metric_known_vectors_and_floor():
+    """The parity metric itself: ||a - ref||_F / max(||ref||_F, 1e-3 * ref0_norm)."""
+    from oracle import rel_l2
+    ref = np.array([[3.0, 4.0], [0.0, 0.0]])                     # Frobenius norm 5
+    a = ref + np.array([[0.0, 0.0], [0.3, 0.4]])                  # error norm 0.5
+    assert rel_l2(a, ref) == pytest.approx(0.1, rel=1e-15)
+    assert rel_l2(ref, ref) == 0.0
+    # the floor takes over once the reference has shrunk below 1e-3 of its initial norm
+    tiny = ref * 1e-6                                             # norm 5e-6
+    assert rel_l2(tiny + 1e-6, tiny, ref0_norm=100.0) == pytest.approx(2e-6 / 0.1, rel=1e-12)
+    assert rel_l2(tiny + 1e-6, tiny, ref0_norm=1e-3) == pytest.approx(2e-6 / 5e-6, rel=1e-12)
+    # a vanished reference without a floor does not divide by zero
+    assert np.isfinite(rel_l2(np.ones(3), np.zeros(3)))
+    # float32 input is measured in double
+    assert rel_l2(np.float32([1.0, 1.0]), np.array([1.0, 1.0 + 1e-12])) == pytest.approx(1e-12 / np.sqrt(2.0 + 2e-12), rel=1e-3)

@@ -60,6 +60,10 @@ def test_static_gradient_matches_handle_path_twice(rfast_lib):
         got = d_grad.cpu().numpy()
         assert np.isfinite(got).all()
         assert np.linalg.norm(got - want) <= TOL * np.linalg.norm(want)
+        # and directly against the CPU oracle's definition of the same gradient
+        from oracle.models import LeastSquares
+        ref = LeastSquares([feat], [target], l2).grad(0, x.astype(np.float64))
+        assert np.linalg.norm(got - ref) <= TOL * np.linalg.norm(ref)
 
 
 def test_static_gradient_rejects_oversize(rfast_lib):
