@@ -289,8 +289,22 @@ int64_t rfast_query(rfast_ctx* ctx, int what);
  *   RFAST_OPT_WAIT_LIMIT_MS     bound of every device-side barrier wait, 1..60000 (default 2000).
  *   RFAST_OPT_PHANTOM_ARRIVALS  failure injection for tests, made on the host: the grid barrier
  *                         expects this many arrivals that nobody makes, so its bounded wait runs
- *                         out and the timeout path is exercised (default 0). */
-enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1, RFAST_OPT_WAIT_LIMIT_MS = 2, RFAST_OPT_PHANTOM_ARRIVALS = 3 };
+ *                         out and the timeout path is exercised (default 0).
+ *   RFAST_OPT_ONE_PASS    sparse-logistic objective.  1 (default): an activation runs as one
+ *                         thread-block cluster whose CTAs keep their slices of the new x and of z
+ *                         in shared memory between the mixing step, the sparse dot products and
+ *                         the tracking step, so every vector crosses HBM once (taken when a
+ *                         cluster of at most 8 CTAs can hold 2 p floats and the batch is at most
+ *                         64 rows; otherwise, or with 0, three kernels per round).  The two paths
+ *                         add the sparse dot products up in different orders: they agree to
+ *                         rounding, each of them bit for bit from run to run.  To be set before
+ *                         rfast_load_schedule (RFAST_ESTATE afterwards).
+ *   RFAST_OPT_CLUSTER_SIZE  CTAs per activation on that path: 0 (default) = the smallest of 1, 2,
+ *                         4, 8 that fits; RFAST_EINVAL if the given size does not fit.  The
+ *                         partial dot products are added per CTA, so results agree to rounding
+ *                         across sizes.  To be set before rfast_load_schedule. */
+enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1, RFAST_OPT_WAIT_LIMIT_MS = 2, RFAST_OPT_PHANTOM_ARRIVALS = 3,
+       RFAST_OPT_ONE_PASS = 4, RFAST_OPT_CLUSTER_SIZE = 5 };
 int rfast_set_option(rfast_ctx* ctx, int option, int64_t value);
 
 /* Waits for the handle's stream; reports a pending asynchronous error. */

@@ -278,7 +278,7 @@ def rfast_compile_host(wl, s):
             "streams": int(counts[3])}
 
 
-OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS = 0, 1, 2, 3
+OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS, OPT_ONE_PASS, OPT_CLUSTER_SIZE = 0, 1, 2, 3, 4, 5
 
 
 def rfast_set_option(handle, option: int, value: int) -> None:

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "logit_fused.cuh"
 #include "persist.cuh"
 #include "rfast_internal.h"
 
@@ -77,6 +78,11 @@ struct rfast_ctx {
     unsigned int* d_bar = nullptr;
     int* d_pstatus = nullptr;
     int max_round_events = 0;
+    // sparse logistic: one cluster per activation, one pass over HBM (logit_fused.cuh)
+    bool opt_fused = true;
+    int fused_cluster = 0, fused_ranges = 0;      // cluster size (0: the path is not available), ranges per CTA
+    int fused_threads = 512, fused_stash = 0;
+    size_t fused_smem = 0;
     int round = 0;
     int64_t launches = 0;
     // recorded span of rounds [graph_r0, graph_r1): a sequence of graphs of about a thousand kernels each
@@ -146,7 +152,7 @@ void free_schedule(rfast_ctx* c) {
     c->has_sched = false;
 }
 
-ModelTraffic traffic_of(int model, bool compensated) {
+ModelTraffic traffic_of(int model, bool compensated, bool one_pass = false) {
     ModelTraffic mt;
     mt.elementwise = (model == RFAST_MODEL_QUAD_DIAG);
     mt.data_streams = (mt.elementwise ? 2 : 0) + (compensated ? 2 : 0);
@@ -155,6 +161,7 @@ ModelTraffic traffic_of(int model, bool compensated) {
     // tracking reads z, g_old, g_new (5).  z's write and the packets are counted elsewhere.
     mt.grad_track_streams = (model == RFAST_MODEL_LOGISTIC_SPARSE ? 4 : 5) + (mt.elementwise ? 0 : (compensated ? 2 : 0));
     mt.method_streams = 2;    // element-wise: d and b, the remembered gradient recomputed; others: g_old read, g_new written
+    if (one_pass) mt.grad_track_streams = 2 + (compensated ? 2 : 0);   // nothing is read twice
     return mt;
 }
 
@@ -221,6 +228,82 @@ int launch_logit_track(rfast_ctx* ctx, const RoundArgs& a, const EvDesc* d_ev, i
     return RFAST_OK;
 }
 
+const void* logit_fused_fn(bool comp, int threads) {
+    if (threads == 512) return comp ? (const void*)k_logit_fused<true, 512> : (const void*)k_logit_fused<false, 512>;
+    return comp ? (const void*)k_logit_fused<true, 1024> : (const void*)k_logit_fused<false, 1024>;
+}
+
+// Sparse logistic, one pass: the smallest cluster (1, 2, 4, 8 CTAs) whose CTAs can each keep
+// their slice of x and z in shared memory, first with 512 threads per CTA and half of an SM's
+// shared memory (two CTAs of different activations share an SM, one streams while the other
+// computes), else with 1024 threads and the whole of it.  want > 0 asks for that cluster size.
+bool plan_logit_fused(rfast_ctx* ctx, int want) {
+    ctx->fused_cluster = 0;
+    if (ctx->model != RFAST_MODEL_LOGISTIC_SPARSE || ctx->batch > kFusedMaxBatch || ctx->batch < 1) return false;
+    int dev = 0, max_smem = 0, sm_smem = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cudaDeviceGetAttribute(&sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    int64_t rows_nnz = 0;
+    cudaMemcpy(&rows_nnz, ctx->sp_ptr + (size_t)ctx->n * ctx->rows, sizeof(int64_t), cudaMemcpyDeviceToHost);
+    const double nnz_per_batch = (double)rows_nnz / std::max<int64_t>(1, (int64_t)ctx->n * ctx->rows) * ctx->batch;
+    for (int threads : {512, 1024}) {
+        const int64_t budget = threads == 512 ? std::min<int64_t>(max_smem, sm_smem / 2 - 1024) : max_smem;
+        for (int cs = 1; cs <= 8; cs *= 2) {
+            if (want > 0 && cs != want) continue;
+            const int R = (ctx->sp_ranges + cs - 1) / cs;
+            if (R * (kLogitRange / 4) > kFusedPerThread * threads) continue;           // float4 of a slice per thread
+            const int64_t fixed = (int64_t)2 * R * kLogitRange * sizeof(float) + 4096;   // slices + the kernel's static arrays
+            if (fixed > budget) continue;
+            // the sampled rows' entries of a slice are kept on chip as far as they fit: room for 1.5 x the mean
+            const int64_t want_stash = (int64_t)(1.5 * nnz_per_batch / cs) + 64;
+            const int stash = (int)(std::max<int64_t>(0, std::min<int64_t>(want_stash, (budget - fixed) / 6)) / 8 * 8);
+            const size_t smem = (size_t)2 * R * kLogitRange * sizeof(float) + (size_t)stash * 6;
+            const void* fn = logit_fused_fn(ctx->compensated, threads);
+            if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); continue; }
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3(cs, 1, 1); cfg.blockDim = dim3(threads, 1, 1); cfg.dynamicSmemBytes = smem;
+            cudaLaunchAttribute at{};
+            at.id = cudaLaunchAttributeClusterDimension;
+            at.val.clusterDim.x = cs; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+            cfg.attrs = &at; cfg.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, fn, &cfg) != cudaSuccess || nclusters < 1) { cudaGetLastError(); continue; }
+            ctx->fused_cluster = cs; ctx->fused_ranges = R; ctx->fused_smem = smem; ctx->fused_stash = stash;
+            ctx->fused_threads = threads;
+            return true;
+        }
+    }
+    return false;
+}
+
+int launch_logit_fused(rfast_ctx* ctx, const RoundArgs& a, const EvDesc* d_ev, int nev) {
+    LogitFusedArgs P{};
+    P.a = a; P.a.ev = d_ev;
+    P.g = grad_args(ctx, d_ev);
+    P.range_ptr = ctx->sp_tile_ptr; P.nranges = ctx->sp_ranges;
+    P.sp_col = ctx->sp_col; P.sp_val = ctx->sp_val; P.label = ctx->label;
+    P.ranges_per_cta = ctx->fused_ranges;
+    P.stash_cap = ctx->fused_stash;
+    P.status = ctx->d_pstatus; P.limit_ns = (unsigned long long)ctx->opt_wait_limit_ms * 1000000ull;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(ctx->fused_cluster, nev, 1); cfg.blockDim = dim3(ctx->fused_threads, 1, 1);
+    cfg.dynamicSmemBytes = ctx->fused_smem; cfg.stream = ctx->stream;
+    cudaLaunchAttribute at{};
+    at.id = cudaLaunchAttributeClusterDimension;
+    at.val.clusterDim.x = ctx->fused_cluster; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    cfg.attrs = &at; cfg.numAttrs = 1;
+    if (ctx->fused_threads == 512) {
+        if (ctx->compensated) CK(cudaLaunchKernelEx(&cfg, k_logit_fused<true, 512>, P));
+        else CK(cudaLaunchKernelEx(&cfg, k_logit_fused<false, 512>, P));
+    } else {
+        if (ctx->compensated) CK(cudaLaunchKernelEx(&cfg, k_logit_fused<true, 1024>, P));
+        else CK(cudaLaunchKernelEx(&cfg, k_logit_fused<false, 1024>, P));
+    }
+    ctx->launches += 1;
+    return RFAST_OK;
+}
+
 // sample gradients of `nev` events (descriptors on the device) into gbuf[par^1]
 int launch_gradients(rfast_ctx* ctx, const EvDesc* d_ev, int nev) {
     GradArgs g = grad_args(ctx, d_ev);
@@ -283,7 +366,8 @@ int check_device_status(rfast_ctx* ctx) {
         int st = 0;
         CK(cudaMemcpyAsync(&st, ctx->d_pstatus, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
         CK(cudaStreamSynchronize(ctx->stream));
-        if (st != 0) return set_err(ctx, RFAST_ETIMEOUT, "a grid barrier of the persistent kernel ran out of time");
+        if (st != 0) return set_err(ctx, RFAST_ETIMEOUT, st == kFusedTimeout ? "the bulk copies of the one-pass kernel did not land in time"
+                                                                              : "a grid barrier of the persistent kernel ran out of time");
     }
     if (ctx->mlp) {
         const int st = mlp_plan_status(ctx->mlp, ctx->stream);
@@ -456,6 +540,7 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
         ctx->dev_bytes += mb;
     }
     CK(cudaStreamSynchronize(ctx->stream));    // the caller's arrays may go away now
+    plan_logit_fused(ctx, 0);
     guard.c = nullptr;
     *out = ctx;
     return RFAST_OK;
@@ -470,7 +555,8 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     CK(cudaStreamSynchronize(ctx->stream));
     Compiled comp;
     std::string err;
-    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated), ctx->buckets, comp, err);
+    const bool one_pass = ctx->model == RFAST_MODEL_LOGISTIC_SPARSE && ctx->opt_fused && ctx->fused_cluster > 0;
+    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated, one_pass), ctx->buckets, comp, err);
     if (rc != RFAST_OK) return set_err(ctx, rc, err);
     free_schedule(ctx);
     ctx->alpha_round.clear();
@@ -596,6 +682,9 @@ static int issue_rounds(rfast_ctx* ctx, int r0, int r1) {
             if (ctx->compensated) k_fused_quad<1, true><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             else k_fused_quad<1, false><<<tile_grid(a.n4, 1, nev), kThreads, 0, ctx->stream>>>(a, ctx->quad_d, ctx->quad_b);
             ctx->launches += 1;
+        } else if (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE && ctx->opt_fused && ctx->fused_cluster > 0) {
+            int rc = launch_logit_fused(ctx, a, a.ev, nev);
+            if (rc != RFAST_OK) return rc;
         } else {
             const int64_t gplane = (int64_t)ctx->n * ctx->stride;
             const dim3 tg = tile_grid(a.n4, 1, nev);
@@ -712,6 +801,16 @@ int rfast_set_option(rfast_ctx* ctx, int option, int64_t value) {
         case RFAST_OPT_WAIT_LIMIT_MS:
             if (value < 1 || value > 60000) return set_err(ctx, RFAST_EINVAL, "wait limit must be 1..60000 ms");
             ctx->opt_wait_limit_ms = value; return RFAST_OK;
+        case RFAST_OPT_ONE_PASS:
+        case RFAST_OPT_CLUSTER_SIZE:
+            if (ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "this option must be set before a schedule is loaded (the byte accounting follows it)");
+            if (option == RFAST_OPT_ONE_PASS) { ctx->opt_fused = value != 0; return RFAST_OK; }
+            if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return set_err(ctx, RFAST_EINVAL, "cluster size must be 0 (automatic), 1, 2, 4 or 8");
+            if (!plan_logit_fused(ctx, (int)value)) {
+                plan_logit_fused(ctx, 0);
+                if (value != 0) return set_err(ctx, RFAST_EINVAL, "the problem does not fit a cluster of that size");
+            }
+            return RFAST_OK;
         case RFAST_OPT_PHANTOM_ARRIVALS:
             if (value < 0 || value > 1024) return set_err(ctx, RFAST_EINVAL, "phantom arrivals must be 0..1024");
             ctx->opt_phantom = value; return RFAST_OK;

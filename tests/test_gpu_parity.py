@@ -371,6 +371,50 @@ def test_parity_with_many_in_neighbours(rfast_lib, name, ov):
         assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
 
 
+@pytest.mark.parametrize("level", [0, 1], ids=["plain", "two-float tracker"])
+@pytest.mark.parametrize("cluster", [-1, 1, 2, 4, 8], ids=["three kernels", "1 CTA", "2 CTAs", "4 CTAs", "8 CTAs"])
+def test_sparse_logistic_one_pass_in_every_cluster_size(rfast_lib, cluster, level):
+    """The sparse-logistic activation as one cluster per activation (slices of x and z kept in
+    shared memory, partial dot products exchanged between the CTAs), in every cluster size, and
+    the three-kernel path it replaces: each against the oracle, each bit-identical on a rerun.
+    p = 9000 gives 18 ranges of 512 coordinates: ragged slices in every size, an empty slice never."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("logistic_tree1024", seed=5, n=48, p=9000, rows=8, K=40, batch=4, nnz=60)
+    wl.compensated = level
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        if cluster < 0:
+            eng.set_option(B.OPT_ONE_PASS, 0)
+        else:
+            eng.set_option(B.OPT_CLUSTER_SIZE, cluster)
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        x1, y1 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        assert eng.query(B.Q_BYTES_TOTAL) == eng.query(B.Q_METHOD_BYTES_TOTAL) + (0 if cluster >= 0 else 2 * 4 * wl.p * wl.schedule.n_events) \
+            + 2 * level * 4 * wl.p * wl.schedule.n_events
+        eng.reset()
+        eng.run()
+        assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
+        with pytest.raises(B.RFastError):                       # the byte accounting follows the option
+            eng.set_option(B.OPT_ONE_PASS, 0)
+
+
+def test_sparse_logistic_one_pass_with_an_empty_slice_and_a_large_batch(rfast_lib):
+    """p = 1500 is three ranges: in a cluster of four the last CTA owns nothing and still meets
+    its peers at the barriers; batch 40 makes a warp take more than one sampled row."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("logistic_tree1024", seed=6, n=24, p=1500, rows=64, K=25, batch=40, nnz=30)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_CLUSTER_SIZE, 4)
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+
+
 def test_coordinate_shards_reproduce_the_whole_bit_for_bit(rfast_lib):
     """The element-wise problem split by coordinate (what `bench.py --shard coords` gives each
     GPU) needs no exchange: three ragged slices run one after the other on this GPU give, side
