@@ -289,7 +289,9 @@ int64_t rfast_query(rfast_ctx* ctx, int what);
  *   RFAST_OPT_WAIT_LIMIT_MS     bound of every device-side barrier wait, 1..60000 (default 2000).
  *   RFAST_OPT_PHANTOM_ARRIVALS  failure injection for tests, made on the host: the grid barrier
  *                         expects this many arrivals that nobody makes, so its bounded wait runs
- *                         out and the timeout path is exercised (default 0).
+ *                         out and the timeout path is exercised (default 0).  The one-pass
+ *                         sparse-logistic kernel takes the same option: its copy barrier then
+ *                         expects 16 bytes per unit that nobody delivers.
  *   RFAST_OPT_ONE_PASS    sparse-logistic objective.  1 (default): an activation runs as one
  *                         thread-block cluster whose CTAs keep their slices of the new x and of z
  *                         in shared memory between the mixing step, the sparse dot products and

@@ -286,6 +286,7 @@ int launch_logit_fused(rfast_ctx* ctx, const RoundArgs& a, const EvDesc* d_ev, i
     P.ranges_per_cta = ctx->fused_ranges;
     P.stash_cap = ctx->fused_stash;
     P.status = ctx->d_pstatus; P.limit_ns = (unsigned long long)ctx->opt_wait_limit_ms * 1000000ull;
+    P.phantom_bytes = (unsigned int)ctx->opt_phantom * 16u;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(ctx->fused_cluster, nev, 1); cfg.blockDim = dim3(ctx->fused_threads, 1, 1);
     cfg.dynamicSmemBytes = ctx->fused_smem; cfg.stream = ctx->stream;

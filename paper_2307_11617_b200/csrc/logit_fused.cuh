@@ -44,6 +44,9 @@ struct LogitFusedArgs {
     int stash_cap;                     // entries of the sampled rows a CTA can keep in shared memory
     int* status;                       // 0, or kFusedTimeout
     unsigned long long limit_ns;       // bound of the wait for the bulk copies
+    unsigned int phantom_bytes;        // bytes the mbarrier expects beyond what is copied (0 in normal use; a
+                                       // host-side failure-injection hook: nobody delivers them, so the bounded
+                                       // wait runs out and the timeout path is exercised)
 };
 
 __device__ __forceinline__ uint32_t fused_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -106,7 +109,7 @@ k_logit_fused(LogitFusedArgs P) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         s_ok = 1;
         if (slice_bytes) {
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fused_smem_u32(&s_bar)), "r"(2u * slice_bytes) : "memory");
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(fused_smem_u32(&s_bar)), "r"(2u * slice_bytes + P.phantom_bytes) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(fused_smem_u32(xs)), "l"(xr + (int64_t)lo4 * 4), "r"(slice_bytes), "r"(fused_smem_u32(&s_bar)) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

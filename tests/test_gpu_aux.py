@@ -123,3 +123,33 @@ def test_bounded_barrier_wait_reports_timeout_and_the_handle_recovers(rfast_lib)
         eng.run()
         x = eng.read(B.STATE_X)
     assert np.linalg.norm(x - orc.X()) <= 1e-5 * np.linalg.norm(orc.X())
+
+
+def test_bounded_copy_wait_of_the_one_pass_kernel_reports_timeout_and_recovers(rfast_lib):
+    """The same for the sparse-logistic cluster kernel: its mbarrier is told (on the host) to
+    expect bytes that no copy delivers; every CTA's bounded wait runs out, the CTAs still meet
+    at their cluster barriers and return, the next synchronising call reports RFAST_ETIMEOUT,
+    and after a reset the same handle runs the schedule correctly.  Nothing faults or hangs."""
+    import time
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    from paper_2307_11617_b200.binding import ETIMEOUT, RFastError
+    wl = build_config("logistic_tree1024", seed=2, n=24, p=9000, rows=8, K=6, batch=4, nnz=60)
+    orc = from_workload(wl, make_model(wl).grad)
+    Bs, s = wl.batch, wl.schedule
+    orc.init_gradients([s.batch_idx[i * Bs:(i + 1) * Bs] for i in range(wl.n)])
+    run_schedule(orc, s)
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_CLUSTER_SIZE, 2)
+        eng.set_option(B.OPT_WAIT_LIMIT_MS, 100)
+        eng.set_option(B.OPT_PHANTOM_ARRIVALS, 1)
+        eng.load_schedule(s)
+        t0 = time.time()
+        with pytest.raises(RFastError) as ei:
+            eng.run(1)
+        assert ei.value.code == ETIMEOUT and time.time() - t0 < 10.0
+        eng.set_option(B.OPT_PHANTOM_ARRIVALS, 0)
+        eng.reset()
+        eng.run()
+        x = eng.read(B.STATE_X)
+    assert np.linalg.norm(x - orc.X()) <= 1e-5 * np.linalg.norm(orc.X())

@@ -371,7 +371,7 @@ def test_parity_with_many_in_neighbours(rfast_lib, name, ov):
         assert eng.read(B.STATE_USED_TAU_RHO).tolist() == orc.used_tau_rho
 
 
-@pytest.mark.parametrize("level", [0, 1], ids=["plain", "two-float tracker"])
+@pytest.mark.parametrize("level", [0, 1, 2], ids=["plain", "two-float tracker", "two-float tracker and sums"])
 @pytest.mark.parametrize("cluster", [-1, 1, 2, 4, 8], ids=["three kernels", "1 CTA", "2 CTAs", "4 CTAs", "8 CTAs"])
 def test_sparse_logistic_one_pass_in_every_cluster_size(rfast_lib, cluster, level):
     """The sparse-logistic activation as one cluster per activation (slices of x and z kept in
@@ -393,7 +393,7 @@ def test_sparse_logistic_one_pass_in_every_cluster_size(rfast_lib, cluster, leve
         _compare(eng, orc, ref0)
         x1, y1 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
         assert eng.query(B.Q_BYTES_TOTAL) == eng.query(B.Q_METHOD_BYTES_TOTAL) + (0 if cluster >= 0 else 2 * 4 * wl.p * wl.schedule.n_events) \
-            + 2 * level * 4 * wl.p * wl.schedule.n_events
+            + 2 * min(level, 1) * 4 * wl.p * wl.schedule.n_events
         eng.reset()
         eng.run()
         assert np.array_equal(x1, eng.read(B.STATE_X)) and np.array_equal(y1, eng.read(B.STATE_Y))
