@@ -187,7 +187,7 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def measure_config(name, args, steps, world, rank, local, cpu_budget_s):
+def measure_config(name, args, steps, world, rank, local, cpu_budget_s, stream=None):
     """One workload on this rank's GPU: timed passes (CUDA events on the engine's stream), the
     end-to-end passes through the C ABI with host buffers, the clocks seen meanwhile, the
     roofline figures and, on rank 0, the oracle on a bounded sample.  Returns the pieces of a
@@ -205,7 +205,8 @@ def measure_config(name, args, steps, world, rank, local, cpu_budget_s):
         from workloads import shard_coordinates
         wl = shard_coordinates(wl_full, rank, world)     # same schedule, this rank's slice of every vector
     t_gen = time.perf_counter() - t_gen
-    stream = torch.cuda.Stream()
+    if stream is None:
+        stream = torch.cuda.Stream()
     t_create = time.perf_counter()
     eng = pkg.Engine(wl, stream.cuda_stream)
     t_create = time.perf_counter() - t_create
@@ -374,11 +375,12 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    # The small, launch-bound configurations are measured before the large one: in a process that
-    # has held and freed the 24 GB of the bandwidth configuration their device allocations land
-    # scattered over the freed range and the same kernels run 9 % slower (softmax_exp16: 92.9
-    # against 84.8 ms per pass, measured both ways in one process); a process of their own gives
-    # the figure measured first here.
+    # One stream for every configuration: torch hands out its pooled streams in turn, and the
+    # launch-bound configurations ran 9 % slower on every second one of them (softmax_exp16: 93.3
+    # against 85.7 ms per pass, three handles in one process on three streams: 85.7, 93.3, 85.7;
+    # on one stream: 85.7 every time).  The small configurations are measured first, the large
+    # one last.
+    stream = torch.cuda.Stream()
     others = {}
     want_others = args.others == "all" or (args.others == "auto" and args.config == "quad_tree64" and not args.small
                                            and args.shard == "replicas")
@@ -386,10 +388,10 @@ def main():
         from workloads import CONFIG_NAMES
         for nm in CONFIG_NAMES:
             if nm != args.config:
-                r = measure_config(nm, args, 3, world, rank, local, cpu_budget_s=4.0)
+                r = measure_config(nm, args, 3, world, rank, local, cpu_budget_s=4.0, stream=stream)
                 r["metric"], r["unit"] = METRIC, UNIT
                 others[nm] = r
-    main_rec = measure_config(args.config, args, args.steps, world, rank, local, cpu_budget_s=15.0)
+    main_rec = measure_config(args.config, args, args.steps, world, rank, local, cpu_budget_s=15.0, stream=stream)
 
     if rank == 0:
         line = {"metric": METRIC, "value": main_rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
