@@ -566,11 +566,22 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
             if (!(s->alpha_round[r] == s->alpha_round[r])) return set_err(ctx, RFAST_ESCHED, "schedule: alpha_round holds a NaN");
         ctx->alpha_round.assign(s->alpha_round, s->alpha_round + s->K);
     }
-    {   // FNV-1a over the raw arrays: a checkpoint is only valid for this very schedule
+    {   // hash of the raw arrays: a checkpoint is only valid for this very schedule.  Eight bytes
+        // per step (multiply and fold), the tail byte by byte: the arrays run to tens of megabytes
+        // and this sits in every rfast_load_schedule
         uint64_t hsh = 1469598103934665603ull;
         auto mix = [&](const void* ptr, size_t bytes) {
             const unsigned char* q = (const unsigned char*)ptr;
-            for (size_t k = 0; k < bytes; ++k) { hsh ^= q[k]; hsh *= 1099511628211ull; }
+            size_t k = 0;
+            for (; k + 8 <= bytes; k += 8) {
+                uint64_t w;
+                std::memcpy(&w, q + k, 8);
+                hsh = (hsh ^ w) * 0x9E3779B97F4A7C15ull;
+                hsh ^= hsh >> 29;
+            }
+            for (; k < bytes; ++k) { hsh ^= q[k]; hsh *= 1099511628211ull; }
+            hsh ^= bytes;
+            hsh *= 1099511628211ull;
         };
         mix(&s->K, sizeof s->K);
         mix(s->act_ptr, (size_t)(s->K + 1) * sizeof(int32_t));
