@@ -133,6 +133,17 @@ def build_workload(name, small=False, tracker="sums"):
     return build_config(name, seed=0, tracker=1 if tracker == "buckets" else 0, **ov)
 
 
+def workload_config(wl, full_p, args, world, sharded=False):
+    """What names the workload and how it was timed: the same dict in both arms."""
+    return {"workload": wl.name, "n": wl.n, "p": full_p, "rounds": wl.schedule.K,
+            "activations_per_step": int(wl.schedule.n_events), "small": bool(args.small), "tracker": args.tracker,
+            # the arithmetic the workload asks of an fp32 engine for its tracker (the oracle is fp64 throughout)
+            "tracker_arithmetic": {0: "plain fp32", 1: "two-float tracker", 2: "two-float tracker and running sums"}[int(wl.compensated)],
+            "l2": "inputs larger than L2" if wl.n * full_p * 4 > 126e6 else "state fits L2",
+            "reset_between_steps": "untimed",
+            "parallelism": f"coordinate shards x{world}" if sharded else f"replicas x{world}"}
+
+
 def oracle_sample(wl, budget_s=15.0):
     """Times the oracle as it stands on a bounded sample of the workload and returns
     (activations/s scaled to the full workload, description, seconds spent)."""
@@ -181,7 +192,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * ev / v,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl.name, "n": wl.n, "p": wl.p, "rounds": wl.schedule.K},
+            "data": "synthetic", "config": workload_config(wl, wl.p, args, args.gpus),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -280,12 +291,7 @@ def measure_config(name, args, steps, world, rank, local, cpu_budget_s, stream=N
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc, "seconds": dt}
 
     rec = {"value": value, "ms_per_step": ms_step, "steps": steps, "warmup": warm,
-           "config": {"workload": wl.name, "n": wl.n, "p": wl_full.p, "rounds": K_rounds,
-                      "activations_per_step": events, "small": bool(args.small), "tracker": args.tracker,
-                      "tracker_arithmetic": {0: "plain fp32", 1: "two-float tracker", 2: "two-float tracker and running sums"}[int(wl.compensated)],
-                      "l2": "inputs larger than L2" if wl.n * wl.p * 4 > 126e6 else "state fits L2",
-                      "reset_between_steps": "untimed",
-                      "parallelism": f"coordinate shards x{world}" if sharded else f"replicas x{world}"},
+           "config": workload_config(wl, wl_full.p, args, world, sharded),
            "scaling": "strong" if sharded else "weak",
            "param_updates_per_s": value * wl_full.p, "gpu_launches": int(launches),
            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
