@@ -415,6 +415,24 @@ def test_sparse_logistic_one_pass_with_an_empty_slice_and_a_large_batch(rfast_li
         _compare(eng, orc, ref0)
 
 
+@pytest.mark.parametrize("p,one_pass", [(200_003, True), (300_001, False)], ids=["1024-thread CTAs", "too large: three kernels"])
+def test_sparse_logistic_large_dimension_paths(rfast_lib, p, one_pass):
+    """p = 200,003 does not fit eight 512-thread CTAs (two per SM) any more and takes the
+    1024-thread variant of the one-pass kernel (49 ranges per CTA, 200 KB of slices); p = 300,001
+    does not fit a cluster of eight at all and falls back to three kernels per round.  Which path
+    ran shows in the byte accounting."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("logistic_tree1024", seed=7, n=8, p=p, rows=8, K=10, batch=4, nnz=300)
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        extra = eng.query(B.Q_BYTES_TOTAL) - eng.query(B.Q_METHOD_BYTES_TOTAL)
+        assert (extra == 0) == one_pass
+
+
 def test_coordinate_shards_reproduce_the_whole_bit_for_bit(rfast_lib):
     """The element-wise problem split by coordinate (what `bench.py --shard coords` gives each
     GPU) needs no exchange: three ragged slices run one after the other on this GPU give, side
