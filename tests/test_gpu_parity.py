@@ -433,6 +433,31 @@ def test_sparse_logistic_large_dimension_paths(rfast_lib, p, one_pass):
         assert (extra == 0) == one_pass
 
 
+def test_sparse_logistic_one_pass_with_more_entries_than_it_can_keep(rfast_lib):
+    """The one-pass kernel keeps the sampled rows' entries of a slice in shared memory between the
+    dot products and the gradient assembly, sized for 1.5 x the mean row; what does not fit is
+    read from global memory again.  Here half of the nodes hold rows forty times denser than the
+    other half, so their slices overflow the store and the second source is exercised."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("logistic_tree1024", seed=9, n=8, p=9000, rows=8, K=30, batch=4, nnz=400)
+    d = wl.data
+    ptr, col, val = d["sp_rowptr"], d["sp_col"], d["sp_val"]
+    keep = np.ones(len(col), bool)
+    for r in range(4 * wl.rows):                              # nodes 0..3: ten entries per row
+        keep[ptr[r] + 10:ptr[r + 1]] = False
+    lens = np.array([keep[ptr[r]:ptr[r + 1]].sum() for r in range(len(ptr) - 1)])
+    wl.data = dict(d, sp_rowptr=np.concatenate([[0], np.cumsum(lens)]).astype(np.int64), sp_col=col[keep], sp_val=val[keep])
+    assert lens.max() >= 30 * lens.min()
+    orc, ref0 = _oracle(wl)
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_CLUSTER_SIZE, 2)
+        eng.load_schedule(wl.schedule)
+        eng.run()
+        _compare(eng, orc, ref0)
+        assert eng.query(B.Q_BYTES_TOTAL) == eng.query(B.Q_METHOD_BYTES_TOTAL)     # the one-pass path ran
+
+
 def test_coordinate_shards_reproduce_the_whole_bit_for_bit(rfast_lib):
     """The element-wise problem split by coordinate (what `bench.py --shard coords` gives each
     GPU) needs no exchange: three ragged slices run one after the other on this GPU give, side
