@@ -40,6 +40,28 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def read_heavy_copy_peak(n_elems=1 << 28):
+    """Context for a roofline fraction above 1: the box's denominator is a plain copy (one read per
+    write); the fused kernel reads about twice what it writes.  This times c = a + b over fp32
+    arrays far larger than L2 (two reads per write, a library element-wise kernel, best of 5) and
+    returns GB/s of the bytes it must move."""
+    import torch
+    a = torch.empty(n_elems, dtype=torch.float32, device="cuda").normal_()
+    b = torch.empty_like(a).normal_()
+    c = torch.empty_like(a)
+    best = 0.0
+    for _ in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.add(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, 3 * 4 * n_elems / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del a, b, c
+    torch.cuda.empty_cache()
+    return best
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -285,6 +307,13 @@ def measure_config(name, args, steps, world, rank, local, cpu_budget_s, stream=N
                 if fused and args.tracker == "sums" and not sharded else None,   # the counters were taken on that workload
                 "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
 
+    if fused and not args.small:
+        try:
+            rh = read_heavy_copy_peak()
+            roofline["read_heavy_copy"] = {"what": "c = a + b over 3 x 1 GiB of fp32 (two reads per write), measured in this run",
+                                           "GB/s": rh, "frac": achieved / rh}
+        except Exception as exc:                               # context only: never fails the run
+            roofline["read_heavy_copy"] = {"error": str(exc)[:200]}
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
         v, desc, dt = oracle_sample(wl_full, budget_s=cpu_budget_s)   # the unsharded workload
