@@ -11,6 +11,7 @@
 #include <climits>
 #include <cmath>
 #include <cstdio>
+#include <thread>
 
 #include "rfast_internal.h"
 
@@ -115,14 +116,40 @@ int check_roots(const HostGraph& R, const HostGraph& C, int root, std::string& e
 namespace {
 struct Pend { int arrival, stamp; };
 
-// Largest usable stamp on one edge at round r; drops what has arrived from the pending list.
-inline int deliver(std::vector<Pend>& q, int r, int tau) {
-    size_t keep = 0;
-    for (size_t k = 0; k < q.size(); ++k) {
-        if (q[k].arrival <= r) tau = std::max(tau, q[k].stamp);
-        else q[keep++] = q[k];
+// Packets in flight on one edge.  A handful at most in practice (bounded by the largest delay and
+// by how long the receiver stays idle), so they live inline; a longer queue spills to the heap.
+struct PendQ {
+    static constexpr int kInline = 14;
+    Pend a[kInline];
+    int n = 0;
+    std::vector<Pend>* more = nullptr;
+    ~PendQ() { delete more; }
+    void push(Pend p) {
+        if (more) { more->push_back(p); return; }
+        if (n < kInline) { a[n++] = p; return; }
+        more = new std::vector<Pend>(a, a + n);
+        more->push_back(p);
     }
-    q.resize(keep);
+};
+
+// Largest usable stamp on one edge at round r; drops what has arrived from the pending list.
+inline int deliver(PendQ& q, int r, int tau) {
+    if (q.more) {
+        std::vector<Pend>& v = *q.more;
+        size_t keep = 0;
+        for (size_t k = 0; k < v.size(); ++k) {
+            if (v[k].arrival <= r) tau = std::max(tau, v[k].stamp);
+            else v[keep++] = v[k];
+        }
+        v.resize(keep);
+        return tau;
+    }
+    int keep = 0;
+    for (int k = 0; k < q.n; ++k) {
+        if (q.a[k].arrival <= r) tau = std::max(tau, q.a[k].stamp);
+        else q.a[keep++] = q.a[k];
+    }
+    q.n = keep;
     return tau;
 }
 }  // namespace
@@ -179,9 +206,14 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
 
     // ---- pass 1: consumed stamps, version lifetimes -----------------------------------------
     const int INF = INT_MAX;
-    std::vector<std::vector<Pend>> pend_v(R.E), pend_c(C.E);
+    std::vector<PendQ> pend_v(R.E), pend_c(C.E);
     std::vector<int> tau_v(R.E, 0), tau_rho(C.E, 0), t(n, 0);
     c.ev_of.assign(n, {});
+    {
+        std::vector<int> cnt(n, 0);
+        for (int64_t ev = 0; ev < nE; ++ev) cnt[c.act_node[ev]]++;
+        for (int i = 0; i < n; ++i) c.ev_of[i].reserve(cnt[i]);
+    }
     std::vector<std::vector<int>>& ev_of = c.ev_of;    // node -> event id of stamp s at [s-1]
     c.used_tau_v.reserve(c.in_r_off[nE]);
     c.used_tau_rho.reserve(c.in_c_off[nE]);
@@ -238,7 +270,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
                 int d = s->send_r[c.out_r_off[ev] + k];
                 if (d >= 0) {
                     v_sent[ev] = 1;
-                    pend_v[R.oeid[R.optr[i] + k]].push_back({r + 1 + d, stamp});
+                    pend_v[R.oeid[R.optr[i] + k]].push({r + 1 + d, stamp});
                 }
             }
             for (int k = 0; k < C.outdeg(i); ++k) {
@@ -246,7 +278,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
                 c.rho_write[vid] = r;
                 rho_last_sender[vid] = r;
                 int d = s->send_c[vid];
-                if (d >= 0) pend_c[C.oeid[C.optr[i] + k]].push_back({r + 1 + d, stamp});
+                if (d >= 0) pend_c[C.oeid[C.optr[i] + k]].push({r + 1 + d, stamp});
             }
         }
     }
@@ -335,76 +367,114 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     }
 
     // ---- pass 3: device descriptors and the method's traffic ---------------------------------
+    // Rounds are independent of one another here once every list's starting offset is known, so
+    // long schedules are filled in by several threads, each on a contiguous span of rounds.
     c.ev.resize(nE);
     c.round_streams.assign(K + 1, 0);
     c.round_streams_method.assign(K + 1, 0);
-    c.mix_slot.reserve(c.in_r_off[nE]);  c.mix_w.reserve(c.in_r_off[nE]);
-    c.news_new.reserve(c.in_c_off[nE]);  c.news_prev.reserve(c.in_c_off[nE]);  c.news_edge.reserve(c.in_c_off[nE]);
-    c.out_cur.reserve(nRho);  c.out_new.reserve(nRho);  c.out_a.reserve(nRho);  c.out_edge.reserve(nRho);
+    std::vector<int64_t> mix_at(K + 1, 0), news_at(K + 1, 0);          // list offsets at the start of each round
     for (int r = 0; r < K; ++r) {
-        int64_t streams = 0, method = 0;
-        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
-            const int i = c.act_node[ev];
-            EvDesc d{};
-            d.node = i;
-            d.v_out = c.v_slot[ev];
-            d.w_self = R.diag[i];
-            d.a_self = C.diag[i];
-            d.stamp = stamp_of[ev];
-            d.g_par = (stamp_of[ev] - 1) & 1;
-            d.sample = (int32_t)(n + ev);
-            d.mix_beg = (int32_t)c.mix_slot.size();
-            for (int e = R.rowptr[i], k = 0; e < R.rowptr[i + 1]; ++e, ++k) {
-                int tau = c.used_tau_v[c.in_r_off[ev] + k];
-                if (tau < 1) continue;                 // stamp 0 is the zero vector: nothing to read
-                int slot = c.v_slot[ev_of[R.col[e]][tau - 1]];
-                if (slot < 0) return fail(err, RFAST_ESCHED, "internal: consumed v version without a row (event %lld)", ev);
-                c.mix_slot.push_back(slot);
-                c.mix_w.push_back(R.w[e]);
-            }
-            d.mix_cnt = (int32_t)c.mix_slot.size() - d.mix_beg;
-            d.news_beg = (int32_t)c.news_new.size();
-            int news_streams = 0;
-            for (int e = C.rowptr[i], k = 0; e < C.rowptr[i + 1]; ++e, ++k) {
-                int tau = c.used_tau_rho[c.in_c_off[ev] + k];
-                int prev = c.prev_tau_rho[c.in_c_off[ev] + k];
-                if (tau <= prev) continue;             // nothing newer: rho[tau] - rho~ = 0
-                const auto& evs = ev_of[C.col[e]];
-                c.news_new.push_back(c.rho_slot[c.out_c_off[evs[tau - 1]] + C.opos[e]]);
-                const bool sub = !buckets && prev >= 1;   // a bucket holds the difference itself
-                c.news_prev.push_back(sub ? c.rho_slot[c.out_c_off[evs[prev - 1]] + C.opos[e]] : -1);
-                c.news_edge.push_back(e);
-                news_streams += 1 + sub;
-            }
-            d.news_cnt = (int32_t)c.news_new.size() - d.news_beg;
-            d.out_beg = (int32_t)c.out_new.size();
-            int out_streams = 0;
-            for (int k = 0; k < C.outdeg(i); ++k) {
-                int e = C.oeid[C.optr[i] + k];
-                int cur = -1;
-                if (buckets) {                         // add to the bucket unless this is its first contribution
+        int64_t nm = 0, nn = 0;
+        for (int64_t q = c.in_r_off[c.act_ptr[r]]; q < c.in_r_off[c.act_ptr[r + 1]]; ++q) nm += c.used_tau_v[q] >= 1;
+        for (int64_t q = c.in_c_off[c.act_ptr[r]]; q < c.in_c_off[c.act_ptr[r + 1]]; ++q) nn += c.used_tau_rho[q] > c.prev_tau_rho[q];
+        mix_at[r + 1] = mix_at[r] + nm;
+        news_at[r + 1] = news_at[r] + nn;
+    }
+    c.mix_slot.resize(mix_at[K]);  c.mix_w.resize(mix_at[K]);
+    c.news_new.resize(news_at[K]);  c.news_prev.resize(news_at[K]);  c.news_edge.resize(news_at[K]);
+    c.out_cur.resize(nRho);  c.out_new.resize(nRho);  c.out_a.resize(nRho);  c.out_edge.resize(nRho);
+    std::vector<int64_t> round_s(K, 0), round_m(K, 0);
+    auto fill = [&](int r_begin, int r_end, int64_t* bad_event) {
+        for (int r = r_begin; r < r_end; ++r) {
+            int64_t streams = 0, method = 0, mix_pos = mix_at[r], news_pos = news_at[r];
+            for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+                const int i = c.act_node[ev];
+                EvDesc d{};
+                d.node = i;
+                d.v_out = c.v_slot[ev];
+                d.w_self = R.diag[i];
+                d.a_self = C.diag[i];
+                d.stamp = stamp_of[ev];
+                d.g_par = (stamp_of[ev] - 1) & 1;
+                d.sample = (int32_t)(n + ev);
+                d.mix_beg = (int32_t)mix_pos;
+                for (int e = R.rowptr[i], k = 0; e < R.rowptr[i + 1]; ++e, ++k) {
+                    int tau = c.used_tau_v[c.in_r_off[ev] + k];
+                    if (tau < 1) continue;                 // stamp 0 is the zero vector: nothing to read
+                    int slot = c.v_slot[ev_of[R.col[e]][tau - 1]];
+                    if (slot < 0 && *bad_event < 0) *bad_event = ev;
+                    c.mix_slot[mix_pos] = slot;
+                    c.mix_w[mix_pos++] = R.w[e];
+                }
+                d.mix_cnt = (int32_t)mix_pos - d.mix_beg;
+                d.news_beg = (int32_t)news_pos;
+                int news_streams = 0;
+                for (int e = C.rowptr[i], k = 0; e < C.rowptr[i + 1]; ++e, ++k) {
+                    int tau = c.used_tau_rho[c.in_c_off[ev] + k];
+                    int prev = c.prev_tau_rho[c.in_c_off[ev] + k];
+                    if (tau <= prev) continue;             // nothing newer: rho[tau] - rho~ = 0
+                    const auto& evs = ev_of[C.col[e]];
+                    c.news_new[news_pos] = c.rho_slot[c.out_c_off[evs[tau - 1]] + C.opos[e]];
+                    const bool sub = !buckets && prev >= 1;   // a bucket holds the difference itself
+                    c.news_prev[news_pos] = sub ? c.rho_slot[c.out_c_off[evs[prev - 1]] + C.opos[e]] : -1;
+                    c.news_edge[news_pos++] = e;
+                    news_streams += 1 + sub;
+                }
+                d.news_cnt = (int32_t)news_pos - d.news_beg;
+                d.out_beg = (int32_t)c.out_c_off[ev];
+                int out_streams = 0;
+                for (int k = 0; k < C.outdeg(i); ++k) {
                     const int64_t vid = c.out_c_off[ev] + k;
-                    if (c.rho_leader[vid] != vid) cur = c.rho_slot[vid];
-                } else if (stamp_of[ev] >= 2) cur = c.rho_slot[c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k];
-                c.out_cur.push_back(cur);
-                c.out_new.push_back(c.rho_slot[c.out_c_off[ev] + k]);
-                c.out_a.push_back(C.w[e]);
-                c.out_edge.push_back(e);
-                out_streams += 1 + (cur >= 0);
+                    int e = C.oeid[C.optr[i] + k];
+                    int cur = -1;
+                    if (buckets) {                         // add to the bucket unless this is its first contribution
+                        if (c.rho_leader[vid] != vid) cur = c.rho_slot[vid];
+                    } else if (stamp_of[ev] >= 2) cur = c.rho_slot[c.out_c_off[ev_of[i][stamp_of[ev] - 2]] + k];
+                    c.out_cur[vid] = cur;
+                    c.out_new[vid] = c.rho_slot[vid];
+                    c.out_a[vid] = C.w[e];
+                    c.out_edge[vid] = e;
+                    out_streams += 1 + (cur >= 0);
+                }
+                d.out_cnt = C.outdeg(i);
+                c.ev[ev] = d;
+                // fp32 streams per coordinate: S1/S2a read x, z, the neighbours' v, write v (if a
+                // packet leaves) and x; S2b/S2c read the news, write z and the running sums
+                const int64_t base = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
+                streams += base + (mt.elementwise ? mt.data_streams : mt.grad_track_streams);
+                // what the method itself must move: x and z read once, the gradient moved once
+                // (remembered one read, new one written), no stream that exists only because the
+                // step is split over several kernels or because of the tracker's arithmetic
+                method += base + mt.method_streams;
             }
-            d.out_cnt = (int32_t)c.out_new.size() - d.out_beg;
-            c.ev[ev] = d;
-            // fp32 streams per coordinate: S1/S2a read x, z, the neighbours' v, write v (if a
-            // packet leaves) and x; S2b/S2c read the news, write z and the running sums
-            const int64_t base = 2 + d.mix_cnt + (d.v_out >= 0) + 1 + news_streams + 1 + out_streams;
-            streams += base + (mt.elementwise ? mt.data_streams : mt.grad_track_streams);
-            // what the method itself must move: x and z read once, the gradient moved once
-            // (remembered one read, new one written), no stream that exists only because the
-            // step is split over several kernels or because of the tracker's arithmetic
-            method += base + mt.method_streams;
+            round_s[r] = streams;
+            round_m[r] = method;
         }
-        c.round_streams[r + 1] = c.round_streams[r] + streams;
-        c.round_streams_method[r + 1] = c.round_streams_method[r] + method;
+    };
+    {
+        int nthreads = 1;
+        if (nE >= 50000) nthreads = (int)std::min<unsigned>(8u, std::max(1u, std::thread::hardware_concurrency()));
+        std::vector<int64_t> bad(nthreads, -1);
+        if (nthreads == 1) {
+            fill(0, K, &bad[0]);
+        } else {
+            std::vector<std::thread> pool;
+            int r0 = 0;
+            for (int th = 0; th < nthreads; ++th) {             // spans of about equally many events
+                const int64_t target = nE * (th + 1) / nthreads;
+                int r1 = th + 1 == nthreads ? K : r0;
+                while (th + 1 < nthreads && r1 < K && c.act_ptr[r1] < target) ++r1;
+                pool.emplace_back(fill, r0, r1, &bad[th]);
+                r0 = r1;
+            }
+            for (auto& t_ : pool) t_.join();
+        }
+        for (int64_t bev : bad)
+            if (bev >= 0) return fail(err, RFAST_ESCHED, "internal: consumed v version without a row (event %lld)", bev);
+    }
+    for (int r = 0; r < K; ++r) {
+        c.round_streams[r + 1] = c.round_streams[r] + round_s[r];
+        c.round_streams_method[r + 1] = c.round_streams_method[r] + round_m[r];
     }
     out = std::move(c);
     return RFAST_OK;
