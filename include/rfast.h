@@ -357,6 +357,14 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s,
                        int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
                        char* err, size_t err_len);
 
+/* Host-only, like rfast_compile_host: compiles the schedule and folds everything the kernels are
+ * driven by (event descriptors, mixing / news / running-sum row lists and weights, the byte
+ * counts per round) into one 64-bit number.  Two compilations of the same problem and schedule
+ * give the same number whatever the number of host threads the compiler used
+ * (environment variable RFAST_COMPILE_THREADS caps it; long schedules use up to 8). */
+int rfast_compile_digest(const rfast_problem* prob, const rfast_schedule* s, uint64_t* digest,
+                         char* err, size_t err_len);
+
 /* No counterpart in the paper: a service entry point for callers that are not allowed to
  * allocate device memory.  Some hosts of this library cannot call cudaMalloc where they need a
  * gradient: a framework that hands the whole GPU to its own memory pool up front, a latency-

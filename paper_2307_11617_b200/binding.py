@@ -87,6 +87,7 @@ def lib():
         L.rfast_version.restype = C.c_char_p
         L.rfast_compile_host.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule)] + [C.c_void_p] * 5 + \
             [C.c_char_p, C.c_size_t]
+        L.rfast_compile_digest.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule), C.POINTER(C.c_uint64), C.c_char_p, C.c_size_t]
         L.rfast_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int64]
         L.rfast_checkpoint_size.argtypes = [C.c_void_p]
         L.rfast_checkpoint_size.restype = C.c_int64
@@ -276,6 +277,18 @@ def rfast_compile_host(wl, s):
     return {"used_tau_v": used_v, "used_tau_rho": used_r, "v_ver": v_ver, "rho_ver": rho_ver,
             "v_rows": int(counts[0]), "rho_rows": int(counts[1]), "events": int(counts[2]),
             "streams": int(counts[3])}
+
+
+def rfast_compile_digest(wl, s) -> int:
+    """One number for everything the compiled schedule drives the kernels with (host only)."""
+    keep = []
+    P, S = _problem(wl, keep), _schedule(s, keep)
+    out = C.c_uint64(0)
+    err = C.create_string_buffer(512)
+    rc = lib().rfast_compile_digest(C.byref(P), C.byref(S), C.byref(out), err, 512)
+    if rc != OK:
+        raise RFastError(rc, err.value.decode())
+    return int(out.value)
 
 
 OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS, OPT_ONE_PASS, OPT_CLUSTER_SIZE = 0, 1, 2, 3, 4, 5

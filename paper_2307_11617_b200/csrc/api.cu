@@ -1127,9 +1127,9 @@ int rfast_write_state(rfast_ctx* ctx, int which, const void* src, size_t bytes) 
     return set_err(ctx, RFAST_ENOMEM, "write_state: host allocation failed");
 }
 
-int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32_t* used_tau_v,
-                       int32_t* used_tau_rho, int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
-                       char* errbuf, size_t err_len) try {
+static int compile_host_impl(const rfast_problem* prob, const rfast_schedule* s, int32_t* used_tau_v,
+                             int32_t* used_tau_rho, int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
+                             uint64_t* digest, char* errbuf, size_t err_len) try {
     std::string err;
     auto done = [&](int rc) {
         if (errbuf && err_len) { std::snprintf(errbuf, err_len, "%s", err.c_str()); }
@@ -1157,10 +1157,32 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32
     if (counts) {
         counts[0] = c.n_v_slots; counts[1] = c.n_rho_slots; counts[2] = c.n_events; counts[3] = c.round_streams[c.K];
     }
+    if (digest) {          // everything the kernels are driven by, folded into one number
+        uint64_t h = 1469598103934665603ull;
+        auto mix = [&](const void* ptr, size_t bytes) {
+            const unsigned char* q = (const unsigned char*)ptr;
+            for (size_t k = 0; k < bytes; ++k) { h ^= q[k]; h *= 1099511628211ull; }
+        };
+        auto vec = [&](const auto& v) { if (!v.empty()) mix(v.data(), v.size() * sizeof(v[0])); };
+        vec(c.ev); vec(c.mix_slot); vec(c.mix_w); vec(c.news_new); vec(c.news_prev); vec(c.news_edge);
+        vec(c.out_cur); vec(c.out_new); vec(c.out_a); vec(c.out_edge); vec(c.round_streams); vec(c.round_streams_method);
+        *digest = h;
+    }
     return done(RFAST_OK);
 } catch (...) {
     if (errbuf && err_len) std::snprintf(errbuf, err_len, "host allocation failed");
     return RFAST_ENOMEM;
+}
+
+int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32_t* used_tau_v,
+                       int32_t* used_tau_rho, int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
+                       char* errbuf, size_t err_len) {
+    return compile_host_impl(prob, s, used_tau_v, used_tau_rho, v_ver, rho_ver, counts, nullptr, errbuf, err_len);
+}
+
+int rfast_compile_digest(const rfast_problem* prob, const rfast_schedule* s, uint64_t* digest, char* errbuf, size_t err_len) {
+    if (!digest) return RFAST_EINVAL;
+    return compile_host_impl(prob, s, nullptr, nullptr, nullptr, nullptr, nullptr, digest, errbuf, err_len);
 }
 
 }  // extern "C"

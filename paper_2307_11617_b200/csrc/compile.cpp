@@ -11,6 +11,7 @@
 #include <climits>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <thread>
 
 #include "rfast_internal.h"
@@ -454,6 +455,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     {
         int nthreads = 1;
         if (nE >= 50000) nthreads = (int)std::min<unsigned>(8u, std::max(1u, std::thread::hardware_concurrency()));
+        if (const char* cap = std::getenv("RFAST_COMPILE_THREADS")) nthreads = std::max(1, std::min(nthreads, std::atoi(cap)));
         std::vector<int64_t> bad(nthreads, -1);
         if (nthreads == 1) {
             fill(0, K, &bad[0]);

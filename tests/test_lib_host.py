@@ -219,3 +219,30 @@ def test_bucket_tracker_rows_hold_exactly_one_consumption(rfast_lib, name, ov):
         if row in by_row:
             assert by_row[row] < first, "bucket row reused before its consumption"
         by_row[row] = last
+
+
+def test_threaded_descriptor_pass_equals_the_single_threaded_one(rfast_lib, monkeypatch):
+    """Schedules of 50,000 events and more have their device descriptors filled in by several
+    host threads, each on a span of rounds.  Everything the kernels are driven by must come out
+    the same as from one thread (digest over descriptors, row lists, weights, byte counts), for
+    the running sums and for the bucket tracker, on a general digraph."""
+    import paper_2307_11617_b200 as pkg
+    from workloads import activation_bernoulli, graph_from_edges, make_schedule
+    wl = build_config("quad_tree64", seed=3, n=48, p=8, K=4)
+    rng = np.random.default_rng(5)
+    n = wl.n
+    edges = {(i, (i + 1) % n) for i in range(n)} | {(int(a), int(b)) for a, b in rng.integers(0, n, size=(3 * n, 2)) if a != b}
+    wl.G_R, wl.G_C = graph_from_edges(n, edges, "row"), graph_from_edges(n, edges, "col")
+    sch = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, 2400, 0.5, rng), 0.2, 4, rng, batch=0)
+    assert sch.n_events >= 50_000
+    for tracker in (0, 1):
+        wl.tracker = tracker
+        monkeypatch.setenv("RFAST_COMPILE_THREADS", "1")
+        one = pkg.rfast_compile_digest(wl, sch)
+        monkeypatch.setenv("RFAST_COMPILE_THREADS", "8")
+        many = pkg.rfast_compile_digest(wl, sch)
+        monkeypatch.delenv("RFAST_COMPILE_THREADS")
+        assert one == many == pkg.rfast_compile_digest(wl, sch)
+    # and the digest does see a difference: another schedule, another number
+    other = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, 2400, 0.5, rng), 0.2, 4, rng, batch=0)
+    assert pkg.rfast_compile_digest(wl, other) != many
