@@ -304,7 +304,9 @@ def measure_config(name, args, steps, world, rank, local, cpu_budget_s, stream=N
     per_launch = max(1, launches // max(1, steps))
     fused = wl.model == "quad_diag"
     roofline = {"bound": "hbm",
-                "kernel": "k_fused_quad" if fused else "one round: k_mix + gradient kernels + tracking pass",
+                "kernel": "k_fused_quad" if fused else
+                          "k_logit_fused (one launch per round)" if wl.model == "logistic_sparse" and per_launch == K_rounds else
+                          "one round: k_mix + gradient kernels + tracking pass",
                 "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
                 "bytes": "what the method must move: x, z read once, the gradient moved once, packets and running sums as compiled",
