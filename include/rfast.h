@@ -211,13 +211,35 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out);
 
 /* Compiles a schedule (Algorithm 2, S.0) for the handle and resets the state to the
  * initial one (round 0).  A second call replaces the schedule and starts over at round 0 as
- * well: rounds are not appended (to continue a run, load the longer schedule and move the
- * state across with rfast_checkpoint_* or rfast_seek + rfast_write_state).  Host side, integers only: for every event and in-edge the stamp
+ * well; rounds are appended with rfast_append_schedule.  Host side, integers only: for every event and in-edge the stamp
  * that is consumed (tau_v, tau_rho of Algorithm 1, i.e. the delays d_v, d_rho of
  * Algorithm 2), then the lifetime of every packet version and a version row for each.
  * Uploads the per-round descriptors.  RFAST_ESCHED if the arrays are inconsistent (sizes,
  * order, ids, codes < -1). */
 int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s);
+
+/* Appends the rounds of `more` to the loaded schedule (Algorithm 2 goes on: k keeps counting).
+ * The state, the packets on their way and the round counter stay as they are; afterwards
+ * rfast_run can go on through the new rounds, and the result equals, bit for bit, that of the
+ * whole schedule loaded at once.  Needs RFAST_OPT_OPEN_END set before the first
+ * rfast_load_schedule: only then does the engine keep, past the end of what is loaded, what a
+ * later activation may still read (per edge the version its receiver holds and every packet
+ * that is on its way or waiting in an inbox, every sender's latest running sums); the rows
+ * of the rounds already loaded never move.  RFAST_ESTATE without that option or without a
+ * schedule; running sums only (not RFAST_TRACKER_BUCKETS, whose last bucket per edge lumps
+ * together what a later round would consume apart).
+ *   more: as for rfast_load_schedule, its rounds and events numbered from 0: act_ptr[0] = 0,
+ *   send codes per (event of `more`, out-edge), delays counted from the event's own round;
+ *   batch_idx holds (n + events of `more`) * B entries of which the first n * B (zeta^0) are
+ *   ignored; alpha_round (optional) has more->K entries -- where only one of the parts gives
+ *   step sizes, the other runs at the problem's alpha.
+ * May be called at any round counter (the rounds not yet run stay as compiled).  The host
+ * cost is that of compiling the whole schedule loaded so far; device pools that have to grow
+ * are copied once.  RFAST_ESCHED as for rfast_load_schedule (nothing is changed then); on
+ * RFAST_ENOMEM / RFAST_ECUDA while the pools are being replaced the handle is left without a
+ * schedule.  Checkpoints are tied to the sequence of loads: a blob saved after an append
+ * restores only into a handle that went through the same load and appends. */
+int rfast_append_schedule(rfast_ctx* ctx, const rfast_schedule* more);
 
 /* Runs the next `rounds` rounds: for every active node S1 (v = x - alpha z), S2a (mix over
  * G_R), the sample gradient at the new x, S2b/S2c (tracking over G_C with the running sums
@@ -304,9 +326,14 @@ int64_t rfast_query(rfast_ctx* ctx, int what);
  *   RFAST_OPT_CLUSTER_SIZE  CTAs per activation on that path: 0 (default) = the smallest of 1, 2,
  *                         4, 8 that fits; RFAST_EINVAL if the given size does not fit.  The
  *                         partial dot products are added per CTA, so results agree to rounding
- *                         across sizes.  To be set before rfast_load_schedule. */
+ *                         across sizes.  To be set before rfast_load_schedule.
+ *   RFAST_OPT_OPEN_END    1: schedules are loaded open-ended, so that rfast_append_schedule can
+ *                         add rounds later (a few more version rows stay occupied at the end of
+ *                         what is loaded; values and byte counts do not change).  Default 0.
+ *                         To be set before rfast_load_schedule; RFAST_EINVAL with
+ *                         RFAST_TRACKER_BUCKETS. */
 enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1, RFAST_OPT_WAIT_LIMIT_MS = 2, RFAST_OPT_PHANTOM_ARRIVALS = 3,
-       RFAST_OPT_ONE_PASS = 4, RFAST_OPT_CLUSTER_SIZE = 5 };
+       RFAST_OPT_ONE_PASS = 4, RFAST_OPT_CLUSTER_SIZE = 5, RFAST_OPT_OPEN_END = 6 };
 int rfast_set_option(rfast_ctx* ctx, int option, int64_t value);
 
 /* Waits for the handle's stream; reports a pending asynchronous error. */
@@ -364,6 +391,17 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s,
  * (environment variable RFAST_COMPILE_THREADS caps it; long schedules use up to 8). */
 int rfast_compile_digest(const rfast_problem* prob, const rfast_schedule* s, uint64_t* digest,
                          char* err, size_t err_len);
+
+/* Host-only companion of rfast_append_schedule (needs no CUDA device): compiles `first`
+ * open-ended, then `first` followed by `more` the way rfast_append_schedule does, and checks
+ * (1) that no version row, row list or event descriptor of the rounds of `first` differs
+ * between the two and (2) that the stamps consumed (tau_v, tau_rho per event and in-edge) and
+ * the final counters t_i are those of the whole schedule compiled in one piece.
+ * counts (optional, int64[6]): version rows of v and of rho for `first` open-ended, for the
+ * appended whole, for the whole compiled in one piece (closed end).  RFAST_OK if both hold,
+ * RFAST_ESCHED with a message otherwise. */
+int rfast_compile_append_check(const rfast_problem* prob, const rfast_schedule* first,
+                               const rfast_schedule* more, int64_t* counts, char* err, size_t err_len);
 
 /* No counterpart in the paper: a service entry point for callers that are not allowed to
  * allocate device memory.  Some hosts of this library cannot call cudaMalloc where they need a

@@ -74,6 +74,9 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.rfast_create.argtypes = [C.POINTER(_Problem), C.c_void_p, C.POINTER(C.c_void_p)]
         L.rfast_load_schedule.argtypes = [C.c_void_p, C.POINTER(_Schedule)]
+        L.rfast_append_schedule.argtypes = [C.c_void_p, C.POINTER(_Schedule)]
+        L.rfast_compile_append_check.argtypes = [C.POINTER(_Problem), C.POINTER(_Schedule), C.POINTER(_Schedule),
+                                                 C.c_void_p, C.c_char_p, C.c_size_t]
         L.rfast_run.argtypes = [C.c_void_p, C.c_int32, C.c_int]
         L.rfast_read_state.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t]
         L.rfast_reset.argtypes = [C.c_void_p]
@@ -193,6 +196,12 @@ def rfast_load_schedule(handle, s) -> None:
     _check(lib().rfast_load_schedule(handle, C.byref(S)), handle)
 
 
+def rfast_append_schedule(handle, more) -> None:
+    keep = []
+    S = _schedule(more, keep)
+    _check(lib().rfast_append_schedule(handle, C.byref(S)), handle)
+
+
 def rfast_run(handle, rounds: int, sync: bool = True) -> None:
     _check(lib().rfast_run(handle, int(rounds), 1 if sync else 0), handle)
 
@@ -291,7 +300,21 @@ def rfast_compile_digest(wl, s) -> int:
     return int(out.value)
 
 
-OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS, OPT_ONE_PASS, OPT_CLUSTER_SIZE = 0, 1, 2, 3, 4, 5
+def rfast_compile_append_check(wl, first, more):
+    """Host only: `first` loaded open-ended and `more` appended keeps every row of `first` in place
+    and consumes the stamps of the whole schedule.  Returns the six row counts; raises otherwise."""
+    keep = []
+    P, S1, S2 = _problem(wl, keep), _schedule(first, keep), _schedule(more, keep)
+    counts = np.zeros(6, np.int64)
+    err = C.create_string_buffer(512)
+    rc = lib().rfast_compile_append_check(C.byref(P), C.byref(S1), C.byref(S2), _ptr(counts), err, 512)
+    if rc != OK:
+        raise RFastError(rc, err.value.decode())
+    return {"first": (int(counts[0]), int(counts[1])), "appended": (int(counts[2]), int(counts[3])),
+            "whole": (int(counts[4]), int(counts[5]))}
+
+
+OPT_PERSISTENT, OPT_GRAPHS, OPT_WAIT_LIMIT_MS, OPT_PHANTOM_ARRIVALS, OPT_ONE_PASS, OPT_CLUSTER_SIZE, OPT_OPEN_END = 0, 1, 2, 3, 4, 5, 6
 
 
 def rfast_set_option(handle, option: int, value: int) -> None:
@@ -355,6 +378,10 @@ class Engine:
     def load_schedule(self, s):
         rfast_load_schedule(self.h, s)
         self.K = int(s.K)
+
+    def append_schedule(self, more):
+        rfast_append_schedule(self.h, more)
+        self.K += int(more.K)
 
     def run(self, rounds=None, sync=True):
         rfast_run(self.h, self.K - self.query(Q_ROUND) if rounds is None else rounds, sync)

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <memory>
 #include <new>
 #include <string>
 #include <vector>
@@ -30,6 +31,84 @@ int  mlp_grad_launch(MlpPlan* plan, const GradArgs& g, const __nv_bfloat16* xb, 
 }  // namespace rfast
 
 static std::string g_create_error;
+
+// Host copy of the raw arrays of an open-ended schedule (what rfast_append_schedule extends).
+struct RawSchedule {
+    std::vector<int32_t> act_ptr, act_node, batch_idx;
+    std::vector<int8_t> send_r, send_c;
+    std::vector<float> alpha_round;
+    bool has_alpha = false;
+    rfast_schedule view() const {
+        rfast_schedule v{};
+        v.K = (int32_t)act_ptr.size() - 1;
+        v.act_ptr = act_ptr.data();  v.act_node = act_node.data();
+        v.send_r = send_r.data();  v.n_send_r = (int64_t)send_r.size();
+        v.send_c = send_c.data();  v.n_send_c = (int64_t)send_c.size();
+        v.batch_idx = batch_idx.empty() ? nullptr : batch_idx.data();  v.n_batch_idx = (int64_t)batch_idx.size();
+        v.alpha_round = has_alpha ? alpha_round.data() : nullptr;
+        return v;
+    }
+};
+
+// raw arrays of a schedule that compile_schedule has accepted
+static std::unique_ptr<RawSchedule> raw_of(const rfast_schedule* s, int batch) {
+    auto raw = std::make_unique<RawSchedule>();
+    const int64_t nE = s->act_ptr[s->K];
+    raw->act_ptr.assign(s->act_ptr, s->act_ptr + s->K + 1);
+    if (nE > 0) raw->act_node.assign(s->act_node, s->act_node + nE);
+    if (s->n_send_r > 0) raw->send_r.assign(s->send_r, s->send_r + s->n_send_r);
+    if (s->n_send_c > 0) raw->send_c.assign(s->send_c, s->send_c + s->n_send_c);
+    if (batch > 0) raw->batch_idx.assign(s->batch_idx, s->batch_idx + s->n_batch_idx);
+    raw->has_alpha = s->alpha_round != nullptr;
+    if (raw->has_alpha) raw->alpha_round.assign(s->alpha_round, s->alpha_round + s->K);
+    return raw;
+}
+
+// raw := raw followed by the rounds of `more` (events and rounds of `more` count from 0; its copy of
+// zeta^0 is dropped).  Returns an error text, or nullptr.
+static const char* append_raw(RawSchedule& raw, const rfast_schedule* more, int n, int batch, float alpha) {
+    if (!more || more->K < 0 || !more->act_ptr) return "schedule: null or K < 0";
+    if (more->act_ptr[0] != 0) return "schedule: act_ptr[0] != 0";
+    for (int r = 0; r < more->K; ++r)
+        if (more->act_ptr[r + 1] < more->act_ptr[r]) return "schedule: act_ptr decreases";
+    const int64_t nE2 = more->act_ptr[more->K];
+    if (nE2 > 0 && !more->act_node) return "schedule: act_node is null";
+    if ((more->n_send_r > 0 && !more->send_r) || (more->n_send_c > 0 && !more->send_c) || more->n_send_r < 0 || more->n_send_c < 0)
+        return "schedule: send codes are null";
+    const int64_t lead = (int64_t)n * batch;
+    if (batch > 0 && (!more->batch_idx || more->n_batch_idx != lead + nE2 * batch))
+        return "schedule: batch_idx must hold (n + events) * B entries";
+    const int K1 = (int)raw.act_ptr.size() - 1;
+    if ((int64_t)K1 + more->K > INT32_MAX / 2 || (int64_t)raw.act_ptr.back() + nE2 > INT32_MAX / 2) return "schedule: too many rounds or events";
+    const int32_t ev0 = raw.act_ptr.back();
+    for (int r = 1; r <= more->K; ++r) raw.act_ptr.push_back(ev0 + more->act_ptr[r]);
+    if (nE2 > 0) raw.act_node.insert(raw.act_node.end(), more->act_node, more->act_node + nE2);
+    if (more->n_send_r > 0) raw.send_r.insert(raw.send_r.end(), more->send_r, more->send_r + more->n_send_r);
+    if (more->n_send_c > 0) raw.send_c.insert(raw.send_c.end(), more->send_c, more->send_c + more->n_send_c);
+    if (batch > 0) raw.batch_idx.insert(raw.batch_idx.end(), more->batch_idx + lead, more->batch_idx + more->n_batch_idx);
+    if (raw.has_alpha || more->alpha_round) {                  // a part without its own step sizes runs at the problem's alpha
+        if (!raw.has_alpha) raw.alpha_round.assign(K1, alpha);
+        raw.has_alpha = true;
+        for (int r = 0; r < more->K; ++r) raw.alpha_round.push_back(more->alpha_round ? more->alpha_round[r] : alpha);
+    }
+    return nullptr;
+}
+
+// Has nothing of the rounds compiled in `o` moved in `c` (the same rounds, more appended)?
+static bool prefix_same(const Compiled& o, const Compiled& c) {
+    const int64_t nE1 = o.n_events;
+    return c.n_events >= nE1 && c.n_v_slots >= o.n_v_slots && c.n_rho_slots >= o.n_rho_slots &&
+           std::equal(o.v_slot.begin(), o.v_slot.end(), c.v_slot.begin()) &&
+           std::equal(o.rho_slot.begin(), o.rho_slot.end(), c.rho_slot.begin()) &&
+           std::equal(o.used_tau_v.begin(), o.used_tau_v.end(), c.used_tau_v.begin()) &&
+           std::equal(o.used_tau_rho.begin(), o.used_tau_rho.end(), c.used_tau_rho.begin()) &&
+           std::equal(o.mix_slot.begin(), o.mix_slot.end(), c.mix_slot.begin()) &&
+           std::equal(o.news_new.begin(), o.news_new.end(), c.news_new.begin()) &&
+           std::equal(o.news_prev.begin(), o.news_prev.end(), c.news_prev.begin()) &&
+           std::equal(o.out_cur.begin(), o.out_cur.end(), c.out_cur.begin()) &&
+           std::equal(o.out_new.begin(), o.out_new.end(), c.out_new.begin()) &&
+           (nE1 == 0 || std::memcmp(o.ev.data(), c.ev.data(), (size_t)nE1 * sizeof(EvDesc)) == 0);
+}
 
 struct rfast_ctx {
     cudaStream_t stream = nullptr;
@@ -83,6 +162,10 @@ struct rfast_ctx {
     int fused_cluster = 0, fused_ranges = 0;      // cluster size (0: the path is not available), ranges per CTA
     int fused_threads = 512, fused_stash = 0;
     size_t fused_smem = 0;
+    // open-ended schedules: rounds may be appended (rfast_append_schedule)
+    bool opt_open_end = false;
+    std::vector<int> holds;                 // rounds at which the loaded schedule was held open (its end, earlier ends)
+    std::unique_ptr<RawSchedule> raw;       // the raw arrays loaded so far (kept only when open-ended)
     int round = 0;
     int64_t launches = 0;
     // recorded span of rounds [graph_r0, graph_r1): a sequence of graphs of about a thousand kernels each
@@ -551,14 +634,23 @@ int rfast_create(const rfast_problem* prob, void* cuda_stream, rfast_ctx** out) 
     return set_err(nullptr, RFAST_EINVAL, "unexpected failure in rfast_create");
 }
 
-int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
-    if (!ctx) return RFAST_EINVAL;
-    CK(cudaStreamSynchronize(ctx->stream));
-    Compiled comp;
-    std::string err;
-    const bool one_pass = ctx->model == RFAST_MODEL_LOGISTIC_SPARSE && ctx->opt_fused && ctx->fused_cluster > 0;
-    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated, one_pass), ctx->buckets, comp, err);
-    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+// Puts a compiled schedule in place: descriptors up, version-row pools, scratch.  `s` holds the raw
+// arrays `comp` was compiled from.  keep_state: rounds were appended to the schedule in place; the
+// rows written so far and the round counter carry over instead of the state starting at round 0.
+static int install_schedule(rfast_ctx* ctx, const rfast_schedule* s, Compiled&& comp, bool keep_state) {
+    int rc;
+    // rounds appended: the version rows written so far carry over into the (possibly larger) pools
+    float *old_v = nullptr, *old_r = nullptr;
+    const int64_t old_nv = ctx->comp.n_v_slots, old_nr = ctx->comp.n_rho_slots;
+    if (keep_state) {
+        old_v = ctx->vbuf;  old_r = ctx->rbuf;
+        auto& al = ctx->sched_allocs;
+        al.erase(std::remove_if(al.begin(), al.end(), [&](void* q) { return q == (void*)old_v || q == (void*)old_r; }), al.end());
+    }
+    struct OldRows {                                   // freed on every way out
+        float *v, *r;
+        ~OldRows() { if (v) cudaFree(v); if (r) cudaFree(r); }
+    } old_rows{old_v, old_r};
     free_schedule(ctx);
     ctx->alpha_round.clear();
     if (s->alpha_round) {
@@ -590,6 +682,7 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
         if (s->n_send_c > 0) mix(s->send_c, (size_t)s->n_send_c);
         if (ctx->batch > 0) mix(s->batch_idx, (size_t)s->n_batch_idx * sizeof(int32_t));
         if (s->alpha_round) mix(s->alpha_round, (size_t)s->K * sizeof(float));
+        for (int b : ctx->holds) mix(&b, sizeof b);     // where rounds were appended: the rows depend on it
         ctx->sched_hash = hsh;
     }
     ctx->comp = std::move(comp);
@@ -618,6 +711,16 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
     CK(dev_alloc(ctx, &ctx->rbuf, (size_t)c.n_rho_slots * ctx->stride * (ctx->rho2 ? 2 : 1), true));
     CK(cudaMemsetAsync(ctx->vbuf, 0, std::max<size_t>(1, (size_t)c.n_v_slots * ctx->stride) * sizeof(float), ctx->stream));
     CK(cudaMemsetAsync(ctx->rbuf, 0, std::max<size_t>(1, (size_t)c.n_rho_slots * ctx->stride * (ctx->rho2 ? 2 : 1)) * sizeof(float), ctx->stream));
+    if (keep_state) {
+        const size_t row = (size_t)ctx->stride * sizeof(float);
+        if (old_v && old_nv > 0) CK(cudaMemcpyAsync(ctx->vbuf, old_v, old_nv * row, cudaMemcpyDeviceToDevice, ctx->stream));
+        if (old_r && old_nr > 0) {
+            CK(cudaMemcpyAsync(ctx->rbuf, old_r, old_nr * row, cudaMemcpyDeviceToDevice, ctx->stream));
+            if (ctx->rho2)                              // the low-order words sit one pool further on
+                CK(cudaMemcpyAsync(ctx->rbuf + (size_t)c.n_rho_slots * ctx->stride, old_r + (size_t)old_nr * ctx->stride,
+                                   old_nr * row, cudaMemcpyDeviceToDevice, ctx->stream));
+        }
+    }
     // scratch of the two-phase gradients: residuals / logits / coefficients per (event, row[, class])
     size_t per_ev = 0;
     if (ctx->model == RFAST_MODEL_LEAST_SQUARES) per_ev = ctx->batch ? ctx->batch : ctx->rows;
@@ -659,14 +762,62 @@ int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
         }
     }
     ctx->has_sched = true;
-    rc = reset_state(ctx);
-    if (rc != RFAST_OK) return rc;
+    if (!keep_state && (rc = reset_state(ctx)) != RFAST_OK) return rc;
     CK(cudaStreamSynchronize(ctx->stream));
     return RFAST_OK;
+}
+
+int rfast_load_schedule(rfast_ctx* ctx, const rfast_schedule* s) try {
+    if (!ctx) return RFAST_EINVAL;
+    CK(cudaStreamSynchronize(ctx->stream));
+    Compiled comp;
+    std::string err;
+    const bool one_pass = ctx->model == RFAST_MODEL_LOGISTIC_SPARSE && ctx->opt_fused && ctx->fused_cluster > 0;
+    std::vector<int> holds;
+    if (ctx->opt_open_end && s && s->K >= 0) holds.push_back(s->K);
+    int rc = compile_schedule(ctx->R, ctx->Cg, s, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated, one_pass), ctx->buckets, comp, err, &holds);
+    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+    ctx->holds = holds;
+    ctx->raw.reset();
+    if (ctx->opt_open_end) ctx->raw = raw_of(s, ctx->batch);   // the raw arrays are what an append extends
+    return install_schedule(ctx, s, std::move(comp), false);
 } catch (const std::bad_alloc&) {
     return set_err(ctx, RFAST_ENOMEM, "host allocation failed");
 } catch (...) {
     return set_err(ctx, RFAST_EINVAL, "unexpected failure in rfast_load_schedule");
+}
+
+int rfast_append_schedule(rfast_ctx* ctx, const rfast_schedule* more) try {
+    if (!ctx) return RFAST_EINVAL;
+    if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
+    if (!ctx->opt_open_end || !ctx->raw)
+        return set_err(ctx, RFAST_ESTATE, "rounds can only be appended to a schedule loaded with RFAST_OPT_OPEN_END set");
+    CK(cudaStreamSynchronize(ctx->stream));
+    // the loaded rounds followed by the new ones, as one raw schedule
+    auto raw = std::make_unique<RawSchedule>(*ctx->raw);
+    if (const char* bad = append_raw(*raw, more, ctx->n, ctx->batch, ctx->alpha)) return set_err(ctx, RFAST_ESCHED, bad);
+    const rfast_schedule all = raw->view();
+    std::vector<int> holds = ctx->holds;                       // every earlier end stays a hold, the new end is open
+    if (holds.empty() || holds.back() != all.K) holds.push_back(all.K);
+    Compiled comp;
+    std::string err;
+    const bool one_pass = ctx->model == RFAST_MODEL_LOGISTIC_SPARSE && ctx->opt_fused && ctx->fused_cluster > 0;
+    int rc = compile_schedule(ctx->R, ctx->Cg, &all, ctx->batch, ctx->rows, traffic_of(ctx->model, ctx->compensated, one_pass), ctx->buckets, comp, err, &holds);
+    if (rc != RFAST_OK) return set_err(ctx, rc, err);
+    // nothing of the rounds already loaded may have moved: same rows, same descriptors
+    if (!prefix_same(ctx->comp, comp))
+        return set_err(ctx, RFAST_ESCHED, "internal: appending rounds would move a version row of the rounds already loaded");
+    const int round = ctx->round;
+    ctx->holds = holds;
+    ctx->raw = std::move(raw);
+    rc = install_schedule(ctx, &all, std::move(comp), true);
+    if (rc != RFAST_OK) return rc;
+    ctx->round = round;
+    return RFAST_OK;
+} catch (const std::bad_alloc&) {
+    return set_err(ctx, RFAST_ENOMEM, "host allocation failed");
+} catch (...) {
+    return set_err(ctx, RFAST_EINVAL, "unexpected failure in rfast_append_schedule");
 }
 
 int rfast_reset(rfast_ctx* ctx) {
@@ -823,6 +974,10 @@ int rfast_set_option(rfast_ctx* ctx, int option, int64_t value) {
                 if (value != 0) return set_err(ctx, RFAST_EINVAL, "the problem does not fit a cluster of that size");
             }
             return RFAST_OK;
+        case RFAST_OPT_OPEN_END:
+            if (ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "this option must be set before a schedule is loaded (the version rows follow it)");
+            if (value != 0 && ctx->buckets) return set_err(ctx, RFAST_EINVAL, "rounds can be appended to running sums only, not to mass buckets");
+            ctx->opt_open_end = value != 0; return RFAST_OK;
         case RFAST_OPT_PHANTOM_ARRIVALS:
             if (value < 0 || value > 1024) return set_err(ctx, RFAST_EINVAL, "phantom arrivals must be 0..1024");
             ctx->opt_phantom = value; return RFAST_OK;
@@ -1178,6 +1333,47 @@ int rfast_compile_host(const rfast_problem* prob, const rfast_schedule* s, int32
                        int32_t* used_tau_rho, int32_t* v_ver, int32_t* rho_ver, int64_t* counts,
                        char* errbuf, size_t err_len) {
     return compile_host_impl(prob, s, used_tau_v, used_tau_rho, v_ver, rho_ver, counts, nullptr, errbuf, err_len);
+}
+
+int rfast_compile_append_check(const rfast_problem* prob, const rfast_schedule* first, const rfast_schedule* more,
+                               int64_t* counts, char* errbuf, size_t err_len) try {
+    std::string err;
+    auto done = [&](int rc) {
+        if (errbuf && err_len) { std::snprintf(errbuf, err_len, "%s", err.c_str()); }
+        return rc;
+    };
+    if (!prob || prob->n <= 0) { err = "problem is null or n <= 0"; return done(RFAST_EINVAL); }
+    HostGraph R, C;
+    int rc;
+    if ((rc = build_host_graph(prob->G_R, prob->n, true, R, err)) != RFAST_OK) return done(rc);
+    if ((rc = build_host_graph(prob->G_C, prob->n, false, C, err)) != RFAST_OK) return done(rc);
+    if ((rc = check_roots(R, C, prob->root, err)) != RFAST_OK) return done(rc);
+    const ModelTraffic mt = traffic_of(prob->model, prob->compensated != 0);
+    const bool buckets = prob->tracker == RFAST_TRACKER_BUCKETS;
+    Compiled c1, c2, whole;
+    std::vector<int> holds;
+    if (first && first->K >= 0) holds.push_back(first->K);
+    if ((rc = compile_schedule(R, C, first, prob->batch, prob->rows, mt, buckets, c1, err, &holds)) != RFAST_OK) return done(rc);
+    auto raw = raw_of(first, prob->batch);
+    if (const char* bad = append_raw(*raw, more, prob->n, prob->batch, prob->alpha)) { err = bad; return done(RFAST_ESCHED); }
+    const rfast_schedule all = raw->view();
+    if (holds.back() != all.K) holds.push_back(all.K);
+    if ((rc = compile_schedule(R, C, &all, prob->batch, prob->rows, mt, buckets, c2, err, &holds)) != RFAST_OK) return done(rc);
+    if (!prefix_same(c1, c2)) { err = "appending rounds moved a version row of the rounds already loaded"; return done(RFAST_ESCHED); }
+    // the stamps consumed are those of the whole schedule compiled at once
+    if ((rc = compile_schedule(R, C, &all, prob->batch, prob->rows, mt, buckets, whole, err)) != RFAST_OK) return done(rc);
+    if (whole.used_tau_v != c2.used_tau_v || whole.used_tau_rho != c2.used_tau_rho || whole.t_end != c2.t_end) {
+        err = "the appended schedule consumes other stamps than the whole schedule compiled at once";
+        return done(RFAST_ESCHED);
+    }
+    if (counts) {
+        counts[0] = c1.n_v_slots; counts[1] = c1.n_rho_slots; counts[2] = c2.n_v_slots; counts[3] = c2.n_rho_slots;
+        counts[4] = whole.n_v_slots; counts[5] = whole.n_rho_slots;
+    }
+    return done(RFAST_OK);
+} catch (const std::bad_alloc&) {
+    if (errbuf && err_len) std::snprintf(errbuf, err_len, "host allocation failed");
+    return RFAST_ENOMEM;
 }
 
 int rfast_compile_digest(const rfast_problem* prob, const rfast_schedule* s, uint64_t* digest, char* errbuf, size_t err_len) {

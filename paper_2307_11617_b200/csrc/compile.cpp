@@ -156,10 +156,17 @@ inline int deliver(PendQ& q, int r, int tau) {
 }  // namespace
 
 int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedule* s, int batch,
-                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err) {
+                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err,
+                     const std::vector<int>* holds) {
     const int n = R.n;
     if (!s || s->K < 0 || !s->act_ptr) return fail(err, RFAST_ESCHED, "schedule: null or K < 0");
     const int K = s->K;
+    if (holds && !holds->empty()) {
+        if (buckets) return fail(err, RFAST_ESCHED, "schedule: rounds can be appended to running sums only, not to mass buckets");
+        for (size_t k = 0; k < holds->size(); ++k)
+            if ((*holds)[k] < 0 || (*holds)[k] > K || (k && (*holds)[k] <= (*holds)[k - 1]))
+                return fail(err, RFAST_ESCHED, "schedule: hold rounds must ascend inside 0 .. K");
+    }
     if (s->act_ptr[0] != 0) return fail(err, RFAST_ESCHED, "schedule: act_ptr[0] != 0");
     for (int r = 0; r < K; ++r)
         if (s->act_ptr[r + 1] < s->act_ptr[r])
@@ -226,7 +233,40 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     c.rho_write.assign(nRho, 0);
     std::vector<int> rho_last_sender(nRho, 0), rho_last_recv(nRho, -1);
     if (buckets) c.rho_leader.assign(nRho, -1);
+    // A hold at round b: whatever an activation in round b or later may still read stays in its
+    // row through round b -- per edge the version its receiver holds and every packet still on
+    // its way or waiting, and every sender's latest running sums.  The rows of the rounds before
+    // b then do not depend on what follows b: rounds can be appended without moving any of them.
+    auto for_pending = [](const PendQ& q, auto&& f) {
+        if (q.more) { for (const Pend& pk : *q.more) f(pk); }
+        else for (int k = 0; k < q.n; ++k) f(q.a[k]);
+    };
+    auto hold = [&](int b) {
+        for (int e = 0; e < R.E; ++e) {
+            const auto& evs = ev_of[R.col[e]];
+            if (tau_v[e] >= 1) c.v_last[evs[tau_v[e] - 1]] = std::max(c.v_last[evs[tau_v[e] - 1]], b);
+            for_pending(pend_v[e], [&](const Pend& pk) {
+                if (pk.stamp > tau_v[e]) c.v_last[evs[pk.stamp - 1]] = std::max(c.v_last[evs[pk.stamp - 1]], b);
+            });
+        }
+        for (int e = 0; e < C.E; ++e) {
+            const auto& evs = ev_of[C.col[e]];
+            auto keep = [&](int stamp) {
+                int64_t vid = c.out_c_off[evs[stamp - 1]] + C.opos[e];
+                rho_last_recv[vid] = std::max(rho_last_recv[vid], b);
+            };
+            if (tau_rho[e] >= 1) keep(tau_rho[e]);
+            for_pending(pend_c[e], [&](const Pend& pk) { if (pk.stamp > tau_rho[e]) keep(pk.stamp); });
+        }
+        for (int i = 0; i < n; ++i)
+            if (t[i] >= 1) {
+                int64_t base = c.out_c_off[ev_of[i][t[i] - 1]];
+                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = std::max(rho_last_sender[base + k], b);
+            }
+    };
+    size_t next_hold = 0;
     for (int r = 0; r < K; ++r) {
+        if (holds && next_hold < holds->size() && (*holds)[next_hold] == r) { hold(r); ++next_hold; }
         for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
             const int i = c.act_node[ev];
             for (int e = R.rowptr[i]; e < R.rowptr[i + 1]; ++e) {
@@ -283,6 +323,7 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
             }
         }
     }
+    if (holds && next_hold < holds->size() && (*holds)[next_hold] == K) hold(K);   // open end: more rounds may follow
     c.tau_v_end = tau_v;
     c.tau_rho_end = tau_rho;
     c.t_end = t;

@@ -88,7 +88,11 @@ struct ModelTraffic {
 
 int build_host_graph(const rfast_graph& g, int n, bool row_stochastic, HostGraph& out, std::string& err);
 int check_roots(const HostGraph& R, const HostGraph& C, int root, std::string& err);
+// holds (optional): ascending rounds b in 0 .. K at which everything a later activation may still
+// read is kept in its row through round b (b = K: the schedule is open-ended).  The rows of the
+// rounds before a hold do not depend on the rounds after it.
 int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedule* s, int batch,
-                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err);
+                     int rows, const ModelTraffic& mt, bool buckets, Compiled& out, std::string& err,
+                     const std::vector<int>* holds = nullptr);
 
 }  // namespace rfast

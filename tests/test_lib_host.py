@@ -246,3 +246,43 @@ def test_threaded_descriptor_pass_equals_the_single_threaded_one(rfast_lib, monk
     # and the digest does see a difference: another schedule, another number
     other = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, 2400, 0.5, rng), 0.2, 4, rng, batch=0)
     assert pkg.rfast_compile_digest(wl, other) != many
+
+
+@pytest.mark.parametrize("name,ov", CASES)
+def test_appended_rounds_move_no_row_and_consume_the_same_stamps(rfast_lib, name, ov):
+    """Rounds handed over a piece at a time (Algorithm 2 goes on counting k): compiled open-ended
+    and then extended, the rounds of the first piece keep every version row, row list and event
+    descriptor, and the stamps consumed are those of the whole schedule compiled in one piece."""
+    import paper_2307_11617_b200 as pkg
+    from workloads import split_schedule
+    wl = build_config(name, seed=11, **ov)
+    s = wl.schedule
+    for cut in sorted({1, s.K // 3, s.K // 2, s.K - 1} - {0, s.K}):
+        first, more = split_schedule(s, wl.G_R, wl.G_C, [cut])
+        assert first.K + more.K == s.K and first.n_events + more.n_events == s.n_events
+        r = pkg.rfast_compile_append_check(wl, first, more)
+        # an open end keeps more alive than a closed one; the pools only ever grow
+        assert r["appended"][0] >= r["first"][0] and r["appended"][1] >= r["first"][1]
+        assert r["appended"][0] >= r["whole"][0] and r["appended"][1] >= r["whole"][1]
+
+
+def test_append_check_rejects_inconsistent_parts(rfast_lib):
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200.binding import ESCHED, RFastError
+    from workloads import split_schedule
+    wl = build_config("ls_ring4", seed=1)
+    first, more = split_schedule(wl.schedule, wl.G_R, wl.G_C, [50])
+    bad = copy.copy(more)
+    bad.send_c = more.send_c[:-1]
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_append_check(wl, first, bad)
+    assert ei.value.code == ESCHED
+    bad = copy.copy(more)
+    bad.act_ptr = more.act_ptr + 1
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_append_check(wl, first, bad)
+    assert ei.value.code == ESCHED
+    wlb = build_config("ls_ring4", seed=1, tracker=1)     # mass buckets: no appending
+    with pytest.raises(RFastError) as ei:
+        pkg.rfast_compile_append_check(wlb, first, more)
+    assert ei.value.code == ESCHED

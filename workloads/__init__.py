@@ -11,7 +11,7 @@ path never import each other.
 from .graphs import (Graph, graph_from_edges, ring_graphs, tree_graphs,
                      binary_tree_parents, exponential_tree_parents,
                      random_tree_parents, sender_csr)
-from .schedules import (Schedule, make_schedule, make_schedule_ack_gated, activation_bernoulli,
+from .schedules import (Schedule, make_schedule, make_schedule_ack_gated, split_schedule, activation_bernoulli,
                         activation_uniform_subset, activation_durations,
                         activation_all, realised_T_D)
 from .configs import CONFIG_NAMES, build_config, shard_coordinates, Workload
@@ -19,7 +19,7 @@ from .configs import CONFIG_NAMES, build_config, shard_coordinates, Workload
 __all__ = [
     "Graph", "graph_from_edges", "ring_graphs", "tree_graphs",
     "binary_tree_parents", "exponential_tree_parents", "random_tree_parents",
-    "sender_csr", "Schedule", "make_schedule", "make_schedule_ack_gated", "activation_bernoulli",
+    "sender_csr", "Schedule", "make_schedule", "make_schedule_ack_gated", "split_schedule", "activation_bernoulli",
     "activation_uniform_subset", "activation_durations", "activation_all",
     "realised_T_D", "CONFIG_NAMES", "build_config", "shard_coordinates", "Workload",
 ]

@@ -104,6 +104,29 @@ def make_schedule(G_R: Graph, G_C: Graph, active_sets, drop: float, max_delay: i
     return Schedule(K, act_ptr, act_node, send_r, send_c, batch, batch_idx)
 
 
+def split_schedule(s: Schedule, G_R: Graph, G_C: Graph, cuts) -> list:
+    """The schedule cut into consecutive parts at the rounds `cuts` (ascending, inside 0..K), each
+    part numbered from its own round 0 and event 0, the way rounds are handed to an engine a
+    piece at a time.  Every part carries the initial samples (the first n*B entries of
+    batch_idx) in front of its own events' samples.  Array slicing only."""
+    n = G_R.n
+    outdeg_R = np.diff(sender_csr(G_R)[0]).astype(np.int64)
+    outdeg_C = np.diff(sender_csr(G_C)[0]).astype(np.int64)
+    off_r = np.concatenate([[0], np.cumsum(outdeg_R[s.act_node])]).astype(np.int64)
+    off_c = np.concatenate([[0], np.cumsum(outdeg_C[s.act_node])]).astype(np.int64)
+    bounds = [0] + [int(c) for c in cuts] + [int(s.K)]
+    parts = []
+    for r0, r1 in zip(bounds[:-1], bounds[1:]):
+        e0, e1 = int(s.act_ptr[r0]), int(s.act_ptr[r1])
+        lead = n * s.batch
+        bi = (np.concatenate([s.batch_idx[:lead], s.batch_idx[lead + e0 * s.batch: lead + e1 * s.batch]]).astype(np.int32)
+              if s.batch > 0 else np.zeros(0, np.int32))
+        parts.append(Schedule(r1 - r0, (s.act_ptr[r0:r1 + 1] - e0).astype(np.int32), s.act_node[e0:e1].copy(),
+                              s.send_r[off_r[e0]:off_r[e1]].copy(), s.send_c[off_c[e0]:off_c[e1]].copy(), s.batch, bi,
+                              None if s.alpha_round is None else s.alpha_round[r0:r1].copy()))
+    return parts
+
+
 def make_schedule_ack_gated(G_R: Graph, G_C: Graph, active_sets, max_delay: int,
                             rng: np.random.Generator, batch: int = 0, rows_per_node: int = 0) -> Schedule:
     """Packet loss as the paper emulates it (Section VI, first paragraph): a node sends a new
