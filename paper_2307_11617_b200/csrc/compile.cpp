@@ -515,6 +515,28 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
         for (int64_t bev : bad)
             if (bev >= 0) return fail(err, RFAST_ESCHED, "internal: consumed v version without a row (event %lld)", bev);
     }
+    // Every index a kernel will dereference is checked here, on the host, before anything is
+    // launched: rows inside their pools, list ranges inside their lists, node ids inside the state.
+    {
+        const int64_t n_mix = (int64_t)c.mix_slot.size(), n_news = (int64_t)c.news_new.size();
+        for (int64_t ev = 0; ev < nE; ++ev) {
+            const EvDesc& d = c.ev[ev];
+            bool good = d.node >= 0 && d.node < n && d.v_out >= -1 && d.v_out < c.n_v_slots &&
+                        d.mix_beg >= 0 && d.mix_cnt >= 0 && (int64_t)d.mix_beg + d.mix_cnt <= n_mix &&
+                        d.news_beg >= 0 && d.news_cnt >= 0 && (int64_t)d.news_beg + d.news_cnt <= n_news &&
+                        d.out_beg >= 0 && d.out_cnt >= 0 && (int64_t)d.out_beg + d.out_cnt <= nRho &&
+                        (d.g_par == 0 || d.g_par == 1) && d.sample >= n && (int64_t)d.sample < n + nE;
+            for (int m = 0; good && m < d.mix_cnt; ++m)
+                good = c.mix_slot[d.mix_beg + m] >= 0 && c.mix_slot[d.mix_beg + m] < c.n_v_slots;
+            for (int m = 0; good && m < d.news_cnt; ++m)
+                good = c.news_new[d.news_beg + m] >= 0 && c.news_new[d.news_beg + m] < c.n_rho_slots &&
+                       c.news_prev[d.news_beg + m] >= -1 && c.news_prev[d.news_beg + m] < c.n_rho_slots;
+            for (int m = 0; good && m < d.out_cnt; ++m)
+                good = c.out_new[d.out_beg + m] >= 0 && c.out_new[d.out_beg + m] < c.n_rho_slots &&
+                       c.out_cur[d.out_beg + m] >= -1 && c.out_cur[d.out_beg + m] < c.n_rho_slots;
+            if (!good) return fail(err, RFAST_ESCHED, "internal: descriptor of event %lld points outside its pools or lists", ev);
+        }
+    }
     for (int r = 0; r < K; ++r) {
         c.round_streams[r + 1] = c.round_streams[r] + round_s[r];
         c.round_streams_method[r + 1] = c.round_streams_method[r] + round_m[r];
