@@ -339,11 +339,11 @@ def rfast_checkpoint_load(handle, blob: np.ndarray) -> None:
 def rfast_diagnostics(handle) -> dict:
     """Consensus error, norm of the mean iterate, conservation residual (Lemma 3) and its scale,
     tracker norm, all computed on the device."""
-    out = np.zeros(7, dtype=np.float64)
-    _check(lib().rfast_diagnostics(handle, _ptr(out), 7), handle)
+    out = np.zeros(8, dtype=np.float64)
+    _check(lib().rfast_diagnostics(handle, _ptr(out), 8), handle)
     return {"consensus_error": out[0], "xbar_norm": out[1], "conservation_residual": out[2],
             "gradient_sum_max": out[3], "tracker_norm": out[4], "full_gradient_norm": out[5],
-            "merit": out[6]}
+            "merit": out[6], "objective": out[7]}
 
 
 STATIC_MAX_ROWS = 65536

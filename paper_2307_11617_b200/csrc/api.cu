@@ -1468,8 +1468,8 @@ int rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes) {
 }
 
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
-    if (!ctx || !out || (n_out != 5 && n_out != 7))
-        return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5 or 7") : RFAST_EINVAL;
+    if (!ctx || !out || (n_out != 5 && n_out != 7 && n_out != 8))
+        return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5, 7 or 8") : RFAST_EINVAL;
     if (!ctx->has_sched) return set_err(ctx, RFAST_ESTATE, "no schedule loaded");
     const Compiled& c = ctx->comp;
     const int n = ctx->n;
@@ -1495,7 +1495,7 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
         CK(cudaMemcpyAsync(d_latest, latest.data(), E * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
         CK(cudaMemcpyAsync(d_buf, buf.data(), E * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
     }
-    const bool want_mf = n_out == 7;
+    const bool want_mf = n_out >= 7;
     const bool ls = ctx->model == RFAST_MODEL_LEAST_SQUARES;
     k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
                                                           ctx->quad_b, ctx->rbuf, ctx->rlo_off(), d_latest, d_buf, n, E,
@@ -1511,18 +1511,19 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     std::vector<double> part((size_t)blocks * kDiagSlots);
     CK(cudaMemcpyAsync(part.data(), ctx->d_diag_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
     CK(cudaStreamSynchronize(ctx->stream));       // the host vectors above may go now
-    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0;
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0, fl = 0;
     for (int b = 0; b < blocks; ++b) {          // fixed order: the same bits on every run
         const double* q = part.data() + (size_t)b * kDiagSlots;
         cons += q[0]; xb2 += q[1];
         res = std::max(res, q[2]); gs = std::max(gs, q[3]);
-        z2 += q[4]; gf2 += q[5];
+        z2 += q[4]; gf2 += q[5]; fl += q[6];
     }
     out[0] = std::sqrt(std::max(cons, 0.0)); out[1] = std::sqrt(xb2); out[2] = res; out[3] = gs; out[4] = std::sqrt(z2);
     if (want_mf) {
         const bool have = ls || ctx->model == RFAST_MODEL_QUAD_DIAG;
         out[5] = have ? std::sqrt(gf2) : std::nan("");
         out[6] = have ? gf2 + std::max(cons, 0.0) : std::nan("");
+        if (n_out == 8) out[7] = have ? fl : std::nan("");
     }
     return RFAST_OK;
 } catch (...) {

@@ -749,10 +749,12 @@ k_logit_track(RoundArgs a, GradArgs g, const int64_t* __restrict__ range_ptr, in
 //   part[block][4] = sum_c sum_i z_ic^2
 //   part[block][5] = sum_c (grad F(xbar))_c^2 for the element-wise objective, where the full gradient
 //                    sum_i d_ic^2 (xbar_c - b_ic) is coordinate-wise; 0 otherwise
+//   part[block][6] = this block's share of F(xbar) = sum_i f_i(xbar) for the element-wise objective:
+//                    sum_c sum_i (d_ic (xbar_c - b_ic))^2 / 2; 0 otherwise
 // g_i is row gsel[i] of gpool (or recomputed for the element-wise objective when gpool is null).
 // xbar_out (may be null) receives the mean iterate in fp32.
 // grid = tiles of kThreads coordinates (scalar: diagnostics favour clarity over speed)
-constexpr int kDiagSlots = 6;
+constexpr int kDiagSlots = 7;
 __global__ void __launch_bounds__(kThreads)
 k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const float* __restrict__ zc,
               const float* __restrict__ gpool, const int* __restrict__ gsel,
@@ -762,7 +764,7 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
               float* __restrict__ xbar_out, double* __restrict__ part) {
     __shared__ double red[kDiagSlots][kThreads];
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0;
+    double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0, fl = 0;
     if (c < p) {
         double sx = 0, sx2 = 0, sz = 0, sg = 0;
         for (int i = 0; i < n; ++i) {
@@ -795,13 +797,15 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
             double gf = 0;
             for (int i = 0; i < n; ++i) {
                 const double d = qd[(int64_t)i * stride + c];
-                gf += d * d * (xbar - (double)qb[(int64_t)i * stride + c]);
+                const double r = d * (xbar - (double)qb[(int64_t)i * stride + c]);
+                gf += d * r;
+                fl += 0.5 * r * r;
             }
             gf2 = gf * gf;
         }
     }
     red[0][threadIdx.x] = cons; red[1][threadIdx.x] = xb2; red[2][threadIdx.x] = res;
-    red[3][threadIdx.x] = gs; red[4][threadIdx.x] = z2; red[5][threadIdx.x] = gf2;
+    red[3][threadIdx.x] = gs; red[4][threadIdx.x] = z2; red[5][threadIdx.x] = gf2; red[6][threadIdx.x] = fl;
     __syncthreads();
     for (int s = kThreads / 2; s > 0; s >>= 1) {
         if (threadIdx.x < s) {
@@ -811,6 +815,7 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
             red[3][threadIdx.x] = fmax(red[3][threadIdx.x], red[3][threadIdx.x + s]);
             red[4][threadIdx.x] += red[4][threadIdx.x + s];
             red[5][threadIdx.x] += red[5][threadIdx.x + s];
+            red[6][threadIdx.x] += red[6][threadIdx.x + s];
         }
         __syncthreads();
     }
@@ -832,14 +837,17 @@ k_diag_ls_residual(const float* __restrict__ feat, const float* __restrict__ tar
     if (lane == 0) res[r] = s - target[r];
 }
 // ... then (grad F(xbar))_c = sum_i [ (1/rows) sum_k a_ik[c] r_ik + l2 xbar_c ], squared and summed
-// per block into part[block][5].  grid = tiles of kThreads coordinates
+// per block into part[block][5]; the block's share of F(xbar) = sum_i [ sum_k r_ik^2 / (2 rows) +
+// l2 |xbar|^2 / 2 ] into part[block][6].  grid = tiles of kThreads coordinates
 __global__ void __launch_bounds__(kThreads)
 k_diag_ls_grad(const float* __restrict__ feat, const float* __restrict__ xbar, const float* __restrict__ res,
                int n, int rows, int F, float l2, double* __restrict__ part) {
-    __shared__ double red[kThreads];
+    __shared__ double red[kThreads], redf[kThreads];
     const int c = blockIdx.x * kThreads + threadIdx.x;
-    double gf = 0;
+    double gf = 0, fl = 0;
+    for (int64_t r = c; r < (int64_t)n * rows; r += (int64_t)gridDim.x * kThreads) fl += 0.5 * (double)res[r] * (double)res[r] / rows;
     if (c < F) {
+        fl += 0.5 * n * (double)l2 * (double)xbar[c] * (double)xbar[c];
         for (int i = 0; i < n; ++i) {
             double s = 0;
             for (int k = 0; k < rows; ++k) {
@@ -850,12 +858,16 @@ k_diag_ls_grad(const float* __restrict__ feat, const float* __restrict__ xbar, c
         }
     }
     red[threadIdx.x] = gf * gf;
+    redf[threadIdx.x] = fl;
     __syncthreads();
     for (int s = kThreads / 2; s > 0; s >>= 1) {
-        if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        if (threadIdx.x < s) { red[threadIdx.x] += red[threadIdx.x + s]; redf[threadIdx.x] += redf[threadIdx.x + s]; }
         __syncthreads();
     }
-    if (threadIdx.x == 0) part[(int64_t)blockIdx.x * kDiagSlots + 5] = red[0];
+    if (threadIdx.x == 0) {
+        part[(int64_t)blockIdx.x * kDiagSlots + 5] = red[0];
+        part[(int64_t)blockIdx.x * kDiagSlots + 6] = redf[0];
+    }
 }
 
 // bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)
