@@ -361,12 +361,17 @@ int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
  *   out[3] max_c | sum_i g_i |   (the scale of out[2])
  *   out[4] || z ||_F
  *   out[5] || grad F(xbar) ||_2, the full gradient of F = sum_i f_i (every row of every shard,
- *          no sampling) at the mean iterate; computed for the element-wise and the least-squares
- *          objective, NaN for the others
+ *          no sampling) at the mean iterate.  For the objectives that sample minibatches
+ *          (softmax, MLP, sparse logistic) it is formed with the kernels the activations use,
+ *          the shards walked in chunks of B rows from a state whose rows all hold xbar; x is
+ *          moved aside and put back bit for bit, the first such call allocates its scratch (a
+ *          copy of x, a double per coordinate) and keeps it while the schedule stays loaded.
+ *          NaN where the shard size is not a multiple of B
  *   out[6] the merit function of the non-convex analysis (Section V-B),
- *          M_F(x) = || grad F(xbar) ||^2 + || x - 1 xbar^T ||^2 = out[5]^2 + out[0]^2 (NaN likewise)
+ *          M_F(x) = || grad F(xbar) ||^2 + || x - 1 xbar^T ||^2 = out[5]^2 + out[0]^2 (NaN where out[5] is)
  *   out[7] F(xbar) = sum_i f_i(xbar), the objective of eq. (1) at the mean iterate over every row
- *          of every shard (the loss curve of the experiments in Section VI; NaN likewise)
+ *          of every shard (the loss curve of the experiments in Section VI); the element-wise and
+ *          the least-squares objective only, NaN for the others
  * n_out is 5 (the first five only), 7 or 8; RFAST_EINVAL otherwise.  out is a caller-owned HOST
  * array of doubles. */
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out);

@@ -137,6 +137,9 @@ struct rfast_ctx {
     int* d_diag_idx = nullptr;  int64_t diag_idx_cap = 0;
     double* d_diag_part = nullptr;
     float* d_xbar = nullptr;  float* d_diag_res = nullptr;
+    // sampled objectives, full gradient at the mean iterate (allocated at the first call that asks
+    // for it): a copy of x, a double per coordinate, descriptors and a batch table over whole shards
+    float* d_diag_x = nullptr;  double* d_diag_acc = nullptr;  EvDesc* d_diag_ev = nullptr;  int* d_diag_bidx = nullptr;
     MlpPlan* mlp = nullptr;
     // compiled schedule
     bool has_sched = false;
@@ -230,6 +233,7 @@ void free_schedule(rfast_ctx* c) {
     c->d_ev = c->d_init_ev = nullptr;
     c->vbuf = c->rbuf = c->scratch = nullptr;
     c->d_diag_idx = nullptr; c->d_diag_part = nullptr; c->d_xbar = nullptr; c->d_diag_res = nullptr;
+    c->d_diag_x = nullptr; c->d_diag_acc = nullptr; c->d_diag_ev = nullptr; c->d_diag_bidx = nullptr;
     c->d_act_ptr = nullptr; c->d_alpha_round = nullptr; c->d_bar = nullptr; c->d_pstatus = nullptr;
     c->persist_ok = false;
     c->has_sched = false;
@@ -1467,6 +1471,74 @@ int rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes) {
     return RFAST_OK;
 }
 
+// Full gradient of F = sum_i f_i at the mean iterate for the objectives that sample minibatches,
+// out of the very kernels the activations use: the shard of every node is walked in chunks of B
+// rows (a minibatch that is rows [cB, (c+1)B) of the shard), all nodes at once, from a state whose
+// rows all hold xbar; the mean over the chunks of a node's minibatch gradients is its full
+// gradient (the L2 term is in each of them).  x (and its bf16 copy) is moved aside and put back,
+// bit for bit; the gradients land in the rows of the gradient pool that hold no remembered
+// gradient.  Leaves sum_c (grad F(xbar))_c^2 per block in part[block][5].
+static int sampled_full_gradient(rfast_ctx* ctx, const RoundView& rv, int blocks) {
+    const int n = ctx->n, B = ctx->batch, chunks = ctx->rows / B;
+    const size_t plane = (size_t)n * ctx->stride;
+    const int n4 = (int)(ctx->stride / 4);
+    if (!ctx->d_diag_x) {
+        CK(dev_alloc(ctx, &ctx->d_diag_x, plane, true));
+        CK(dev_alloc(ctx, &ctx->d_diag_acc, (size_t)ctx->stride, true));
+        CK(dev_alloc(ctx, &ctx->d_diag_ev, (size_t)chunks * n, true));
+        CK(dev_alloc(ctx, &ctx->d_diag_bidx, (size_t)chunks * n * B, true));
+        if (!ctx->d_xbar) {
+            CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
+            CK(cudaMemsetAsync(ctx->d_xbar, 0, ctx->stride * sizeof(float), ctx->stream));
+        }
+        std::vector<int> bidx((size_t)chunks * n * B);
+        for (int c = 0; c < chunks; ++c)
+            for (int i = 0; i < n; ++i)
+                for (int k = 0; k < B; ++k) bidx[((size_t)c * n + i) * B + k] = c * B + k;
+        CK(cudaMemcpy(ctx->d_diag_bidx, bidx.data(), bidx.size() * sizeof(int), cudaMemcpyHostToDevice));
+    }
+    std::vector<EvDesc> evs((size_t)chunks * n);
+    std::vector<int> sel(n);
+    for (int i = 0; i < n; ++i) sel[i] = ((rv.t[i] & 1) ^ 1) * n + i;          // the row that holds no remembered gradient
+    for (int c = 0; c < chunks; ++c)
+        for (int i = 0; i < n; ++i) {
+            EvDesc d{};
+            d.node = i; d.v_out = -1; d.g_par = rv.t[i] & 1; d.sample = c * n + i;
+            evs[(size_t)c * n + i] = d;
+        }
+    CK(cudaMemcpy(ctx->d_diag_ev, evs.data(), evs.size() * sizeof(EvDesc), cudaMemcpyHostToDevice));
+    int* d_sel = ctx->d_diag_idx;                                                // n ints, free again by now
+    CK(cudaMemcpyAsync(d_sel, sel.data(), n * sizeof(int), cudaMemcpyHostToDevice, ctx->stream));
+    CK(cudaMemcpyAsync(ctx->d_diag_x, ctx->x, plane * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+    k_diag_fill_rows<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(ctx->x, ctx->d_xbar, ctx->stride, n4);
+    if (ctx->xb) k_rows_to_bf16<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(ctx->x, ctx->xb, ctx->stride, n4);
+    CK(cudaMemsetAsync(ctx->d_diag_acc, 0, ctx->stride * sizeof(double), ctx->stream));
+    int* const sched_bidx = ctx->d_batch_idx;
+    const int64_t launches = ctx->launches;                                      // counts what rfast_run launches only
+    ctx->d_batch_idx = ctx->d_diag_bidx;
+    int rc = RFAST_OK;
+    for (int c = 0; c < chunks && rc == RFAST_OK; ++c) {
+        const EvDesc* ev = ctx->d_diag_ev + (size_t)c * n;
+        rc = launch_gradients(ctx, ev, n);
+        if (rc == RFAST_OK && ctx->model == RFAST_MODEL_LOGISTIC_SPARSE) {
+            RoundArgs a{};
+            a.stride = ctx->stride; a.n4 = n4;
+            rc = launch_logit_track(ctx, a, ev, n, 1);
+        }
+        if (rc == RFAST_OK)
+            k_diag_accumulate<<<blocks, kThreads, 0, ctx->stream>>>(ctx->gbuf, d_sel, n, ctx->stride, ctx->p, ctx->d_diag_acc);
+    }
+    ctx->d_batch_idx = sched_bidx;
+    ctx->launches = launches;
+    // x back in place whatever happened above
+    cudaMemcpyAsync(ctx->x, ctx->d_diag_x, plane * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream);
+    if (ctx->xb) k_rows_to_bf16<<<dim3((n4 + kThreads - 1) / kThreads, n), kThreads, 0, ctx->stream>>>(ctx->x, ctx->xb, ctx->stride, n4);
+    if (rc != RFAST_OK) return rc;
+    k_diag_norm2<<<blocks, kThreads, 0, ctx->stream>>>(ctx->d_diag_acc, ctx->p, 1.0 / chunks, ctx->d_diag_part);
+    CK(cudaGetLastError());
+    return RFAST_OK;
+}
+
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     if (!ctx || !out || (n_out != 5 && n_out != 7 && n_out != 8))
         return ctx ? set_err(ctx, RFAST_EINVAL, "diagnostics: n_out must be 5, 7 or 8") : RFAST_EINVAL;
@@ -1497,9 +1569,15 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     }
     const bool want_mf = n_out >= 7;
     const bool ls = ctx->model == RFAST_MODEL_LEAST_SQUARES;
+    const bool sampled = want_mf && ctx->batch > 0 && ctx->rows % ctx->batch == 0 &&
+                         (ctx->model == RFAST_MODEL_SOFTMAX || ctx->model == RFAST_MODEL_MLP || ctx->model == RFAST_MODEL_LOGISTIC_SPARSE);
+    if (sampled && !ctx->d_xbar) {                     // the mean iterate is wanted on the device
+        CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
+        CK(cudaMemsetAsync(ctx->d_xbar, 0, ctx->stride * sizeof(float), ctx->stream));
+    }
     k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
                                                           ctx->quad_b, ctx->rbuf, ctx->rlo_off(), d_latest, d_buf, n, E,
-                                                          ctx->stride, ctx->p, want_mf && ls ? ctx->d_xbar : nullptr,
+                                                          ctx->stride, ctx->p, want_mf && (ls || sampled) ? ctx->d_xbar : nullptr,
                                                           ctx->d_diag_part);
     if (want_mf && ls) {
         k_diag_ls_residual<<<dim3((ctx->rows + 7) / 8, n), 256, 0, ctx->stream>>>(ctx->feat, ctx->target, ctx->d_xbar,
@@ -1508,6 +1586,10 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
                                                                ctx->F, ctx->l2, ctx->d_diag_part);
     }
     CK(cudaGetLastError());
+    if (sampled) {
+        int rc = sampled_full_gradient(ctx, rv, blocks);
+        if (rc != RFAST_OK) return rc;
+    }
     std::vector<double> part((size_t)blocks * kDiagSlots);
     CK(cudaMemcpyAsync(part.data(), ctx->d_diag_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
     CK(cudaStreamSynchronize(ctx->stream));       // the host vectors above may go now
@@ -1520,10 +1602,10 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     }
     out[0] = std::sqrt(std::max(cons, 0.0)); out[1] = std::sqrt(xb2); out[2] = res; out[3] = gs; out[4] = std::sqrt(z2);
     if (want_mf) {
-        const bool have = ls || ctx->model == RFAST_MODEL_QUAD_DIAG;
+        const bool have = ls || sampled || ctx->model == RFAST_MODEL_QUAD_DIAG;
         out[5] = have ? std::sqrt(gf2) : std::nan("");
         out[6] = have ? gf2 + std::max(cons, 0.0) : std::nan("");
-        if (n_out == 8) out[7] = have ? fl : std::nan("");
+        if (n_out == 8) out[7] = have && !sampled ? fl : std::nan("");
     }
     return RFAST_OK;
 } catch (...) {

@@ -870,6 +870,39 @@ k_diag_ls_grad(const float* __restrict__ feat, const float* __restrict__ xbar, c
     }
 }
 
+// Full gradient at the mean iterate for the sampled objectives, out of the minibatch kernels:
+// every row of the state := xbar (grid = (tiles, n)) ...
+__global__ void __launch_bounds__(kThreads)
+k_diag_fill_rows(float* __restrict__ x, const float* __restrict__ xbar, int64_t stride, int n4) {
+    const int i4 = blockIdx.x * kThreads + threadIdx.x;
+    if (i4 >= n4) return;
+    reinterpret_cast<float4*>(x + (int64_t)blockIdx.y * stride)[i4] = reinterpret_cast<const float4*>(xbar)[i4];
+}
+// ... acc_c += sum_i (row sel[i] of the gradient pool)_c after each chunk of shard rows ...
+__global__ void __launch_bounds__(kThreads)
+k_diag_accumulate(const float* __restrict__ gpool, const int* __restrict__ sel, int n, int64_t stride, int64_t p,
+                  double* __restrict__ acc) {
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= p) return;
+    double s = 0;
+    for (int i = 0; i < n; ++i) s += (double)gpool[(int64_t)sel[i] * stride + c];
+    acc[c] += s;
+}
+// ... and part[block][5] = sum_c (acc_c / chunks)^2 (the mean over the chunks is the full-shard gradient)
+__global__ void __launch_bounds__(kThreads)
+k_diag_norm2(const double* __restrict__ acc, int64_t p, double inv_chunks, double* __restrict__ part) {
+    __shared__ double red[kThreads];
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const double v = c < p ? acc[c] * inv_chunks : 0.0;
+    red[threadIdx.x] = v * v;
+    __syncthreads();
+    for (int s = kThreads / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) part[(int64_t)blockIdx.x * kDiagSlots + 5] = red[0];
+}
+
 // bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)
 __global__ void __launch_bounds__(kThreads)
 k_rows_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int n4) {
