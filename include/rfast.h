@@ -370,8 +370,8 @@ int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
  *   out[6] the merit function of the non-convex analysis (Section V-B),
  *          M_F(x) = || grad F(xbar) ||^2 + || x - 1 xbar^T ||^2 = out[5]^2 + out[0]^2 (NaN where out[5] is)
  *   out[7] F(xbar) = sum_i f_i(xbar), the objective of eq. (1) at the mean iterate over every row
- *          of every shard (the loss curve of the experiments in Section VI); the element-wise and
- *          the least-squares objective only, NaN for the others
+ *          of every shard (the loss curve of the experiments in Section VI); NaN for a softmax
+ *          objective with more than 32 classes
  * n_out is 5 (the first five only), 7 or 8; RFAST_EINVAL otherwise.  out is a caller-owned HOST
  * array of doubles. */
 int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out);

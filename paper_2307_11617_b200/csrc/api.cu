@@ -139,6 +139,7 @@ struct rfast_ctx {
     float* d_xbar = nullptr;  float* d_diag_res = nullptr;
     // sampled objectives, full gradient at the mean iterate (allocated at the first call that asks
     // for it): a copy of x, a double per coordinate, descriptors and a batch table over whole shards
+    double* d_diag_rowloss = nullptr;
     float* d_diag_x = nullptr;  double* d_diag_acc = nullptr;  EvDesc* d_diag_ev = nullptr;  int* d_diag_bidx = nullptr;
     MlpPlan* mlp = nullptr;
     // compiled schedule
@@ -233,6 +234,7 @@ void free_schedule(rfast_ctx* c) {
     c->d_ev = c->d_init_ev = nullptr;
     c->vbuf = c->rbuf = c->scratch = nullptr;
     c->d_diag_idx = nullptr; c->d_diag_part = nullptr; c->d_xbar = nullptr; c->d_diag_res = nullptr;
+    c->d_diag_rowloss = nullptr;
     c->d_diag_x = nullptr; c->d_diag_acc = nullptr; c->d_diag_ev = nullptr; c->d_diag_bidx = nullptr;
     c->d_act_ptr = nullptr; c->d_alpha_round = nullptr; c->d_bar = nullptr; c->d_pstatus = nullptr;
     c->persist_ok = false;
@@ -1571,13 +1573,16 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     const bool ls = ctx->model == RFAST_MODEL_LEAST_SQUARES;
     const bool sampled = want_mf && ctx->batch > 0 && ctx->rows % ctx->batch == 0 &&
                          (ctx->model == RFAST_MODEL_SOFTMAX || ctx->model == RFAST_MODEL_MLP || ctx->model == RFAST_MODEL_LOGISTIC_SPARSE);
-    if (sampled && !ctx->d_xbar) {                     // the mean iterate is wanted on the device
+    const bool sampled_model = ctx->model == RFAST_MODEL_SOFTMAX || ctx->model == RFAST_MODEL_MLP || ctx->model == RFAST_MODEL_LOGISTIC_SPARSE;
+    const bool lossy = n_out == 8 && sampled_model && (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE || ctx->C <= 32);
+    if (lossy && !ctx->d_diag_rowloss) CK(dev_alloc(ctx, &ctx->d_diag_rowloss, (size_t)n * ctx->rows, true));
+    if ((sampled || lossy) && !ctx->d_xbar) {          // the mean iterate is wanted on the device
         CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
         CK(cudaMemsetAsync(ctx->d_xbar, 0, ctx->stride * sizeof(float), ctx->stream));
     }
     k_diagnostics<<<blocks, kThreads, 0, ctx->stream>>>(ctx->x, ctx->z, ctx->zc, ctx->gbuf, d_gsel, ctx->quad_d,
                                                           ctx->quad_b, ctx->rbuf, ctx->rlo_off(), d_latest, d_buf, n, E,
-                                                          ctx->stride, ctx->p, want_mf && (ls || sampled) ? ctx->d_xbar : nullptr,
+                                                          ctx->stride, ctx->p, want_mf && (ls || sampled || lossy) ? ctx->d_xbar : nullptr,
                                                           ctx->d_diag_part);
     if (want_mf && ls) {
         k_diag_ls_residual<<<dim3((ctx->rows + 7) / 8, n), 256, 0, ctx->stream>>>(ctx->feat, ctx->target, ctx->d_xbar,
@@ -1589,6 +1594,20 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
     if (sampled) {
         int rc = sampled_full_gradient(ctx, rv, blocks);
         if (rc != RFAST_OK) return rc;
+    }
+    std::vector<double> rowloss;
+    if (lossy) {                                           // F(xbar): every row of every shard, a warp per row
+        const dim3 grid((ctx->rows + 7) / 8, n);
+        if (ctx->model == RFAST_MODEL_SOFTMAX)
+            k_diag_loss_softmax<<<grid, 256, 0, ctx->stream>>>(ctx->feat, ctx->label, ctx->d_xbar, ctx->d_diag_rowloss, ctx->rows, ctx->F, ctx->C);
+        else if (ctx->model == RFAST_MODEL_MLP)
+            k_diag_loss_mlp<<<grid, 256, 8 * (size_t)ctx->H * sizeof(double), ctx->stream>>>(ctx->feat, ctx->label, ctx->d_xbar, ctx->d_diag_rowloss,
+                                                                                             ctx->rows, ctx->F, ctx->H, ctx->C);
+        else
+            k_diag_loss_logistic<<<grid, 256, 0, ctx->stream>>>(ctx->sp_ptr, ctx->sp_col, ctx->sp_val, ctx->label, ctx->d_xbar, ctx->d_diag_rowloss, ctx->rows);
+        CK(cudaGetLastError());
+        rowloss.resize((size_t)n * ctx->rows);
+        CK(cudaMemcpyAsync(rowloss.data(), ctx->d_diag_rowloss, rowloss.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
     }
     std::vector<double> part((size_t)blocks * kDiagSlots);
     CK(cudaMemcpyAsync(part.data(), ctx->d_diag_part, part.size() * sizeof(double), cudaMemcpyDeviceToHost, ctx->stream));
@@ -1605,7 +1624,18 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
         const bool have = ls || sampled || ctx->model == RFAST_MODEL_QUAD_DIAG;
         out[5] = have ? std::sqrt(gf2) : std::nan("");
         out[6] = have ? gf2 + std::max(cons, 0.0) : std::nan("");
-        if (n_out == 8) out[7] = have && !sampled ? fl : std::nan("");
+        if (n_out == 8) {
+            out[7] = have && !sampled_model ? fl : std::nan("");
+            if (lossy) {                                   // mean loss per shard + the L2 term of every node, fixed order
+                double tot = 0;
+                for (int i = 0; i < n; ++i) {
+                    double si = 0;
+                    for (int k = 0; k < ctx->rows; ++k) si += rowloss[(size_t)i * ctx->rows + k];
+                    tot += si / ctx->rows;
+                }
+                out[7] = tot + 0.5 * n * (double)ctx->l2 * xb2;
+            }
+        }
     }
     return RFAST_OK;
 } catch (...) {

@@ -903,6 +903,82 @@ k_diag_norm2(const double* __restrict__ acc, int64_t p, double inv_chunks, doubl
     if (threadIdx.x == 0) part[(int64_t)blockIdx.x * kDiagSlots + 5] = red[0];
 }
 
+// Objective of eq. (1) at the mean iterate for the sampled objectives: one warp per shard row, the
+// row's loss (without the L2 term) in double into rowloss[node * rows + k].  Plain and slow on
+// purpose (diagnostics).  grid = (ceil(rows / 8), n), 256 threads.
+//   softmax: x = [W (C x F) | bias (C)], loss = logsumexp(W a + bias) - (W a + bias)[label]
+__global__ void __launch_bounds__(256)
+k_diag_loss_softmax(const float* __restrict__ feat, const int* __restrict__ label, const float* __restrict__ xbar,
+                    double* __restrict__ rowloss, int rows, int F, int C) {
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (k >= rows) return;
+    const int64_t r = (int64_t)blockIdx.y * rows + k;
+    const float* a = feat + r * F;
+    const int lab = label[r];
+    double mx = -1e300, own = 0, se = 0;
+    double lg[32];                                        // C <= 32 classes here
+    for (int c = 0; c < C; ++c) {
+        double s = 0;
+        for (int f = lane; f < F; f += 32) s += (double)xbar[(int64_t)c * F + f] * (double)a[f];
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        s += (double)xbar[(int64_t)C * F + c];
+        lg[c] = s;
+        mx = fmax(mx, s);
+        if (c == lab) own = s;
+    }
+    for (int c = 0; c < C; ++c) se += exp(lg[c] - mx);
+    if (lane == 0) rowloss[r] = mx + log(se) - own;
+}
+//   sparse logistic: loss = log(1 + exp(-y a.x))
+__global__ void __launch_bounds__(256)
+k_diag_loss_logistic(const int64_t* __restrict__ sp_ptr, const int* __restrict__ sp_col, const float* __restrict__ sp_val,
+                     const int* __restrict__ label, const float* __restrict__ xbar, double* __restrict__ rowloss, int rows) {
+    const int k = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (k >= rows) return;
+    const int64_t r = (int64_t)blockIdx.y * rows + k;
+    double s = 0;
+    for (int64_t q = sp_ptr[r] + lane; q < sp_ptr[r + 1]; q += 32) s += (double)sp_val[q] * (double)xbar[sp_col[q]];
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const double m = (double)label[r] * s;
+    if (lane == 0) rowloss[r] = m > 0 ? log1p(exp(-m)) : -m + log1p(exp(m));
+}
+//   MLP: x = [W1 (H x F) | b1 (H) | W2 (C x H) | b2 (C)]; the operands of A W1^T rounded to bf16 (the
+//   matrix product the tensor cores take), everything else as it is; dynamic shared memory: 8 * H doubles
+__global__ void __launch_bounds__(256)
+k_diag_loss_mlp(const float* __restrict__ feat, const int* __restrict__ label, const float* __restrict__ xbar,
+                double* __restrict__ rowloss, int rows, int F, int H, int C) {
+    extern __shared__ double hs_all[];
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k = blockIdx.x * 8 + w;
+    if (k >= rows) return;
+    double* hs = hs_all + (size_t)w * H;
+    const int64_t r = (int64_t)blockIdx.y * rows + k;
+    const float* a = feat + r * F;
+    const float *W1 = xbar, *b1 = xbar + (int64_t)H * F, *W2 = b1 + H, *b2 = W2 + (int64_t)C * H;
+    for (int j = 0; j < H; ++j) {
+        double s = 0;
+        for (int f = lane; f < F; f += 32)
+            s += (double)__bfloat162float(__float2bfloat16_rn(W1[(int64_t)j * F + f])) * (double)__bfloat162float(__float2bfloat16_rn(a[f]));
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) hs[j] = fmax(s + (double)b1[j], 0.0);
+    }
+    __syncwarp();
+    const int lab = label[r];
+    double mx = -1e300, own = 0, se = 0;
+    double lg[32];
+    for (int c = 0; c < C; ++c) {
+        double s = 0;
+        for (int j = lane; j < H; j += 32) s += (double)W2[(int64_t)c * H + j] * hs[j];
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        s += (double)b2[c];
+        lg[c] = s;
+        mx = fmax(mx, s);
+        if (c == lab) own = s;
+    }
+    for (int c = 0; c < C; ++c) se += exp(lg[c] - mx);
+    if (lane == 0) rowloss[r] = mx + log(se) - own;
+}
+
 // bf16 copy (round-to-nearest-even) of every row.  grid = (tiles, rows)
 __global__ void __launch_bounds__(kThreads)
 k_rows_to_bf16(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, int64_t stride, int n4) {
