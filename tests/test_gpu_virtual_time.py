@@ -48,6 +48,8 @@ def test_async_beats_sync_in_virtual_time_with_a_straggler(rfast_lib):
             for r in range(0, sch.K, every):
                 eng.run(every)
                 curve.append(((r + every) * unit, global_loss(eng.read(B.STATE_X))))
+                on_device = eng.diagnostics()["objective"] / n          # the same curve without leaving the GPU
+                assert abs(on_device - curve[-1][1]) <= 1e-5 * abs(curve[-1][1])
             assert rel_l2(eng.read(B.STATE_X), orc.X()) <= 1e-5       # both modes in parity with the oracle
             d = eng.diagnostics()
         curves[name] = curve
