@@ -108,6 +108,11 @@ class ClockSampler:
 FUSED_TRAFFIC = {"kernel_sha256": "73cc8e072e4fec398daf558dd6e2cd7ab9a5112ad452c89c5a03fbc5c624155c", "ratio": 0.96}
 
 
+# The same for k_logit_fused (profiles/k_logit_fused_logistic_tree1024_small_ncu.md): rounds 10 and
+# 11 of the small case, 4.299 / 3.877 GB of DRAM traffic against 4.209 / 3.806 GB of method bytes.
+LOGIT_TRAFFIC = {"kernel_sha256": "754ea1df116f86cecdc60a01b47522d0994ce8a0021521bc5be5fb64fdd00077", "ratio": 1.02}
+
+
 def _fused_kernel_source():
     """The part of kernels.cuh that the fused kernel is made of: load/store helpers, the shared
     tracking tail and k_fused_quad itself."""
@@ -123,6 +128,17 @@ def fused_traffic_ratio():
     try:
         if hashlib.sha256(_fused_kernel_source().encode()).hexdigest() == FUSED_TRAFFIC["kernel_sha256"]:
             return FUSED_TRAFFIC["ratio"]
+    except (OSError, ValueError):
+        pass
+    return None                      # the kernel changed since the counters were taken
+
+
+def logit_traffic_ratio():
+    import hashlib
+    try:
+        path = os.path.join(ROOT, "paper_2307_11617_b200", "csrc", "logit_fused.cuh")
+        if hashlib.sha256((open(path).read() + _fused_kernel_source()).encode()).hexdigest() == LOGIT_TRAFFIC["kernel_sha256"]:
+            return LOGIT_TRAFFIC["ratio"]
     except (OSError, ValueError):
         pass
     return None                      # the kernel changed since the counters were taken
@@ -354,7 +370,9 @@ def measure_config(name, args, steps, world, rank, local, cpu_budget_s, stream=N
                 "implementation_bytes": {"per_step": bytes_impl, "achieved": achieved_impl, "frac": achieved_impl / peak,
                                          "what": "every stream the kernels touch (re-reads between the kernels of a split step, low-order tracker words)"},
                 "traffic": (fused_traffic_ratio() and fused_traffic_ratio() * bytes_impl / per_launch)
-                if fused and args.tracker == "sums" and not sharded else None,   # the counters were taken on that workload
+                if fused and args.tracker == "sums" and not sharded else          # the counters were taken on that workload
+                (logit_traffic_ratio() and logit_traffic_ratio() * bytes_method / K_rounds)
+                if wl.model == "logistic_sparse" and per_launch == K_rounds and args.tracker == "sums" else None,
                 "note": None if hbm_bound else "state is L2-resident: latency-bound, no roofline claim"}
 
     if fused and not args.small:
