@@ -12,6 +12,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <atomic>
 #include <thread>
 
 #include "rfast_internal.h"
@@ -213,8 +214,12 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
     }
 
     // ---- pass 1: consumed stamps, version lifetimes -----------------------------------------
+    // What an edge delivers depends on that edge alone: the rounds in which its sender sent (with
+    // which delay code) and the rounds in which its receiver was active.  So the replay runs edge
+    // by edge -- a packet sent in round r with delay d is usable from round r + 1 + d, a receiver
+    // active in round r takes the largest stamp usable by then -- and long schedules spread the
+    // edges over several threads.  Every edge writes its own entries only.
     const int INF = INT_MAX;
-    std::vector<PendQ> pend_v(R.E), pend_c(C.E);
     std::vector<int> tau_v(R.E, 0), tau_rho(C.E, 0), t(n, 0);
     c.ev_of.assign(n, {});
     {
@@ -223,107 +228,146 @@ int compile_schedule(const HostGraph& R, const HostGraph& C, const rfast_schedul
         for (int i = 0; i < n; ++i) c.ev_of[i].reserve(cnt[i]);
     }
     std::vector<std::vector<int>>& ev_of = c.ev_of;    // node -> event id of stamp s at [s-1]
-    c.used_tau_v.reserve(c.in_r_off[nE]);
-    c.used_tau_rho.reserve(c.in_c_off[nE]);
-    c.prev_tau_rho.reserve(c.in_c_off[nE]);
+    std::vector<int> ev_round(nE);
+    c.used_tau_v.assign(c.in_r_off[nE], 0);
+    c.used_tau_rho.assign(c.in_c_off[nE], 0);
+    c.prev_tau_rho.assign(c.in_c_off[nE], 0);
     c.v_write.assign(nE, 0);
     c.v_last.assign(nE, 0);
     std::vector<char> v_sent(nE, 0);
     const int64_t nRho = c.out_c_off[nE];
     c.rho_write.assign(nRho, 0);
     std::vector<int> rho_last_sender(nRho, 0), rho_last_recv(nRho, -1);
+    std::vector<int> v_last_edge(c.out_r_off[nE], -1);     // per (event, G_R out-edge): last round its v is read
     if (buckets) c.rho_leader.assign(nRho, -1);
+    for (int r = 0; r < K; ++r)
+        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
+            const int i = c.act_node[ev];
+            ev_round[ev] = r;
+            ev_of[i].push_back(ev);
+            c.v_write[ev] = r;
+            for (int k = 0; k < R.outdeg(i); ++k) v_sent[ev] |= s->send_r[c.out_r_off[ev] + k] >= 0;
+            for (int k = 0; k < C.outdeg(i); ++k) { c.rho_write[c.out_c_off[ev] + k] = r; rho_last_sender[c.out_c_off[ev] + k] = r; }
+        }
+    for (int i = 0; i < n; ++i) {
+        t[i] = (int)ev_of[i].size();
+        if (!buckets)                                     // S2c of the next activation reads the sender's current running sums
+            for (size_t q = 0; q + 1 < ev_of[i].size(); ++q) {
+                const int64_t base = c.out_c_off[ev_of[i][q]];
+                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = ev_round[ev_of[i][q + 1]];
+            }
+    }
     // A hold at round b: whatever an activation in round b or later may still read stays in its
     // row through round b -- per edge the version its receiver holds and every packet still on
     // its way or waiting, and every sender's latest running sums.  The rows of the rounds before
     // b then do not depend on what follows b: rounds can be appended without moving any of them.
+    static const std::vector<int> no_holds;
+    const std::vector<int>& H = holds ? *holds : no_holds;
     auto for_pending = [](const PendQ& q, auto&& f) {
         if (q.more) { for (const Pend& pk : *q.more) f(pk); }
         else for (int k = 0; k < q.n; ++k) f(q.a[k]);
     };
-    auto hold = [&](int b) {
-        for (int e = 0; e < R.E; ++e) {
-            const auto& evs = ev_of[R.col[e]];
-            if (tau_v[e] >= 1) c.v_last[evs[tau_v[e] - 1]] = std::max(c.v_last[evs[tau_v[e] - 1]], b);
-            for_pending(pend_v[e], [&](const Pend& pk) {
-                if (pk.stamp > tau_v[e]) c.v_last[evs[pk.stamp - 1]] = std::max(c.v_last[evs[pk.stamp - 1]], b);
-            });
-        }
-        for (int e = 0; e < C.E; ++e) {
-            const auto& evs = ev_of[C.col[e]];
-            auto keep = [&](int stamp) {
-                int64_t vid = c.out_c_off[evs[stamp - 1]] + C.opos[e];
-                rho_last_recv[vid] = std::max(rho_last_recv[vid], b);
-            };
-            if (tau_rho[e] >= 1) keep(tau_rho[e]);
-            for_pending(pend_c[e], [&](const Pend& pk) { if (pk.stamp > tau_rho[e]) keep(pk.stamp); });
-        }
-        for (int i = 0; i < n; ++i)
-            if (t[i] >= 1) {
-                int64_t base = c.out_c_off[ev_of[i][t[i] - 1]];
-                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = std::max(rho_last_sender[base + k], b);
+    auto edge_r = [&](int e) {
+        const std::vector<int>& S = ev_of[R.col[e]];
+        const std::vector<int>& A = ev_of[R.recv[e]];
+        const int kin = e - R.rowptr[R.recv[e]], kout = R.opos[e];
+        PendQ q;
+        int tau = 0;
+        size_t ps = 0, h = 0;
+        auto read_in = [&](int stamp, int r) { int& l = v_last_edge[c.out_r_off[S[stamp - 1]] + kout]; l = std::max(l, r); };
+        auto admit = [&](int before) {                       // the packets sent in rounds < before
+            for (; ps < S.size() && ev_round[S[ps]] < before; ++ps) {
+                const int d = s->send_r[c.out_r_off[S[ps]] + kout];
+                if (d >= 0) q.push({ev_round[S[ps]] + 1 + d, (int)ps + 1});
             }
+        };
+        auto hold = [&](int b) {
+            admit(b);
+            if (tau >= 1) read_in(tau, b);
+            for_pending(q, [&](const Pend& pk) { if (pk.stamp > tau) read_in(pk.stamp, b); });
+        };
+        for (int ev : A) {
+            const int r = ev_round[ev];
+            for (; h < H.size() && H[h] <= r; ++h) hold(H[h]);
+            admit(r);
+            tau = deliver(q, r, tau);
+            c.used_tau_v[c.in_r_off[ev] + kin] = tau;
+            if (tau >= 1) read_in(tau, r);
+        }
+        for (; h < H.size(); ++h) hold(H[h]);
+        tau_v[e] = tau;
     };
-    size_t next_hold = 0;
-    for (int r = 0; r < K; ++r) {
-        if (holds && next_hold < holds->size() && (*holds)[next_hold] == r) { hold(r); ++next_hold; }
-        for (int ev = c.act_ptr[r]; ev < c.act_ptr[r + 1]; ++ev) {
-            const int i = c.act_node[ev];
-            for (int e = R.rowptr[i]; e < R.rowptr[i + 1]; ++e) {
-                int tau = deliver(pend_v[e], r, tau_v[e]);
-                tau_v[e] = tau;
-                c.used_tau_v.push_back(tau);
-                if (tau >= 1) {
-                    int pe = ev_of[R.col[e]][tau - 1];
-                    c.v_last[pe] = std::max(c.v_last[pe], r);
-                }
+    auto edge_c = [&](int e) {
+        const std::vector<int>& S = ev_of[C.col[e]];
+        const std::vector<int>& A = ev_of[C.recv[e]];
+        const int kin = e - C.rowptr[C.recv[e]], kout = C.opos[e];
+        PendQ q;
+        int tau = 0;
+        size_t ps = 0, h = 0;
+        auto vid_of = [&](int stamp) { return c.out_c_off[S[stamp - 1]] + kout; };
+        auto read_in = [&](int stamp, int r) { int& l = rho_last_recv[vid_of(stamp)]; l = std::max(l, r); };
+        auto admit = [&](int before) {
+            for (; ps < S.size() && ev_round[S[ps]] < before; ++ps) {
+                const int d = s->send_c[c.out_c_off[S[ps]] + kout];
+                if (d >= 0) q.push({ev_round[S[ps]] + 1 + d, (int)ps + 1});
             }
-            for (int e = C.rowptr[i]; e < C.rowptr[i + 1]; ++e) {
-                int prev = tau_rho[e];
-                int tau = deliver(pend_c[e], r, prev);
-                c.used_tau_rho.push_back(tau);
-                c.prev_tau_rho.push_back(prev);
-                if (tau > prev && buckets) {           // news: the contributions of stamps prev+1 .. tau, one row
-                    const auto& evs = ev_of[C.col[e]];
-                    const int64_t lead = c.out_c_off[evs[prev]] + C.opos[e];
-                    for (int st = prev + 1; st <= tau; ++st) c.rho_leader[c.out_c_off[evs[st - 1]] + C.opos[e]] = lead;
-                    rho_last_recv[lead] = r;
-                } else if (tau > prev) {               // news: rho[tau] - rho[prev] is read
-                    const auto& evs = ev_of[C.col[e]];
-                    int64_t vn = c.out_c_off[evs[tau - 1]] + C.opos[e];
-                    rho_last_recv[vn] = std::max(rho_last_recv[vn], r);
-                    if (prev >= 1) {
-                        int64_t vp = c.out_c_off[evs[prev - 1]] + C.opos[e];
-                        rho_last_recv[vp] = std::max(rho_last_recv[vp], r);
-                    }
-                }
-                tau_rho[e] = tau;
+        };
+        auto hold = [&](int b) {
+            admit(b);
+            if (tau >= 1) read_in(tau, b);
+            for_pending(q, [&](const Pend& pk) { if (pk.stamp > tau) read_in(pk.stamp, b); });
+        };
+        for (int ev : A) {
+            const int r = ev_round[ev];
+            for (; h < H.size() && H[h] <= r; ++h) hold(H[h]);
+            admit(r);
+            const int prev = tau;
+            tau = deliver(q, r, prev);
+            c.used_tau_rho[c.in_c_off[ev] + kin] = tau;
+            c.prev_tau_rho[c.in_c_off[ev] + kin] = prev;
+            if (tau > prev && buckets) {                   // news: the contributions of stamps prev+1 .. tau, one row
+                const int64_t lead = vid_of(prev + 1);
+                for (int st = prev + 1; st <= tau; ++st) c.rho_leader[vid_of(st)] = lead;
+                rho_last_recv[lead] = r;
+            } else if (tau > prev) {                       // news: rho[tau] - rho[prev] is read
+                read_in(tau, r);
+                if (prev >= 1) read_in(prev, r);
             }
-            const int stamp = ++t[i];
-            if (stamp >= 2 && !buckets) {              // S2c reads the sender's current running sums
-                int64_t base = c.out_c_off[ev_of[i][stamp - 2]];
-                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = r;
+        }
+        for (; h < H.size(); ++h) hold(H[h]);
+        tau_rho[e] = tau;
+    };
+    {
+        int nthreads = 1;
+        if (nE >= 50000) nthreads = (int)std::min<unsigned>(8u, std::max(1u, std::thread::hardware_concurrency()));
+        if (const char* cap = std::getenv("RFAST_COMPILE_THREADS")) nthreads = std::max(1, std::min(nthreads, std::atoi(cap)));
+        std::atomic<int> next{0};
+        auto work = [&]() {
+            for (int e; (e = next.fetch_add(1)) < R.E + C.E;) {
+                if (e < R.E) edge_r(e); else edge_c(e - R.E);
             }
-            ev_of[i].push_back(ev);
-            c.v_write[ev] = r;
-            c.v_last[ev] = r;
-            for (int k = 0; k < R.outdeg(i); ++k) {
-                int d = s->send_r[c.out_r_off[ev] + k];
-                if (d >= 0) {
-                    v_sent[ev] = 1;
-                    pend_v[R.oeid[R.optr[i] + k]].push({r + 1 + d, stamp});
-                }
-            }
-            for (int k = 0; k < C.outdeg(i); ++k) {
-                int64_t vid = c.out_c_off[ev] + k;
-                c.rho_write[vid] = r;
-                rho_last_sender[vid] = r;
-                int d = s->send_c[vid];
-                if (d >= 0) pend_c[C.oeid[C.optr[i] + k]].push({r + 1 + d, stamp});
-            }
+        };
+        if (nthreads == 1) work();
+        else {
+            std::vector<std::thread> pool;
+            for (int th = 0; th < nthreads; ++th) pool.emplace_back(work);
+            for (auto& t_ : pool) t_.join();
         }
     }
-    if (holds && next_hold < holds->size() && (*holds)[next_hold] == K) hold(K);   // open end: more rounds may follow
+    for (int64_t ev = 0; ev < nE; ++ev) {
+        int last = c.v_write[ev];
+        for (int64_t q = c.out_r_off[ev]; q < c.out_r_off[ev + 1]; ++q) last = std::max(last, v_last_edge[q]);
+        c.v_last[ev] = last;
+    }
+    for (int b : H)                                        // every sender's latest running sums as of round b
+        for (int i = 0; i < n; ++i) {
+            const auto& evs = ev_of[i];
+            const size_t tb = std::lower_bound(evs.begin(), evs.end(), b, [&](int ev, int rb) { return ev_round[ev] < rb; }) - evs.begin();
+            if (tb >= 1) {
+                const int64_t base = c.out_c_off[evs[tb - 1]];
+                for (int k = 0; k < C.outdeg(i); ++k) rho_last_sender[base + k] = std::max(rho_last_sender[base + k], b);
+            }
+        }
     c.tau_v_end = tau_v;
     c.tau_rho_end = tau_rho;
     c.t_end = t;
