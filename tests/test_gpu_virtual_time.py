@@ -58,3 +58,39 @@ def test_async_beats_sync_in_virtual_time_with_a_straggler(rfast_lib):
     assert curves["async"][-1][1] < sync_final                         # better at equal simulated time
     t_reach = next(t for t, loss in curves["async"] if loss <= sync_final)
     assert t_reach <= T / 2, (t_reach, curves)                          # and at least twice as fast to that loss
+
+
+def test_async_beats_sync_on_the_full_size_mlp_with_heavy_tailed_compute_times(rfast_lib):
+    """The same claim on the non-convex objective at the benchmarked size (n = 64, MLP 784-512-10,
+    lognormal compute times): no oracle is needed, the loss curve F(xbar) comes from the device.
+    A synchronous iteration lasts as long as its slowest node's compute time (the maximum of 64
+    lognormal draws); R-FAST nodes go on at their own pace, with delays and losses."""
+    import copy
+    import paper_2307_11617_b200 as pkg
+    wl = build_config("mlp_tree64", seed=0)
+    n, T = wl.n, wl.schedule.K                                         # one round = one time unit
+    rng = np.random.default_rng(7)
+    dur = np.maximum(1, np.rint(np.exp(rng.standard_normal((T, n))))).max(axis=1)
+    end = np.cumsum(dur)                                               # when each synchronous iteration is through
+    k_sync = int((end <= T).sum())
+    s_sync = make_schedule(wl.G_R, wl.G_C, activation_all(n, k_sync), 0.0, 0, rng, batch=wl.batch, rows_per_node=wl.rows)
+    curves = {}
+    for name, sch, every in (("async", wl.schedule, 25), ("sync", s_sync, 5)):
+        w = copy.copy(wl)
+        w.schedule = sch
+        with pkg.Engine(w) as eng:
+            eng.load_schedule(sch)
+            f0 = eng.diagnostics()["objective"] / n
+            curve = []
+            for r in range(0, sch.K, every):
+                eng.run(min(every, sch.K - r))
+                rr = min(r + every, sch.K)
+                d = eng.diagnostics()
+                curve.append((float(rr) if name == "async" else float(end[rr - 1]), d["objective"] / n))
+                assert d["conservation_residual"] <= 1e-5 * max(d["gradient_sum_max"], d["tracker_norm"])
+        curves[name] = curve
+        assert curve[-1][1] < f0
+    sync_final = curves["sync"][-1][1]
+    assert curves["async"][-1][1] <= 0.1 * sync_final                   # far lower at equal simulated time
+    t_reach = next(t for t, loss in curves["async"] if loss <= sync_final)
+    assert t_reach <= T / 3, (t_reach, curves)                          # and at least three times as fast to that loss
