@@ -133,3 +133,25 @@ def test_coordinate_shards_partition_the_problem_and_the_oracle_agrees():
     assert np.array_equal(np.concatenate(Z, axis=1), whole.Z())
     with pytest.raises(ValueError):
         shard_coordinates(build_config("ls_ring4", seed=0), 0, 2)
+
+
+def test_split_schedule_parts_tile_the_schedule():
+    """Cutting a schedule into consecutive parts is array slicing only: laid end to end again
+    (events renumbered, each part's copy of the initial samples dropped) the parts are the
+    schedule."""
+    import numpy as np
+    from workloads import build_config, split_schedule
+    wl = build_config("softmax_exp16", seed=3, F=12, C=4, rows=16, K=90, batch=4)
+    s = wl.schedule
+    parts = split_schedule(s, wl.G_R, wl.G_C, [7, 30, 31])
+    assert [p.K for p in parts] == [7, 23, 1, 59]
+    lead = wl.n * s.batch
+    assert np.array_equal(np.concatenate([p.act_node for p in parts]), s.act_node)
+    assert np.array_equal(np.concatenate([p.send_r for p in parts]), s.send_r)
+    assert np.array_equal(np.concatenate([p.send_c for p in parts]), s.send_c)
+    assert np.array_equal(np.concatenate([s.batch_idx[:lead]] + [p.batch_idx[lead:] for p in parts]), s.batch_idx)
+    ev0 = 0
+    for p in parts:
+        assert p.act_ptr[0] == 0 and np.array_equal(p.batch_idx[:lead], s.batch_idx[:lead])
+        ev0 += p.n_events
+    assert ev0 == s.n_events
