@@ -767,6 +767,7 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
     double cons = 0, xb2 = 0, res = 0, gs = 0, z2 = 0, gf2 = 0, fl = 0;
     if (c < p) {
         double sx = 0, sx2 = 0, sz = 0, sg = 0;
+#pragma unroll 8
         for (int i = 0; i < n; ++i) {
             const double xv = x[(int64_t)i * stride + c];
             double zv = z[(int64_t)i * stride + c];
@@ -795,6 +796,7 @@ k_diagnostics(const float* __restrict__ x, const float* __restrict__ z, const fl
         if (xbar_out) xbar_out[c] = (float)xbar;
         if (!gpool) {
             double gf = 0;
+#pragma unroll 8
             for (int i = 0; i < n; ++i) {
                 const double d = qd[(int64_t)i * stride + c];
                 const double r = d * (xbar - (double)qb[(int64_t)i * stride + c]);
