@@ -365,7 +365,7 @@ int     rfast_checkpoint_load(rfast_ctx* ctx, const void* src, size_t bytes);
  *          (softmax, MLP, sparse logistic) it is formed with the kernels the activations use,
  *          the shards walked in chunks of B rows from a state whose rows all hold xbar; x is
  *          moved aside and put back bit for bit, the first such call allocates its scratch (a
- *          copy of x, a double per coordinate) and keeps it while the schedule stays loaded.
+ *          copy of x, a double per coordinate) and keeps it for the life of the handle.
  *          NaN where the shard size is not a multiple of B
  *   out[6] the merit function of the non-convex analysis (Section V-B),
  *          M_F(x) = || grad F(xbar) ||^2 + || x - 1 xbar^T ||^2 = out[5]^2 + out[0]^2 (NaN where out[5] is)

@@ -336,11 +336,14 @@ def rfast_checkpoint_load(handle, blob: np.ndarray) -> None:
     _check(lib().rfast_checkpoint_load(handle, _ptr(blob), blob.nbytes), handle)
 
 
-def rfast_diagnostics(handle) -> dict:
+def rfast_diagnostics(handle, full: bool = True) -> dict:
     """Consensus error, norm of the mean iterate, conservation residual (Lemma 3) and its scale,
-    tracker norm, all computed on the device."""
-    out = np.zeros(8, dtype=np.float64)
-    _check(lib().rfast_diagnostics(handle, _ptr(out), 8), handle)
+    tracker norm, all computed on the device in one pass over the state; with full=True also the
+    full gradient, the merit function and the objective at the mean iterate (a pass over every
+    row of every shard)."""
+    n_out = 8 if full else 5
+    out = np.full(8, np.nan, dtype=np.float64)
+    _check(lib().rfast_diagnostics(handle, _ptr(out), n_out), handle)
     return {"consensus_error": out[0], "xbar_norm": out[1], "conservation_residual": out[2],
             "gradient_sum_max": out[3], "tracker_norm": out[4], "full_gradient_norm": out[5],
             "merit": out[6], "objective": out[7]}
@@ -430,8 +433,8 @@ class Engine:
     def restore(self, blob):
         rfast_checkpoint_load(self.h, blob)
 
-    def diagnostics(self):
-        return rfast_diagnostics(self.h)
+    def diagnostics(self, full=True):
+        return rfast_diagnostics(self.h, full)
 
     def close(self):
         if self.h:

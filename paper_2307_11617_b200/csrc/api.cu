@@ -138,7 +138,7 @@ struct rfast_ctx {
     double* d_diag_part = nullptr;
     float* d_xbar = nullptr;  float* d_diag_res = nullptr;
     // sampled objectives, full gradient at the mean iterate (allocated at the first call that asks
-    // for it): a copy of x, a double per coordinate, descriptors and a batch table over whole shards
+    // for it, kept for the life of the handle): a copy of x, a double per coordinate, descriptors and a batch table over whole shards
     double* d_diag_rowloss = nullptr;
     float* d_diag_x = nullptr;  double* d_diag_acc = nullptr;  EvDesc* d_diag_ev = nullptr;  int* d_diag_bidx = nullptr;
     MlpPlan* mlp = nullptr;
@@ -234,8 +234,6 @@ void free_schedule(rfast_ctx* c) {
     c->d_ev = c->d_init_ev = nullptr;
     c->vbuf = c->rbuf = c->scratch = nullptr;
     c->d_diag_idx = nullptr; c->d_diag_part = nullptr; c->d_xbar = nullptr; c->d_diag_res = nullptr;
-    c->d_diag_rowloss = nullptr;
-    c->d_diag_x = nullptr; c->d_diag_acc = nullptr; c->d_diag_ev = nullptr; c->d_diag_bidx = nullptr;
     c->d_act_ptr = nullptr; c->d_alpha_round = nullptr; c->d_bar = nullptr; c->d_pstatus = nullptr;
     c->persist_ok = false;
     c->has_sched = false;
@@ -515,7 +513,8 @@ void rfast_destroy(rfast_ctx* c) {
     free_schedule(c);
     if (c->mlp) mlp_plan_destroy(c->mlp);
     void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
-                    c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb, c->row_tmp};
+                    c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb, c->row_tmp,
+                    c->d_diag_rowloss, c->d_diag_x, c->d_diag_acc, c->d_diag_ev, c->d_diag_bidx};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete c;
 }
@@ -1485,10 +1484,11 @@ static int sampled_full_gradient(rfast_ctx* ctx, const RoundView& rv, int blocks
     const size_t plane = (size_t)n * ctx->stride;
     const int n4 = (int)(ctx->stride / 4);
     if (!ctx->d_diag_x) {
-        CK(dev_alloc(ctx, &ctx->d_diag_x, plane, true));
-        CK(dev_alloc(ctx, &ctx->d_diag_acc, (size_t)ctx->stride, true));
-        CK(dev_alloc(ctx, &ctx->d_diag_ev, (size_t)chunks * n, true));
-        CK(dev_alloc(ctx, &ctx->d_diag_bidx, (size_t)chunks * n * B, true));
+        // sizes follow the problem, not the schedule: kept for the life of the handle
+        CK(dev_alloc(ctx, &ctx->d_diag_x, plane, false));
+        CK(dev_alloc(ctx, &ctx->d_diag_acc, (size_t)ctx->stride, false));
+        CK(dev_alloc(ctx, &ctx->d_diag_ev, (size_t)chunks * n, false));
+        CK(dev_alloc(ctx, &ctx->d_diag_bidx, (size_t)chunks * n * B, false));
         if (!ctx->d_xbar) {
             CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
             CK(cudaMemsetAsync(ctx->d_xbar, 0, ctx->stride * sizeof(float), ctx->stream));
@@ -1575,7 +1575,7 @@ int rfast_diagnostics(rfast_ctx* ctx, double* out, int32_t n_out) try {
                          (ctx->model == RFAST_MODEL_SOFTMAX || ctx->model == RFAST_MODEL_MLP || ctx->model == RFAST_MODEL_LOGISTIC_SPARSE);
     const bool sampled_model = ctx->model == RFAST_MODEL_SOFTMAX || ctx->model == RFAST_MODEL_MLP || ctx->model == RFAST_MODEL_LOGISTIC_SPARSE;
     const bool lossy = n_out == 8 && sampled_model && (ctx->model == RFAST_MODEL_LOGISTIC_SPARSE || ctx->C <= 32);
-    if (lossy && !ctx->d_diag_rowloss) CK(dev_alloc(ctx, &ctx->d_diag_rowloss, (size_t)n * ctx->rows, true));
+    if (lossy && !ctx->d_diag_rowloss) CK(dev_alloc(ctx, &ctx->d_diag_rowloss, (size_t)n * ctx->rows, false));
     if ((sampled || lossy) && !ctx->d_xbar) {          // the mean iterate is wanted on the device
         CK(dev_alloc(ctx, &ctx->d_xbar, (size_t)ctx->stride, true));
         CK(cudaMemsetAsync(ctx->d_xbar, 0, ctx->stride * sizeof(float), ctx->stream));
