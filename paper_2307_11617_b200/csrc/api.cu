@@ -149,7 +149,10 @@ struct rfast_ctx {
     int *d_mix_slot = nullptr, *d_news_new = nullptr, *d_news_prev = nullptr, *d_out_cur = nullptr,
         *d_out_new = nullptr, *d_batch_idx = nullptr;
     float *d_mix_w = nullptr, *d_out_a = nullptr;
-    std::vector<void*> sched_allocs;
+    struct Block { void* p; size_t bytes; };
+    std::vector<Block> sched_allocs;        // device blocks owned by the loaded schedule
+    std::vector<Block> spare;               // blocks of the schedule being replaced, handed out again while the
+                                            // next one is put in place (a re-load then allocates nothing)
     std::vector<float> alpha_round;         // per-round step size, empty: constant alpha
     uint64_t sched_hash = 0;                // identity of the loaded schedule (checkpoints)
     // persistent multi-round kernel (L2-resident problems)
@@ -199,10 +202,25 @@ template <class T>
 cudaError_t dev_alloc(rfast_ctx* c, T** ptr, size_t count, bool sched = false) {
     *ptr = nullptr;
     if (count == 0) count = 1;
-    cudaError_t e = cudaMalloc((void**)ptr, count * sizeof(T));
+    const size_t want = count * sizeof(T);
+    if (sched) {                                   // a block of the replaced schedule that fits (not more than twice the size)
+        int best = -1;
+        for (int k = 0; k < (int)c->spare.size(); ++k)
+            if (c->spare[k].bytes >= want && c->spare[k].bytes <= 2 * want + 256 &&
+                (best < 0 || c->spare[k].bytes < c->spare[best].bytes)) best = k;
+        if (best >= 0) {
+            const rfast_ctx::Block b = c->spare[best];
+            c->spare.erase(c->spare.begin() + best);
+            *ptr = (T*)b.p;
+            c->dev_bytes += b.bytes;  c->sched_bytes += b.bytes;
+            c->sched_allocs.push_back(b);
+            return cudaSuccess;
+        }
+    }
+    cudaError_t e = cudaMalloc((void**)ptr, want);
     if (e == cudaSuccess) {
-        c->dev_bytes += count * sizeof(T);
-        if (sched) { c->sched_allocs.push_back(*ptr); c->sched_bytes += count * sizeof(T); }
+        c->dev_bytes += want;
+        if (sched) { c->sched_allocs.push_back({*ptr, want}); c->sched_bytes += want; }
     }
     return e;
 }
@@ -223,11 +241,18 @@ int upload_rows(rfast_ctx* ctx, float* dst, const float* src, int64_t rows) {
     return RFAST_OK;
 }
 
-void free_schedule(rfast_ctx* c) {
+void drop_spare(rfast_ctx* c) {
+    for (auto& b : c->spare) cudaFree(b.p);
+    c->spare.clear();
+}
+
+// recycle: the blocks are kept aside for the schedule that is about to be put in place
+void free_schedule(rfast_ctx* c, bool recycle = false) {
     for (auto& gc : c->graph_chunks) cudaGraphExecDestroy(gc.exec);
     c->graph_chunks.clear();
     c->graph_r0 = c->graph_r1 = -1;
-    for (void* q : c->sched_allocs) cudaFree(q);
+    if (recycle) c->spare.insert(c->spare.end(), c->sched_allocs.begin(), c->sched_allocs.end());
+    else for (auto& b : c->sched_allocs) cudaFree(b.p);
     c->sched_allocs.clear();
     c->dev_bytes -= c->sched_bytes;
     c->sched_bytes = 0;
@@ -511,6 +536,7 @@ void rfast_destroy(rfast_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->stream);
     free_schedule(c);
+    drop_spare(c);
     if (c->mlp) mlp_plan_destroy(c->mlp);
     void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
                     c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb, c->row_tmp,
@@ -650,13 +676,17 @@ static int install_schedule(rfast_ctx* ctx, const rfast_schedule* s, Compiled&& 
     if (keep_state) {
         old_v = ctx->vbuf;  old_r = ctx->rbuf;
         auto& al = ctx->sched_allocs;
-        al.erase(std::remove_if(al.begin(), al.end(), [&](void* q) { return q == (void*)old_v || q == (void*)old_r; }), al.end());
+        al.erase(std::remove_if(al.begin(), al.end(), [&](const rfast_ctx::Block& b) { return b.p == (void*)old_v || b.p == (void*)old_r; }), al.end());
     }
     struct OldRows {                                   // freed on every way out
         float *v, *r;
         ~OldRows() { if (v) cudaFree(v); if (r) cudaFree(r); }
     } old_rows{old_v, old_r};
-    free_schedule(ctx);
+    struct Spare {                                     // what the new schedule did not take over is freed on every way out
+        rfast_ctx* c;
+        ~Spare() { drop_spare(c); }
+    } spare{ctx};
+    free_schedule(ctx, true);
     ctx->alpha_round.clear();
     if (s->alpha_round) {
         for (int r = 0; r < s->K; ++r)
