@@ -336,6 +336,21 @@ enum { RFAST_OPT_PERSISTENT = 0, RFAST_OPT_GRAPHS = 1, RFAST_OPT_WAIT_LIMIT_MS =
        RFAST_OPT_ONE_PASS = 4, RFAST_OPT_CLUSTER_SIZE = 5, RFAST_OPT_OPEN_END = 6 };
 int rfast_set_option(rfast_ctx* ctx, int option, int64_t value);
 
+/* Read-back of x and y that runs under the work that follows (no counterpart in the paper: a
+ * service call for callers that run one schedule after another).  rfast_snapshot enqueues, on the
+ * handle's stream, a copy of x and y -- as of everything enqueued so far -- into a second pair of
+ * device arrays (allocated at the first call, kept for the life of the handle: 2 n p floats), and on
+ * a stream of the handle's own the transfer of that copy into x_dst and y_dst, caller-owned HOST
+ * arrays float [n][p] (unpadded, as RFAST_STATE_X / RFAST_STATE_Y deliver them; page-locked memory
+ * if the transfer is to overlap anything).  It returns at once; rfast_load_schedule, rfast_reset
+ * and rfast_run may follow immediately and do not disturb the snapshot.  The destinations hold the
+ * snapshot after rfast_snapshot_wait has returned; a second rfast_snapshot before that queues
+ * behind the first (on the device, the host does not wait) and its transfer may overwrite the
+ * same destinations.  The values are bit for bit those of rfast_read_state at the same point.
+ * RFAST_EINVAL on a null destination, RFAST_ENOMEM / RFAST_ECUDA as reported by the runtime. */
+int rfast_snapshot(rfast_ctx* ctx, float* x_dst, float* y_dst);
+int rfast_snapshot_wait(rfast_ctx* ctx);
+
 /* Waits for the handle's stream; reports a pending asynchronous error. */
 int rfast_sync(rfast_ctx* ctx);
 

@@ -98,6 +98,8 @@ def lib():
         L.rfast_checkpoint_load.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         L.rfast_diagnostics.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.rfast_seek.argtypes = [C.c_void_p, C.c_int32]
+        L.rfast_snapshot.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.rfast_snapshot_wait.argtypes = [C.c_void_p]
         L.rfast_write_state.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t]
         L.rfast_read_packet.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]
         L.rfast_write_packet.argtypes = [C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t]
@@ -229,6 +231,19 @@ def rfast_read_state(handle, which: int, shape, out=None) -> np.ndarray:
     assert out.dtype == dt and out.flags.c_contiguous
     _check(lib().rfast_read_state(handle, int(which), _ptr(out), out.nbytes), handle)
     return out
+
+
+def rfast_snapshot(handle, x_out: np.ndarray, y_out: np.ndarray) -> None:
+    """x_out, y_out: C-contiguous float32 [n][p] host arrays (page-locked for an overlapped transfer)
+    that must stay alive until rfast_snapshot_wait."""
+    for a in (x_out, y_out):
+        if a.dtype != np.float32 or not a.flags["C_CONTIGUOUS"]:
+            raise ValueError("snapshot destinations must be C-contiguous float32 arrays")
+    _check(lib().rfast_snapshot(handle, _ptr(x_out), _ptr(y_out)), handle)
+
+
+def rfast_snapshot_wait(handle) -> None:
+    _check(lib().rfast_snapshot_wait(handle), handle)
 
 
 def rfast_seek(handle, rnd: int) -> None:
@@ -432,6 +447,14 @@ class Engine:
 
     def restore(self, blob):
         rfast_checkpoint_load(self.h, blob)
+
+    def snapshot(self, x_out, y_out):
+        if x_out.shape != (self.n, self.p) or y_out.shape != (self.n, self.p):
+            raise ValueError("snapshot destinations must be [n][p]")
+        rfast_snapshot(self.h, x_out, y_out)
+
+    def snapshot_wait(self):
+        rfast_snapshot_wait(self.h)
 
     def diagnostics(self, full=True):
         return rfast_diagnostics(self.h, full)

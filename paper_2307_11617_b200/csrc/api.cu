@@ -173,6 +173,10 @@ struct rfast_ctx {
     bool opt_open_end = false;
     std::vector<int> holds;                 // rounds at which the loaded schedule was held open (its end, earlier ends)
     std::unique_ptr<RawSchedule> raw;       // the raw arrays loaded so far (kept only when open-ended)
+    // snapshot of x and y whose transfer to the host runs under the work that follows (rfast_snapshot)
+    float *snap_x = nullptr, *snap_y = nullptr;
+    cudaStream_t snap_stream = nullptr;
+    cudaEvent_t snap_ready = nullptr, snap_done = nullptr;
     int round = 0;
     int64_t launches = 0;
     // recorded span of rounds [graph_r0, graph_r1): a sequence of graphs of about a thousand kernels each
@@ -537,10 +541,13 @@ void rfast_destroy(rfast_ctx* c) {
     cudaStreamSynchronize(c->stream);
     free_schedule(c);
     drop_spare(c);
+    if (c->snap_stream) { cudaStreamSynchronize(c->snap_stream); cudaStreamDestroy(c->snap_stream); }
+    if (c->snap_ready) cudaEventDestroy(c->snap_ready);
+    if (c->snap_done) cudaEventDestroy(c->snap_done);
     if (c->mlp) mlp_plan_destroy(c->mlp);
     void* ptrs[] = {c->x, c->z, c->zc, c->gbuf, c->x0, c->quad_d, c->quad_b, c->feat, c->target, c->label,
                     c->sp_ptr, c->sp_tile_ptr, c->sp_col, c->sp_val, c->xb, c->row_tmp,
-                    c->d_diag_rowloss, c->d_diag_x, c->d_diag_acc, c->d_diag_ev, c->d_diag_bidx};
+                    c->d_diag_rowloss, c->d_diag_x, c->d_diag_acc, c->d_diag_ev, c->d_diag_bidx, c->snap_x, c->snap_y};
     for (void* q : ptrs) if (q) cudaFree(q);
     delete c;
 }
@@ -1147,6 +1154,37 @@ int packet_row(rfast_ctx* ctx, int graph, int id, int stamp, int* row, std::stri
 }  // namespace
 
 extern "C" {
+
+int rfast_snapshot(rfast_ctx* ctx, float* x_dst, float* y_dst) {
+    if (!ctx || !x_dst || !y_dst) return ctx ? set_err(ctx, RFAST_EINVAL, "snapshot: null destination") : RFAST_EINVAL;
+    const size_t plane = (size_t)ctx->n * ctx->stride * sizeof(float);
+    if (!ctx->snap_stream) {
+        CK(dev_alloc(ctx, &ctx->snap_x, (size_t)ctx->n * ctx->stride, false));
+        CK(dev_alloc(ctx, &ctx->snap_y, (size_t)ctx->n * ctx->stride, false));
+        CK(cudaEventCreateWithFlags(&ctx->snap_ready, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&ctx->snap_done, cudaEventDisableTiming));
+        CK(cudaStreamCreateWithFlags(&ctx->snap_stream, cudaStreamNonBlocking));
+        CK(cudaEventRecord(ctx->snap_done, ctx->snap_stream));
+    }
+    // the copy on the device waits for the previous snapshot's transfer (it reads the same buffers),
+    // the transfer for the copy; the handle's stream is free again after the copy
+    CK(cudaStreamWaitEvent(ctx->stream, ctx->snap_done, 0));
+    CK(cudaMemcpyAsync(ctx->snap_x, ctx->x, plane, cudaMemcpyDeviceToDevice, ctx->stream));
+    CK(cudaMemcpyAsync(ctx->snap_y, ctx->z, plane, cudaMemcpyDeviceToDevice, ctx->stream));
+    CK(cudaEventRecord(ctx->snap_ready, ctx->stream));
+    CK(cudaStreamWaitEvent(ctx->snap_stream, ctx->snap_ready, 0));
+    const size_t rowb = (size_t)ctx->p * sizeof(float);
+    CK(cudaMemcpy2DAsync(x_dst, rowb, ctx->snap_x, ctx->stride * sizeof(float), rowb, ctx->n, cudaMemcpyDeviceToHost, ctx->snap_stream));
+    CK(cudaMemcpy2DAsync(y_dst, rowb, ctx->snap_y, ctx->stride * sizeof(float), rowb, ctx->n, cudaMemcpyDeviceToHost, ctx->snap_stream));
+    CK(cudaEventRecord(ctx->snap_done, ctx->snap_stream));
+    return RFAST_OK;
+}
+
+int rfast_snapshot_wait(rfast_ctx* ctx) {
+    if (!ctx) return RFAST_EINVAL;
+    if (ctx->snap_stream) CK(cudaStreamSynchronize(ctx->snap_stream));
+    return RFAST_OK;
+}
 
 int rfast_seek(rfast_ctx* ctx, int32_t round) {
     if (!ctx) return RFAST_EINVAL;

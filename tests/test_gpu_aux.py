@@ -170,3 +170,29 @@ def test_bounded_copy_wait_of_the_one_pass_kernel_reports_timeout_and_recovers(r
         eng.run()
         x = eng.read(B.STATE_X)
     assert np.linalg.norm(x - orc.X()) <= 1e-5 * np.linalg.norm(orc.X())
+
+
+def test_snapshot_equals_read_state_and_survives_what_follows(rfast_lib):
+    """rfast_snapshot: x and y as of the call, delivered while the handle already does other work."""
+    import torch
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("quad_tree64", seed=8, n=16, p=70_001, K=30)
+    xs = [torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy() for _ in range(2)]
+    ys = [torch.empty((wl.n, wl.p), dtype=torch.float32, pin_memory=True).numpy() for _ in range(2)]
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(wl.schedule)
+        eng.run(11)
+        x11, y11 = eng.read(B.STATE_X), eng.read(B.STATE_Y)
+        eng.snapshot(xs[0], ys[0])
+        eng.run(sync=False)                          # the state moves on at once
+        eng.snapshot(xs[1], ys[1])                   # queues behind the first
+        eng.load_schedule(wl.schedule)               # a new pass starts; the snapshots are not disturbed
+        eng.run(5)
+        eng.snapshot_wait()
+        assert np.array_equal(xs[0], x11) and np.array_equal(ys[0], y11)
+        eng.reset()
+        eng.run()
+        assert np.array_equal(xs[1], eng.read(B.STATE_X)) and np.array_equal(ys[1], eng.read(B.STATE_Y))
+        with pytest.raises(ValueError):
+            eng.snapshot(xs[0][:, :-1], ys[0])
