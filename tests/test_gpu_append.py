@@ -141,3 +141,30 @@ def test_append_needs_an_open_end(rfast_lib):
         with pytest.raises(RFastError) as ei:
             eng.set_option(B.OPT_OPEN_END, 1)                   # mass buckets lump what a later round would split
         assert ei.value.code == EINVAL
+
+
+def test_append_with_empty_parts(rfast_lib):
+    """Degenerate pieces: nothing loaded at first (K = 0), an empty piece in the middle, an empty
+    piece at the end; the result is still the whole schedule's, bit for bit."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    wl = build_config("softmax_exp16", seed=9, F=48, C=5, rows=64, K=60, batch=8)
+    s = wl.schedule
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(s)
+        eng.run()
+        want = eng.read(B.STATE_X), eng.read(B.STATE_Y), eng.read(B.STATE_RHO_LATEST)
+    parts = split_schedule(s, wl.G_R, wl.G_C, [0, 25, 25, s.K])
+    assert [p.K for p in parts] == [0, 25, 0, s.K - 25, 0]
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_OPEN_END, 1)
+        eng.load_schedule(parts[0])
+        x0 = eng.read(B.STATE_X)
+        eng.run()                                            # nothing to run yet
+        assert eng.query(B.Q_ROUND) == 0 and np.array_equal(eng.read(B.STATE_X), x0)
+        for part in parts[1:]:
+            eng.append_schedule(part)
+            eng.run()
+        assert eng.query(B.Q_ROUND) == s.K
+        assert np.array_equal(eng.read(B.STATE_X), want[0]) and np.array_equal(eng.read(B.STATE_Y), want[1])
+        assert np.array_equal(eng.read(B.STATE_RHO_LATEST), want[2])
