@@ -286,3 +286,32 @@ def test_append_check_rejects_inconsistent_parts(rfast_lib):
     with pytest.raises(RFastError) as ei:
         pkg.rfast_compile_append_check(wlb, first, more)
     assert ei.value.code == ESCHED
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_append_check_on_random_general_digraphs(rfast_lib, seed):
+    """Ring plus random chords in both graphs, heavy loss, delays up to 9 rounds, sparse
+    activations (packets wait in inboxes for many rounds), several random cuts: the rows of the
+    loaded rounds never move and the consumed stamps are the whole schedule's."""
+    import paper_2307_11617_b200 as pkg
+    from workloads import activation_bernoulli, make_schedule, split_schedule
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(3, 14))
+    wl = build_config("quad_tree64", seed=seed, n=n, p=8, K=10)
+
+    def edges():
+        e = {(i, (i + 1) % n) for i in range(n)}
+        while len(e) < n + int(rng.integers(0, 2 * n)):
+            a, b = rng.integers(0, n, size=2)
+            if a != b:
+                e.add((int(a), int(b)))
+        return e
+    wl.G_R, wl.G_C = graph_from_edges(n, edges(), "row"), graph_from_edges(n, edges(), "col")
+    K = int(rng.integers(20, 90))
+    s = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, K, float(rng.uniform(0.15, 0.9)), rng),
+                      float(rng.uniform(0.0, 0.7)), int(rng.integers(0, 10)), rng)
+    sv, _ = brute_force_stamps(wl.G_R, s, s.send_r)
+    assert list(pkg.rfast_compile_host(wl, s)["used_tau_v"]) == sv
+    for cut in sorted(set(int(c) for c in rng.integers(0, K + 1, size=4))):
+        first, more = split_schedule(s, wl.G_R, wl.G_C, [cut])
+        pkg.rfast_compile_append_check(wl, first, more)
