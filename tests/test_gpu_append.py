@@ -168,3 +168,44 @@ def test_append_with_empty_parts(rfast_lib):
         assert eng.query(B.Q_ROUND) == s.K
         assert np.array_equal(eng.read(B.STATE_X), want[0]) and np.array_equal(eng.read(B.STATE_Y), want[1])
         assert np.array_equal(eng.read(B.STATE_RHO_LATEST), want[2])
+
+
+@pytest.mark.parametrize("name,ov", [("quad_tree64", dict(n=12, p=5003, K=60)),
+                                     ("softmax_exp16", dict(n=12, F=40, C=5, rows=32, K=60, batch=8))],
+                         ids=["quad", "softmax"])
+def test_append_on_general_digraphs(rfast_lib, name, ov):
+    """Several in- and out-neighbours per node in both graphs, heavy loss and delays up to six
+    rounds: many packets are on their way or waiting in an inbox when a piece ends."""
+    import paper_2307_11617_b200 as pkg
+    from paper_2307_11617_b200 import binding as B
+    from workloads import activation_bernoulli, graph_from_edges, make_schedule
+    wl = build_config(name, seed=21, **ov)
+    rng = np.random.default_rng(22)
+    n = wl.n
+
+    def edges():
+        e = {(i, (i + 1) % n) for i in range(n)}
+        while len(e) < 3 * n:
+            a, b = rng.integers(0, n, size=2)
+            if a != b:
+                e.add((int(a), int(b)))
+        return e
+    wl.G_R, wl.G_C = graph_from_edges(n, edges(), "row"), graph_from_edges(n, edges(), "col")
+    s = make_schedule(wl.G_R, wl.G_C, activation_bernoulli(n, wl.schedule.K, 0.4, rng), 0.4, 6, rng,
+                      batch=wl.batch, rows_per_node=wl.rows)
+    wl.schedule = s
+    with pkg.Engine(wl) as eng:
+        eng.load_schedule(s)
+        eng.run()
+        want = {v: eng.read(getattr(B, v)) for v in ("STATE_X", "STATE_Y", "STATE_RHO_LATEST", "STATE_RHO_BUF", "STATE_TAU_V", "STATE_TAU_RHO")}
+    cuts = [7, 8, 30, 47]
+    parts = split_schedule(s, wl.G_R, wl.G_C, cuts)
+    with pkg.Engine(wl) as eng:
+        eng.set_option(B.OPT_OPEN_END, 1)
+        eng.load_schedule(parts[0])
+        for part in parts[1:]:
+            eng.run()
+            eng.append_schedule(part)
+        eng.run()
+        for v, ref in want.items():
+            assert np.array_equal(eng.read(getattr(B, v)), ref), v
